@@ -1,0 +1,429 @@
+"""CPU oracle for the W4A8 modality-specific static-quantized (MSQ) linear path.
+
+TEST INFRASTRUCTURE ONLY.  This file is the slow, plain definition the CUDA
+kernels are compared against.  It is imported by the tests, by the smoke check
+and by the benchmark's CPU-baseline leg, and by nothing else; the product path
+never calls it and shares no code, table or constant with it.
+
+Every function restates, in NumPy, one step of the method as the paper (MQuant,
+arXiv 2502.00425) defines it, and names the passage it follows.  Quantization
+is not an approximation of something else: the codes ARE the definition, so
+the oracle is the algorithm written out step by step.  Where the paper leaves a
+choice open the reading taken is stated next to the code.
+
+Precision.  The paper fixes no arithmetic type.  Real-valued reference results
+(dense rotation, attention, dequantized outputs) are computed in float64.  The
+decisions that produce an integer (activation and weight codes, the static
+scales the codes depend on) are taken in float32, the precision the kernels use,
+so that both sides round the same number; the float32 fast transform keeps one
+canonical butterfly order for the same reason.
+
+Parity pins (tests/test_oracle_*.py) tie every function to something other than
+itself: integer identities of the Hadamard matrix, the closed form of the first
+transform coefficient (Sec. 3.2, the equation between Eq. 7 and Eq. 9), the
+scale formula of Eq. 2 on hand-made arrays, hand-worked rounding and clamping
+cases, brute-force integer products, the printed index map of App. A.2 and the
+three cases of Eq. 5, and the attention-invariance claim of Sec. 3.1.
+No function here is "parity unpinned".
+"""
+from __future__ import annotations
+
+import numpy as np
+
+TEXT, VISUAL = 0, 1
+INT8_MIN, INT8_MAX = -128, 127
+INT4_MIN, INT4_MAX = -8, 7
+
+
+# ----------------------------------------------------------------------------- bf16
+def bf16_rne(x):
+    """Round float32 values to the nearest bfloat16 (ties to even); returns float32.
+
+    bfloat16 is the upper 16 bits of an IEEE float32, so rounding adds half an
+    ulp of the kept part (plus the parity bit) and truncates."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    u = x.view(np.uint32).astype(np.uint64)
+    r = ((u + 0x7FFF + ((u >> 16) & 1)) >> 16) << 16
+    out = r.astype(np.uint32).view(np.float32).copy()
+    out[np.isnan(x)] = np.float32(np.nan)
+    return out
+
+
+# ----------------------------------------------------------------------------- Hadamard
+def hadamard_matrix(n: int) -> np.ndarray:
+    """Unnormalised Walsh-Hadamard matrix of order n = 2^k with entries +-1.
+
+    App. A.3: H_2 = [[1,1],[1,-1]]/sqrt(2) and H_{2^k} = H_2 (x) H_{2^(k-1)};
+    the 1/sqrt(2) factors are left out here (they collect into 1/sqrt(n))."""
+    if n < 1 or (n & (n - 1)) != 0:
+        raise ValueError("Hadamard order must be a power of two")
+    H = np.ones((1, 1), dtype=np.int64)
+    H2 = np.array([[1, 1], [1, -1]], dtype=np.int64)
+    while H.shape[0] < n:
+        H = np.kron(H2, H)
+    return H
+
+
+def rotate_dense(x, n: int) -> np.ndarray:
+    """Block-diagonal rotation x . (I_{K/n} (x) H_n / sqrt(n)) as a dense float64 product.
+
+    Sec. 3.2 takes H orthonormal (entries 1/sqrt(n)).  The paper defines H only
+    for powers of two; for an input width K that is not one (18944 = 148 x 128)
+    the rotation is read as block-diagonal over consecutive blocks of n columns,
+    which is still orthogonal, so the computational-invariance argument of
+    App. A.14 carries over."""
+    x = np.asarray(x, dtype=np.float64)
+    K = x.shape[-1]
+    if n == 0:
+        return x.copy()
+    if K % n:
+        raise ValueError("K must be a multiple of the rotation block")
+    H = hadamard_matrix(n).astype(np.float64) / np.sqrt(np.float64(n))
+    blocks = x.reshape(x.shape[:-1] + (K // n, n))
+    return (blocks @ H).reshape(x.shape)
+
+
+def fwht_blocks(x, n: int, dtype=np.float32) -> np.ndarray:
+    """Fast Walsh-Hadamard transform of every length-n block of the last axis.
+
+    The fast form of App. A.3's Kronecker recursion: log2(n) butterfly stages
+    with strides h = 1, 2, 4, ..., n/2, each replacing the pair (v[i], v[i+h])
+    (for i with bit h clear) by (v[i] + v[i+h], v[i] - v[i+h]); afterwards one
+    multiplication by 1/sqrt(n) (Sec. 3.2: orthonormal H).  In float32 this is
+    the canonical rounding order: every add/sub and the final multiply rounds
+    once, the normalisation constant is float32(1/sqrt(n))."""
+    x = np.asarray(x)
+    K = x.shape[-1]
+    if n == 0:
+        return x.astype(dtype)
+    if n < 1 or (n & (n - 1)) != 0 or K % n:
+        raise ValueError("rotation block must be a power of two dividing K")
+    v = x.astype(dtype).reshape(-1, K // n, n).copy()
+    h = 1
+    while h < n:
+        w = v.reshape(v.shape[0], v.shape[1], n // (2 * h), 2, h)
+        a = w[:, :, :, 0, :].copy()
+        b = w[:, :, :, 1, :].copy()
+        w[:, :, :, 0, :] = a + b
+        w[:, :, :, 1, :] = a - b
+        h *= 2
+    c = dtype(1.0) / np.sqrt(dtype(n)) if dtype == np.float64 else np.float32(1.0 / np.sqrt(np.float64(n)))
+    v = v * c
+    return v.reshape(x.shape).astype(dtype)
+
+
+# ----------------------------------------------------------------------------- modality table
+def row_modality(T: int, seg_end, seg_mod) -> np.ndarray:
+    """Modality of each row from the segment table (Eq. 3: each contiguous span of
+    the sequence carries the scale of its modality).  A row belongs to the first
+    segment whose exclusive end exceeds it; rows past the last end are text."""
+    out = np.zeros(T, dtype=np.uint8)
+    seg_end = np.asarray(seg_end, dtype=np.int64)
+    for t in range(T):
+        for e, m in zip(seg_end.tolist(), np.asarray(seg_mod).tolist()):
+            if t < e:
+                out[t] = m
+                break
+    return out
+
+
+# ----------------------------------------------------------------------------- scales and quantizers
+def static_scale(values, qmax: int = 127) -> np.float32:
+    """Eq. 2: s = max|x| / (2^(b-1) - 1), in float32.  An empty or all-zero
+    tensor gets s = 1 so that the quantizer stays defined."""
+    values = np.asarray(values, dtype=np.float32)
+    if values.size == 0:
+        return np.float32(1.0)
+    m = np.float32(np.max(np.abs(values)))
+    if not (m > 0):
+        return np.float32(1.0)
+    return np.float32(m / np.float32(qmax))
+
+
+def calibrate_static_scales(x_calib, seg_end, seg_mod, rot_block: int):
+    """MSQ calibration (Sec. 3.1, Eq. 3; Algorithm 1 step 6(b)): one static
+    per-tensor scale for the visual rows and one for the text rows, each the
+    Eq. 2 scale over all calibration values of that modality.  The statistic is
+    taken on the numbers the quantizer will see, i.e. after the online rotation
+    when there is one (the quantizer sits behind the transform in Fig. 4(a))."""
+    x_calib = np.asarray(x_calib, dtype=np.float32)
+    r = fwht_blocks(x_calib, rot_block, np.float32)
+    mod = row_modality(x_calib.shape[0], seg_end, seg_mod)
+    return static_scale(r[mod == VISUAL]), static_scale(r[mod == TEXT])
+
+
+def quantize_act_int8(r, s_rows) -> np.ndarray:
+    """Eq. 2 with z = 0 and b = 8, scale chosen per row by modality (Eq. 3):
+    q = clamp(round(r * (1/s)), -128, 127).
+
+    Readings: symmetric (Eq. 2's own scale formula is the symmetric one);
+    round-to-nearest with ties to even; the clamp covers the full two's-complement
+    range "determined by the bit-width"; the division is done as a multiplication
+    by the float32 reciprocal of s, computed once per scale, since that is what a
+    static-scale kernel does (quantize_act_int8_divide below is the literal x/s).
+    NaN maps to 0 and infinities saturate."""
+    r = np.asarray(r, dtype=np.float32)
+    s_rows = np.asarray(s_rows, dtype=np.float32).reshape(-1, 1)
+    inv = (np.float32(1.0) / s_rows).astype(np.float32)
+    y = (r * inv).astype(np.float32)
+    with np.errstate(invalid="ignore"):
+        q = np.rint(y)
+    q = np.where(np.isnan(q), 0.0, q)
+    return np.clip(q, INT8_MIN, INT8_MAX).astype(np.int8)
+
+
+def quantize_act_int8_divide(r, s_rows) -> np.ndarray:
+    """Eq. 2 literally, with a true float32 division x / s (informational twin)."""
+    r = np.asarray(r, dtype=np.float32)
+    s_rows = np.asarray(s_rows, dtype=np.float32).reshape(-1, 1)
+    with np.errstate(invalid="ignore"):
+        q = np.rint((r / s_rows).astype(np.float32))
+    q = np.where(np.isnan(q), 0.0, q)
+    return np.clip(q, INT8_MIN, INT8_MAX).astype(np.int8)
+
+
+def row_scales(T: int, seg_end, seg_mod, s_vis, s_txt) -> np.ndarray:
+    mod = row_modality(T, seg_end, seg_mod)
+    return np.where(mod == VISUAL, np.float32(s_vis), np.float32(s_txt)).astype(np.float32)
+
+
+def quantize_weight_int4(w):
+    """Per-output-channel symmetric 4-bit round-to-nearest weight quantizer
+    (Eq. 2 with b = 4, z = 0; Algorithm 1 outputs per-channel weight scales).
+    s_w[n] = max_k |W[n,k]| / 7 (1 for an all-zero row); codes clamp to [-8, 7];
+    offline, so the division is the literal one of Eq. 2.  Plain rounding stands
+    in for GPTQ, which needs the paper's calibration data."""
+    w = np.asarray(w, dtype=np.float32)
+    m = np.max(np.abs(w), axis=1).astype(np.float32)
+    s = np.where(m > 0, m / np.float32(7.0), np.float32(1.0)).astype(np.float32)
+    q = np.rint((w / s[:, None]).astype(np.float32))
+    return np.clip(q, INT4_MIN, INT4_MAX).astype(np.int8), s
+
+
+def pack_w4(q) -> np.ndarray:
+    """Two 4-bit two's-complement codes per byte: byte j of row n holds code
+    (n, 2j) in its low nibble and code (n, 2j+1) in its high nibble."""
+    q = np.asarray(q, dtype=np.int8)
+    u = (q.astype(np.int16) & 0xF).astype(np.uint8)
+    return (u[:, 0::2] | (u[:, 1::2] << 4)).astype(np.uint8)
+
+
+def unpack_w4(p) -> np.ndarray:
+    p = np.asarray(p, dtype=np.uint8)
+    lo = (p & 0xF).astype(np.int16)
+    hi = (p >> 4).astype(np.int16)
+    lo = np.where(lo >= 8, lo - 16, lo)
+    hi = np.where(hi >= 8, hi - 16, hi)
+    out = np.empty((p.shape[0], p.shape[1] * 2), dtype=np.int8)
+    out[:, 0::2] = lo
+    out[:, 1::2] = hi
+    return out
+
+
+# ----------------------------------------------------------------------------- GEMM and dequant
+def int_gemm(qx, qw) -> np.ndarray:
+    """acc[t,n] = sum_k qx[t,k] * qw[n,k] as exact integers.
+
+    The products are formed by a float64 matrix multiplication (a library
+    primitive used as one step): every partial sum is an integer far below 2^53
+    (|acc| <= 128 * 8 * K), so float64 represents it exactly."""
+    qx = np.asarray(qx)
+    qw = np.asarray(qw)
+    K = qx.shape[1]
+    if 128.0 * 128.0 * K >= 2.0 ** 53:
+        raise ValueError("K too large for exact float64 accumulation")
+    acc = qx.astype(np.float64) @ qw.astype(np.float64).T
+    out = acc.astype(np.int64)
+    if np.any(np.abs(out) > 2 ** 31 - 1):
+        raise OverflowError("int32 accumulator overflow")
+    return out.astype(np.int32)
+
+
+def int_gemm_loops(qx, qw) -> np.ndarray:
+    """The same sum as three nested loops over Python integers (tiny shapes only)."""
+    T, K = np.shape(qx)
+    N = np.shape(qw)[0]
+    qx = np.asarray(qx).tolist()
+    qw = np.asarray(qw).tolist()
+    out = np.zeros((T, N), dtype=np.int64)
+    for t in range(T):
+        for n in range(N):
+            a = 0
+            for k in range(K):
+                a += qx[t][k] * qw[n][k]
+            out[t, n] = a
+    return out
+
+
+def dequant(acc, s_rows, s_w, bias=None, dtype=np.float64) -> np.ndarray:
+    """y[t,n] = acc[t,n] * (s_a(t) * s_w[n]) (+ bias[n]): Eq. 2's "multiply the
+    integers back by the scale" for both operands of the product at once.
+    dtype=float32 reproduces the kernel's rounding order (scale product first)."""
+    acc = np.asarray(acc)
+    s_rows = np.asarray(s_rows, dtype=np.float32).astype(dtype).reshape(-1, 1)
+    s_w = np.asarray(s_w, dtype=np.float32).astype(dtype).reshape(1, -1)
+    y = acc.astype(dtype) * (s_rows * s_w).astype(dtype)
+    y = y.astype(dtype)
+    if bias is not None:
+        y = (y + np.asarray(bias, dtype=np.float32).astype(dtype).reshape(1, -1)).astype(dtype)
+    return y
+
+
+def linear_w4a8_msq(x, seg_end, seg_mod, s_vis, s_txt, rot_block, qw, s_w, bias=None):
+    """The whole hot path on one activation tile (Sec. 3.1 + Fig. 4(a)):
+    rotate -> per-modality static int8 quantize -> integer GEMM against the 4-bit
+    weight codes -> dequantize -> bfloat16.  Returns every intermediate."""
+    x = np.asarray(x, dtype=np.float32)
+    T = x.shape[0]
+    r = fwht_blocks(x, rot_block, np.float32)
+    s_rows = row_scales(T, seg_end, seg_mod, s_vis, s_txt)
+    qx = quantize_act_int8(r, s_rows)
+    acc = int_gemm(qx, qw)
+    y64 = dequant(acc, s_rows, s_w, bias, np.float64)
+    y32 = dequant(acc, s_rows, s_w, bias, np.float32)
+    return {"rotated": r, "s_rows": s_rows, "qx": qx, "acc": acc, "y64": y64, "y32": y32,
+            "y_bf16": bf16_rne(y32)}
+
+
+# ----------------------------------------------------------------------------- AIFS
+def aifs_perm(is_visual, is_pad=None) -> np.ndarray:
+    """AIFS order (Sec. 3.1; App. A.2: AIFS(1..L) = (m..n, 1..m-1, n+1..L)):
+    all visual tokens first, in their original order, then all text tokens in
+    their original order.  Generalised to any number of visual spans (the
+    paper's own prompts interleave three images).  Left-pad tokens of a batched
+    sequence travel with the visual block (App. A.4)."""
+    is_visual = np.asarray(is_visual).astype(bool)
+    first = is_visual.copy()
+    if is_pad is not None:
+        first |= np.asarray(is_pad).astype(bool)
+    idx = np.arange(is_visual.shape[0], dtype=np.int32)
+    return np.concatenate([idx[first], idx[~first]]).astype(np.int32)
+
+
+def inverse_perm(perm) -> np.ndarray:
+    perm = np.asarray(perm)
+    inv = np.empty_like(perm)
+    inv[perm] = np.arange(perm.shape[0], dtype=perm.dtype)
+    return inv
+
+
+def aifs_gather(x, perm) -> np.ndarray:
+    """E^u[i] = E[perm[i]]."""
+    return np.asarray(x)[np.asarray(perm)]
+
+
+def aifs_scatter(x_u, perm) -> np.ndarray:
+    """Inverse of aifs_gather: out[perm[i]] = x_u[i]."""
+    x_u = np.asarray(x_u)
+    out = np.empty_like(x_u)
+    out[np.asarray(perm)] = x_u
+    return out
+
+
+def remap_positions(perm, pos_ids=None) -> np.ndarray:
+    """App. A.2: the rotary embedding of a moved token uses its ORIGINAL index."""
+    perm = np.asarray(perm)
+    if pos_ids is None:
+        pos_ids = np.arange(perm.shape[0], dtype=np.int32)
+    return np.asarray(pos_ids)[perm].astype(np.int32)
+
+
+def causal_mask(L: int) -> np.ndarray:
+    """Eq. 4 as a boolean "may attend" matrix: allowed(i,j) <=> j <= i."""
+    i = np.arange(L)[:, None]
+    j = np.arange(L)[None, :]
+    return j <= i
+
+
+def unified_mask(perm, is_pad=None) -> np.ndarray:
+    """The unified causal mask M^u of Eq. 5 for an arbitrary interleaving:
+    row i (original token perm[i]) may attend column j (original token perm[j])
+    iff perm[j] <= perm[i], i.e. iff it could in the original order (Eq. 4).
+    Padded tokens are attended by nobody (App. A.4); a pad row keeps its own
+    diagonal so its (discarded) softmax stays defined."""
+    perm = np.asarray(perm, dtype=np.int64)
+    allowed = perm[None, :] <= perm[:, None]
+    if is_pad is not None:
+        pad_u = np.asarray(is_pad).astype(bool)[perm]
+        allowed = allowed & ~pad_u[None, :]
+        allowed = allowed | (np.eye(perm.shape[0], dtype=bool) & pad_u[:, None])
+    return allowed
+
+
+def unified_mask_single_span(m: int, n: int, L: int) -> np.ndarray:
+    """Eq. 5 case by case for ONE visual span at 1-based original positions m..n.
+
+    With N_v = n - m + 1 visual tokens first, then the m-1 leading text tokens,
+    then the trailing text (1-based unified indices i, j):
+      visual row   (i <= N_v):        j <= i, or j among the leading text (N_v < j <= n);
+      leading text (N_v < i <= n):    N_v < j <= i;
+      trailing     (i > n):           j <= i.
+    (The printed equation writes n - m for the visual count; with inclusive
+    bounds m..n the count is n - m + 1, which is the value used here.)"""
+    nv = n - m + 1
+    allowed = np.zeros((L, L), dtype=bool)
+    for i in range(1, L + 1):
+        for j in range(1, L + 1):
+            if i <= nv:
+                ok = (j <= i) or (nv < j <= n)
+            elif i <= n:
+                ok = nv < j <= i
+            else:
+                ok = j <= i
+            allowed[i - 1, j - 1] = ok
+    return allowed
+
+
+def segments_after_aifs(perm, is_visual, is_pad=None):
+    """Segment table of the reordered rows: [visual (and pad) block][text block]."""
+    first = np.asarray(is_visual).astype(bool)
+    if is_pad is not None:
+        first = first | np.asarray(is_pad).astype(bool)
+    n_first = int(first.sum())
+    L = int(np.asarray(perm).shape[0])
+    return np.array([n_first, L], dtype=np.int32), np.array([VISUAL, TEXT], dtype=np.uint8)
+
+
+# ----------------------------------------------------------------------------- attention checker
+def rope(x, pos_ids, base: float = 10000.0) -> np.ndarray:
+    """Rotary position embedding of App. A.2: consecutive channel pairs
+    (2i, 2i+1) are rotated by angle pos * theta_i, theta_i = base^(-2i/D),
+    i = 0..D/2-1.  float64; x is [L, D]."""
+    x = np.asarray(x, dtype=np.float64)
+    L, D = x.shape
+    theta = base ** (-2.0 * np.arange(D // 2, dtype=np.float64) / D)
+    ang = np.asarray(pos_ids, dtype=np.float64)[:, None] * theta[None, :]
+    c, s = np.cos(ang), np.sin(ang)
+    out = np.empty_like(x)
+    out[:, 0::2] = x[:, 0::2] * c - x[:, 1::2] * s
+    out[:, 1::2] = x[:, 0::2] * s + x[:, 1::2] * c
+    return out
+
+
+def attention(q, k, v, allowed) -> np.ndarray:
+    """Softmax(Q K^T / sqrt(D) + M) V with M = 0 where allowed, -inf elsewhere
+    (Eq. 4 / Eq. 5), single head, float64."""
+    q = np.asarray(q, dtype=np.float64)
+    k = np.asarray(k, dtype=np.float64)
+    v = np.asarray(v, dtype=np.float64)
+    s = q @ k.T / np.sqrt(np.float64(q.shape[1]))
+    s = np.where(allowed, s, -np.inf)
+    s = s - s.max(axis=1, keepdims=True)
+    p = np.exp(s)
+    p /= p.sum(axis=1, keepdims=True)
+    return p @ v
+
+
+# ----------------------------------------------------------------------------- helpers for neighbouring steps
+def rotate_weight_input_dim(w, n: int) -> np.ndarray:
+    """Offline counterpart of the online rotation: W' = W . blockdiag(H_n/sqrt(n))
+    along the input dimension, float64, so that (x H)(W H)^T = x W^T (App. A.14)."""
+    return rotate_dense(np.asarray(w, dtype=np.float64), n)
+
+
+def quantize_act_int8_dynamic(r):
+    """Per-token dynamic A8 (the baseline MSQ replaces, Sec. 1): every row gets
+    its own Eq. 2 scale from its own abs-max."""
+    r = np.asarray(r, dtype=np.float32)
+    s = np.array([static_scale(row) for row in r], dtype=np.float32)
+    return quantize_act_int8(r, s), s

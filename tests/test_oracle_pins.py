@@ -1,0 +1,401 @@
+"""Pins for the CPU oracle: each function is tied to something other than itself
+(integer identities, closed forms, hand-worked cases, brute force, the paper's
+printed maps), chosen so that a dropped term, a wrong sign or index or a
+transposed operand fails at least one of them.  CPU only."""
+import itertools
+import os
+
+import numpy as np
+import pytest
+
+from oracle import mq_oracle as O
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _read_ints(name):
+    rows = []
+    with open(os.path.join(GOLD, name)) as f:
+        for line in f:
+            line = line.strip()
+            if line and not line.startswith("#"):
+                rows.append([int(v) for v in line.split()])
+    return rows
+
+
+# ----------------------------------------------------------------------------- Hadamard / FWHT (App. A.3, Sec. 3.2)
+def test_hadamard_h4_matches_hand_written_fixture():
+    assert np.array_equal(O.hadamard_matrix(4), np.array(_read_ints("hadamard_h4.txt")))
+
+
+@pytest.mark.parametrize("n", [1, 2, 4, 8, 16, 32, 64])
+def test_hadamard_gram_is_n_identity_in_integers(n):
+    H = O.hadamard_matrix(n)
+    assert set(np.unique(H).tolist()) <= {-1, 1}
+    assert np.array_equal(H @ H.T, n * np.eye(n, dtype=np.int64))
+    assert np.array_equal(H, H.T)
+    # Sylvester closed form: H[i,j] = (-1)^popcount(i & j)
+    i, j = np.meshgrid(np.arange(n), np.arange(n), indexing="ij")
+    pc = np.vectorize(lambda v: bin(v).count("1"))(i & j)
+    assert np.array_equal(H, np.where(pc % 2 == 0, 1, -1))
+
+
+@pytest.mark.parametrize("n", [2, 4, 8, 16, 32, 64, 128])
+@pytest.mark.parametrize("dtype", [np.float32, np.float64])
+def test_fwht_equals_dense_hadamard_product(n, dtype):
+    rng = np.random.default_rng(n)
+    x = rng.standard_normal((5, 3 * n)).astype(np.float32)
+    fast = O.fwht_blocks(x, n, dtype).astype(np.float64)
+    dense = O.rotate_dense(x, n)
+    tol = (1e-6 if dtype == np.float32 else 1e-13) * np.abs(x).max() * np.sqrt(n)
+    assert np.max(np.abs(fast - dense)) <= tol
+
+
+def test_fwht_unit_impulse_gives_hadamard_columns():
+    n = 16
+    H = O.hadamard_matrix(n) / np.sqrt(n)
+    for j in range(n):
+        e = np.zeros((1, n), np.float32)
+        e[0, j] = 1.0
+        assert np.allclose(O.fwht_blocks(e, n, np.float64)[0], H[j], atol=1e-15)
+
+
+def test_fwht_first_coefficient_is_sqrt_n_times_mean():
+    # Sec. 3.2: (H W)_{0j} = sqrt(n) * mean(w_{:,j}) for the normalised transform,
+    # = sum_r w_{rj} without the normalisation (App. A.3).
+    rng = np.random.default_rng(7)
+    n = 128
+    x = rng.standard_normal((4, 2 * n))
+    y = O.fwht_blocks(x, n, np.float64)
+    for b in range(2):
+        blk = x[:, b * n:(b + 1) * n]
+        assert np.allclose(y[:, b * n], np.sqrt(n) * blk.mean(axis=1), rtol=1e-12)
+        assert np.allclose(y[:, b * n] * np.sqrt(n), blk.sum(axis=1), rtol=1e-12)
+
+
+def test_fwht_preserves_norm_and_is_an_involution():
+    rng = np.random.default_rng(8)
+    x = rng.standard_normal((6, 256))
+    y = O.fwht_blocks(x, 64, np.float64)
+    assert np.allclose(np.linalg.norm(y, axis=1), np.linalg.norm(x, axis=1), rtol=1e-12)
+    assert np.allclose(O.fwht_blocks(y, 64, np.float64), x, atol=1e-12)
+    y32 = O.fwht_blocks(x.astype(np.float32), 64, np.float32)
+    assert np.allclose(np.linalg.norm(y32, axis=1), np.linalg.norm(x, axis=1), rtol=1e-5)
+
+
+def test_fwht_blocks_are_independent_and_ordered():
+    # a value in block 1 must not leak into block 0, and block b lands at columns b*n..
+    n = 8
+    x = np.zeros((1, 3 * n), np.float32)
+    x[0, n + 2] = 1.0
+    y = O.fwht_blocks(x, n, np.float64)
+    assert np.all(y[0, :n] == 0) and np.all(y[0, 2 * n:] == 0)
+    assert np.allclose(y[0, n:2 * n], O.hadamard_matrix(n)[2] / np.sqrt(n))
+
+
+def test_fwht_float32_exact_on_small_integers():
+    # sums of small integers are exact in float32, so with n a power of four the
+    # float32 transform equals the integer transform divided by sqrt(n) exactly.
+    n = 64
+    rng = np.random.default_rng(3)
+    x = rng.integers(-8, 9, size=(3, n)).astype(np.float32)
+    want = (x.astype(np.int64) @ O.hadamard_matrix(n)) / 8.0
+    assert np.array_equal(O.fwht_blocks(x, n, np.float32).astype(np.float64), want)
+
+
+def test_rotation_off_is_identity():
+    x = np.arange(12, dtype=np.float32).reshape(3, 4)
+    assert np.array_equal(O.fwht_blocks(x, 0), x)
+    assert np.array_equal(O.rotate_dense(x, 0), x)
+
+
+# ----------------------------------------------------------------------------- scales (Eq. 2, Eq. 3)
+def test_static_scale_closed_form():
+    x = np.array([[0.5, -3.0, 2.0], [1.0, 254.0, -7.0]], np.float32)
+    assert O.static_scale(x) == np.float32(2.0)            # 254 / 127
+    assert O.static_scale(np.array([-63.5], np.float32)) == np.float32(0.5)
+    assert O.static_scale(np.zeros(4, np.float32)) == np.float32(1.0)
+    assert O.static_scale(np.zeros(0, np.float32)) == np.float32(1.0)
+    assert O.static_scale(np.array([7.0, -3.5], np.float32), qmax=7) == np.float32(1.0)
+
+
+def test_calibration_is_per_modality_and_after_rotation():
+    # rows 0..1 visual, row 2 text; rotation block 4 turns [a,a,a,a] into [2a,0,0,0]
+    x = np.array([[1, 1, 1, 1], [-3, -3, -3, -3], [0.25, 0.25, 0.25, 0.25]], np.float32)
+    s_v, s_t = O.calibrate_static_scales(x, [2, 3], [1, 0], 4)
+    assert s_v == np.float32(6.0 / 127.0) and s_t == np.float32(0.5 / 127.0)
+    s_v0, s_t0 = O.calibrate_static_scales(x, [2, 3], [1, 0], 0)
+    assert s_v0 == np.float32(3.0 / 127.0) and s_t0 == np.float32(0.25 / 127.0)
+    # the element that sets the scale quantizes to +-127 exactly
+    r = O.fwht_blocks(x, 4)
+    q = O.quantize_act_int8(r, O.row_scales(3, [2, 3], [1, 0], s_v, s_t))
+    assert q[1, 0] == -127 and q[2, 0] == 127 and q[0, 0] == 42  # 2/6*127 = 42.33
+
+
+def test_calibration_missing_modality_gives_one():
+    x = np.ones((2, 4), np.float32)
+    s_v, s_t = O.calibrate_static_scales(x, [2], [0], 0)
+    assert s_v == np.float32(1.0) and s_t == np.float32(1.0 / 127.0)
+
+
+def test_row_modality_lookup():
+    assert O.row_modality(6, [2, 5], [1, 0]).tolist() == [1, 1, 0, 0, 0, 0]
+    assert O.row_modality(5, [1, 3, 5], [0, 1, 0]).tolist() == [0, 1, 1, 0, 0]
+    assert O.row_modality(3, [], []).tolist() == [0, 0, 0]
+
+
+# ----------------------------------------------------------------------------- activation quantizer (Eq. 2)
+def test_act_quantizer_hand_cases():
+    s = np.float32(0.5)  # a power of two: r/s is exact
+    r = np.array([[0.0, 0.5, -0.5, 1.0, 63.5, -64.0, 100.0, -100.0,
+                   0.25, 0.75, 1.25, -0.25, -0.75, 0.26, np.inf, -np.inf, np.nan]], np.float32)
+    q = O.quantize_act_int8(r, [s])
+    #   ties go to the even code: 0.5->0, 1.5->2, 2.5->2, -0.5->-0, -1.5->-2
+    assert q.tolist() == [[0, 1, -1, 2, 127, -128, 127, -128, 0, 2, 2, 0, -2, 1, 127, -128, 0]]
+    assert np.array_equal(O.quantize_act_int8_divide(r, [s]), q)
+
+
+def test_act_quantizer_exact_multiples_error_bound_and_idempotence():
+    rng = np.random.default_rng(5)
+    s = np.float32(0.037)
+    k = np.arange(-128, 128, dtype=np.float32)
+    assert np.array_equal(O.quantize_act_int8((k * s).reshape(1, -1), [s])[0], k.astype(np.int8))
+    r = rng.uniform(-127 * s, 127 * s, size=(4, 500)).astype(np.float32)
+    q = O.quantize_act_int8(r, np.full(4, s))
+    assert np.max(np.abs(q.astype(np.float64) * s - r)) <= 0.5 * s * (1 + 1e-5)
+    rq = (q.astype(np.float32) * s).astype(np.float32)
+    assert np.array_equal(O.quantize_act_int8(rq, np.full(4, s)), q)
+
+
+def test_act_quantizer_uses_the_row_scale():
+    r = np.array([[10.0, -10.0], [10.0, -10.0]], np.float32)
+    q = O.quantize_act_int8(r, O.row_scales(2, [1, 2], [1, 0], 1.0, 0.25))
+    assert q.tolist() == [[10, -10], [40, -40]]
+
+
+# ----------------------------------------------------------------------------- weight quantizer and packing
+def test_weight_quantizer_hand_cases():
+    w = np.array([[7.0, -3.5, 0.49, 0.51, -7.0, 1.5, 2.5, 0.0],
+                  [0, 0, 0, 0, 0, 0, 0, 0],
+                  [-14.0, 14.0, 1.0, 3.0, -1.0, 5.0, -15.9, 16.0]], np.float32)
+    q, s = O.quantize_weight_int4(w)
+    assert s.tolist() == [1.0, 1.0, np.float32(16.0 / 7.0)]
+    assert q[0].tolist() == [7, -4, 0, 1, -7, 2, 2, 0]     # -3.5 -> -4 and 2.5 -> 2: ties to even
+    assert q[1].tolist() == [0] * 8
+    assert q[2].tolist() == [-6, 6, 0, 1, 0, 2, -7, 7]
+    assert q.min() >= -8 and q.max() <= 7
+
+
+def test_weight_error_bound():
+    rng = np.random.default_rng(9)
+    w = rng.standard_normal((16, 64)).astype(np.float32)
+    q, s = O.quantize_weight_int4(w)
+    assert np.max(np.abs(q * s[:, None].astype(np.float64) - w) / s[:, None]) <= 0.5 + 1e-5
+
+
+def test_pack_layout_and_roundtrip_over_all_byte_values():
+    q = np.array([[-8, 7, 1, -1]], np.int8)
+    p = O.pack_w4(q)
+    assert p.tolist() == [[0x78, 0xF1]]                    # low nibble = even k
+    allb = np.arange(256, dtype=np.uint8).reshape(1, 256)
+    codes = O.unpack_w4(allb)
+    assert codes.min() == -8 and codes.max() == 7
+    assert np.array_equal(O.pack_w4(codes), allb)
+    # byte 0xF8 = low nibble 8 (-8), high nibble 15 (-1)
+    assert O.unpack_w4(np.array([[0xF8]], np.uint8)).tolist() == [[-8, -1]]
+
+
+# ----------------------------------------------------------------------------- integer GEMM
+def test_int_gemm_against_python_loops_and_structure():
+    rng = np.random.default_rng(11)
+    qx = rng.integers(-128, 128, size=(5, 24)).astype(np.int8)
+    qw = rng.integers(-8, 8, size=(7, 24)).astype(np.int8)
+    acc = O.int_gemm(qx, qw)
+    assert acc.dtype == np.int32 and acc.shape == (5, 7)
+    assert np.array_equal(acc, O.int_gemm_loops(qx, qw))
+    # an all-ones activation row returns the weight row sums (catches a transposed operand)
+    ones = np.ones((1, 24), np.int8)
+    assert np.array_equal(O.int_gemm(ones, qw)[0], qw.astype(np.int64).sum(axis=1))
+    assert np.max(np.abs(acc)) <= 128 * 8 * 24
+
+
+def test_int_gemm_extreme_values_exact():
+    K = 4096
+    qx = np.full((2, K), -128, np.int8)
+    qw = np.full((3, K), -8, np.int8)
+    assert np.all(O.int_gemm(qx, qw) == 128 * 8 * K)
+
+
+# ----------------------------------------------------------------------------- dequant
+def test_dequant_exact_with_power_of_two_scales():
+    acc = np.array([[3, -5], [1 << 20, 7]], np.int32)
+    y = O.dequant(acc, [0.5, 0.25], [2.0, 0.125], bias=[1.0, -1.0], dtype=np.float32)
+    assert y.tolist() == [[4.0, -1.3125], [524289.0, -0.78125]]
+    assert np.array_equal(O.dequant(acc, [0.5, 0.25], [2.0, 0.125], bias=[1.0, -1.0]), y.astype(np.float64))
+
+
+def test_bf16_rne_hand_cases():
+    f = lambda bits: np.array([bits], np.uint32).view(np.float32)
+    assert O.bf16_rne(f(0x3F808000)).view(np.uint32)[0] == 0x3F800000   # tie -> even (down)
+    assert O.bf16_rne(f(0x3F818000)).view(np.uint32)[0] == 0x3F820000   # tie -> even (up)
+    assert O.bf16_rne(f(0x3F808001)).view(np.uint32)[0] == 0x3F810000   # above the tie
+    assert O.bf16_rne(f(0x3F807FFF)).view(np.uint32)[0] == 0x3F800000
+    assert O.bf16_rne(np.array([1.0, -2.5, 0.0], np.float32)).tolist() == [1.0, -2.5, 0.0]
+
+
+# ----------------------------------------------------------------------------- whole linear
+def test_rotation_invariance_without_quantization():
+    # App. A.14 (computational invariance): (x H)(W H)^T = x W^T for orthogonal H
+    rng = np.random.default_rng(13)
+    x = rng.standard_normal((6, 256))
+    w = rng.standard_normal((5, 256))
+    lhs = O.rotate_dense(x, 128) @ O.rotate_weight_input_dim(w, 128).T
+    assert np.allclose(lhs, x @ w.T, rtol=1e-11, atol=1e-11)
+
+
+def test_linear_quantization_error_bound_and_msq_benefit():
+    from paper_2502_00425_b200 import synth
+    c = synth.config1()
+    qw, s_w = O.quantize_weight_int4(c.w)
+    s_v, s_t = O.calibrate_static_scales(c.x_calib, c.seg_calib.seg_end, c.seg_calib.seg_mod, 0)
+    out = O.linear_w4a8_msq(c.x, c.seg.seg_end, c.seg.seg_mod, s_v, s_t, 0, qw, s_w)
+    exact = c.x.astype(np.float64) @ c.w.astype(np.float64).T
+    # |y - xW^T| <= sum_k (|x| s_w/2 + |w| s_a/2 + s_a s_w/4): half a step on each operand
+    s_a = out["s_rows"].astype(np.float64)[:, None]
+    bound = (np.abs(c.x).astype(np.float64) @ (np.ones_like(c.w, dtype=np.float64) * (s_w[:, None] / 2)).T
+             + s_a / 2 * np.abs(c.w).astype(np.float64).sum(axis=1)[None, :]
+             + c.K * s_a * s_w[None, :] / 4)
+    assert np.all(np.abs(out["y64"] - exact) <= bound * (1 + 1e-6))
+    assert np.abs(out["qx"]).max() == 127                  # scales came from these rows: no clipping
+    # Sec. 3.1 advantage (3): with one shared scale the text rows lose resolution
+    s_one = max(s_v, s_t)
+    shared = O.linear_w4a8_msq(c.x, c.seg.seg_end, c.seg.seg_mod, s_one, s_one, 0, qw, s_w)
+    txt = slice(48, 64)
+    err_msq = np.linalg.norm(out["y64"][txt] - exact[txt])
+    err_one = np.linalg.norm(shared["y64"][txt] - exact[txt])
+    assert err_msq < err_one
+    # float32 dequant and bf16 output stay within the stated tolerances of float64
+    assert np.max(np.abs(out["y32"] - out["y64"]) / np.maximum(np.abs(out["y64"]), 1e-30)) <= 1e-5
+    rel = np.abs(out["y_bf16"].astype(np.float64) - out["y64"]) / np.maximum(np.abs(out["y64"]), 2.0 ** -126)
+    assert rel.max() <= 2.0 ** -8
+
+
+# ----------------------------------------------------------------------------- AIFS (Sec. 3.1, App. A.2, A.4)
+def test_aifs_perm_matches_printed_index_map():
+    (m, n, L), order = _read_ints("aifs_index_map.txt")
+    is_vis = np.zeros(L, np.uint8)
+    is_vis[m - 1:n] = 1
+    perm = O.aifs_perm(is_vis)
+    assert (perm + 1).tolist() == order
+    assert (perm + 1).tolist() == list(range(m, n + 1)) + list(range(1, m)) + list(range(n + 1, L + 1))
+    inv = O.inverse_perm(perm)
+    assert np.array_equal(perm[inv], np.arange(L)) and np.array_equal(inv[perm], np.arange(L))
+
+
+def test_aifs_perm_is_a_stable_partition_for_many_spans():
+    is_vis = np.array([0, 1, 1, 0, 0, 1, 0, 1, 1, 0], np.uint8)
+    perm = O.aifs_perm(is_vis)
+    assert perm.tolist() == [1, 2, 5, 7, 8, 0, 3, 4, 6, 9]
+    x = np.arange(20).reshape(10, 2)
+    xu = O.aifs_gather(x, perm)
+    assert np.array_equal(xu[:, 0] // 2, perm)
+    assert np.array_equal(O.aifs_scatter(xu, perm), x)
+    assert np.array_equal(O.remap_positions(perm), perm)
+    assert np.array_equal(O.remap_positions(perm, np.arange(10) + 100), perm + 100)
+    se, sm = O.segments_after_aifs(perm, is_vis)
+    assert se.tolist() == [5, 10] and sm.tolist() == [1, 0]
+
+
+@pytest.mark.parametrize("m,n,L", [(3, 5, 8), (1, 4, 6), (4, 7, 7), (2, 2, 5), (1, 5, 5)])
+def test_unified_mask_reduces_to_eq5_cases_for_one_span(m, n, L):
+    is_vis = np.zeros(L, np.uint8)
+    is_vis[m - 1:n] = 1
+    perm = O.aifs_perm(is_vis)
+    assert np.array_equal(O.unified_mask(perm), O.unified_mask_single_span(m, n, L))
+    # and it is the original causal mask seen through the permutation
+    assert np.array_equal(O.unified_mask(perm), O.causal_mask(L)[np.ix_(perm, perm)])
+
+
+def test_causal_mask_is_lower_triangular():
+    assert np.array_equal(O.causal_mask(4), np.tril(np.ones((4, 4), bool)))
+
+
+def _attn_case(rng, is_vis, is_pad=None, D=8):
+    L = len(is_vis)
+    q, k, v = (rng.standard_normal((L, D)) for _ in range(3))
+    pos = np.arange(L)
+    allowed = O.causal_mask(L)
+    if is_pad is not None:
+        padb = np.asarray(is_pad).astype(bool)
+        allowed = (allowed & ~padb[None, :]) | (np.eye(L, dtype=bool) & padb[:, None])
+    ref = O.attention(O.rope(q, pos), O.rope(k, pos), v, allowed)
+    perm = O.aifs_perm(is_vis, is_pad)
+    pos_u = O.remap_positions(perm, pos)
+    out_u = O.attention(O.rope(q[perm], pos_u), O.rope(k[perm], pos_u), v[perm], O.unified_mask(perm, is_pad))
+    return ref, out_u, perm
+
+
+@pytest.mark.parametrize("pattern", ["tvt", "vt", "tv", "tvtvtvt", "t", "v"])
+def test_aifs_attention_is_invariant(pattern):
+    # Sec. 3.1: with the unified mask and the original position ids, attention on the
+    # reordered sequence equals attention on the original one (here: 1e-5 in float64).
+    rng = np.random.default_rng(len(pattern))
+    is_vis = np.concatenate([np.full(rng.integers(1, 6), 1 if ch == "v" else 0) for ch in pattern]).astype(np.uint8)
+    ref, out_u, perm = _attn_case(rng, is_vis)
+    assert np.max(np.abs(out_u - ref[perm])) <= 1e-5
+    assert np.max(np.abs(O.aifs_scatter(out_u, perm) - ref)) <= 1e-5
+
+
+def test_aifs_attention_with_left_pads():
+    # App. A.4: left pads travel with the visual block and nobody attends to them
+    rng = np.random.default_rng(42)
+    is_pad = np.array([1, 1, 1, 0, 0, 0, 0, 0, 0, 0], np.uint8)
+    is_vis = np.array([0, 0, 0, 0, 0, 1, 1, 1, 0, 0], np.uint8)
+    ref, out_u, perm = _attn_case(rng, is_vis, is_pad)
+    assert perm.tolist() == [0, 1, 2, 5, 6, 7, 3, 4, 8, 9]
+    real = ~is_pad.astype(bool)[perm]
+    assert np.max(np.abs(out_u[real] - ref[perm][real])) <= 1e-5
+    m = O.unified_mask(perm, is_pad)
+    assert not m[real][:, ~real].any()
+
+
+def test_wrong_positions_break_the_invariance():
+    # planting the mistake "positions follow the new order" must be visible
+    rng = np.random.default_rng(1)
+    is_vis = np.array([0, 0, 1, 1, 1, 0, 0], np.uint8)
+    L, D = 7, 8
+    q, k, v = (rng.standard_normal((L, D)) for _ in range(3))
+    pos = np.arange(L)
+    ref = O.attention(O.rope(q, pos), O.rope(k, pos), v, O.causal_mask(L))
+    perm = O.aifs_perm(is_vis)
+    bad = O.attention(O.rope(q[perm], pos), O.rope(k[perm], pos), v[perm], O.unified_mask(perm))
+    assert np.max(np.abs(bad - ref[perm])) > 1e-3
+    bad2 = O.attention(O.rope(q[perm], pos[perm]), O.rope(k[perm], pos[perm]), v[perm], O.causal_mask(L))
+    assert np.max(np.abs(bad2 - ref[perm])) > 1e-3
+
+
+def test_rope_is_a_rotation_depending_on_relative_position():
+    rng = np.random.default_rng(2)
+    x = rng.standard_normal((3, 8))
+    assert np.allclose(O.rope(x, [0, 0, 0]), x)
+    assert np.allclose(np.linalg.norm(O.rope(x, [5, 9, 2]), axis=1), np.linalg.norm(x, axis=1))
+    a, b = rng.standard_normal((1, 8)), rng.standard_normal((1, 8))
+    d1 = O.rope(a, [7]) @ O.rope(b, [3]).T
+    d2 = O.rope(a, [14]) @ O.rope(b, [10]).T
+    assert np.allclose(d1, d2)
+    # first pair rotates by pos * theta_0 = pos (theta_0 = base^0 = 1)
+    e = np.zeros((1, 8)); e[0, 0] = 1.0
+    assert np.allclose(O.rope(e, [0.5])[0, :2], [np.cos(0.5), np.sin(0.5)])
+
+
+def test_rms_split_cost_fixture():
+    # Sec. 4.3: one input row split off a K-row GEMM costs 1/K of it
+    for K, N, denom in _read_ints("rms_cost.txt"):
+        assert (2 * 1 * N) * denom == 2 * K * N
+
+
+def test_dynamic_quantizer_uses_row_absmax():
+    r = np.array([[1.0, -2.0], [0.5, 0.25]], np.float32)
+    q, s = O.quantize_act_int8_dynamic(r)
+    assert s.tolist() == [np.float32(2 / 127), np.float32(0.5 / 127)]
+    assert q.tolist() == [[64, -127], [127, 64]]
