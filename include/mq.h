@@ -1,0 +1,212 @@
+/*
+ * mq.h -- C ABI of the B200-native W4A8 modality-specific static-quantized (MSQ)
+ * linear path of MQuant (arXiv 2502.00425).
+ *
+ * Conventions shared by every call
+ * --------------------------------
+ *  - Every function returns an int status (MQ_OK = 0, negative = error) and never
+ *    throws.  mq_status_string() names a status.
+ *  - Unless a parameter says "host", every pointer is DEVICE memory owned by the
+ *    caller.  The library never allocates, frees or keeps device memory; scratch
+ *    comes from a caller-provided workspace sized by mq_workspace_bytes().
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls
+ *    enqueue work on it and return without synchronising, except
+ *    mq_last_device_status(), which waits for the stream.
+ *  - Activations are row-major [rows, cols] with a leading dimension `ld*` counted
+ *    in ELEMENTS.  bf16 activations are the usual upper-16-bits-of-float32 format.
+ *    Base pointers must be 16-byte aligned and row pitches multiples of 16 bytes,
+ *    otherwise MQ_ERR_ALIGNMENT.
+ *  - Weights are W[N,K] (output channel x input channel), so Y = X . W^T.
+ *  - Token modality is given by a segment table (Sec. 3.1, Eq. 3: the text and
+ *    visual spans of the sequence each use their own static scale): row t has the
+ *    modality seg_mod[i] of the first segment i with t < seg_end[i]; rows beyond the
+ *    last end are text.  After AIFS (Sec. 3.1) a sequence has two segments,
+ *    [visual][text]; without AIFS the same calls take one segment per span.
+ *  - Quantization follows Eq. 2 with zero-point 0: codes = clamp(round(x / s)),
+ *    round-to-nearest-even, int8 range [-128,127] for activations and int4 range
+ *    [-8,7] for weights; activation division is a multiplication by the float32
+ *    reciprocal of the static scale.
+ *  - Bad arguments are rejected on the host before anything is enqueued.  Waits
+ *    inside kernels are bounded; if one ever expires the kernel records
+ *    MQ_ERR_TIMEOUT in the workspace status word and returns.
+ */
+#ifndef MQ_H_
+#define MQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define MQ_VERSION 1
+
+/* status codes */
+#define MQ_OK 0
+#define MQ_ERR_INVALID_ARG (-1)
+#define MQ_ERR_UNSUPPORTED (-2)
+#define MQ_ERR_ALIGNMENT (-3)
+#define MQ_ERR_CUDA (-4)
+#define MQ_ERR_TIMEOUT (-5)
+#define MQ_ERR_WORKSPACE (-6)
+
+/* modalities */
+#define MQ_TEXT 0
+#define MQ_VISUAL 1
+
+/* mq_linear_desc.flags */
+#define MQ_FLAG_X_IS_INT8 1u /* X is already int8 codes [T,K]; skip rotation + quantization */
+#define MQ_FLAG_Y_IS_F32 2u  /* write Y as float32 instead of bfloat16 */
+
+/* Rows of the weight tile and columns of the K block of the GEMM weight layout. */
+#define MQ_W_TILE_N 128
+#define MQ_W_TILE_K 128
+
+typedef struct mq_segments {
+  int32_t n_seg;          /* number of segments (>= 0) */
+  const int32_t* seg_end; /* device, [n_seg] exclusive cumulative row ends, non-decreasing */
+  const uint8_t* seg_mod; /* device, [n_seg] MQ_TEXT / MQ_VISUAL */
+} mq_segments;
+
+typedef struct mq_linear_desc {
+  int32_t T;          /* rows (tokens) of X and Y, >= 0 */
+  int32_t K;          /* input channels, multiple of 32 */
+  int32_t N;          /* output channels, multiple of 16 */
+  int32_t rot_block;  /* online Hadamard block: 0 = off, else 32..1024 power of two dividing K */
+  int32_t group_size; /* weight scale group along K: 0 = one scale per output channel */
+  uint32_t flags;     /* MQ_FLAG_* */
+} mq_linear_desc;
+
+int mq_version(void);
+const char* mq_status_string(int status);
+
+/* Bytes of scratch mq_w4a8_msq_linear needs for this problem (0 on a bad desc).
+ * Holds the status word, the int8 activation codes when X arrives as bf16, and
+ * split-K partial accumulators for small T.  The workspace must be 256-byte aligned. */
+size_t mq_workspace_bytes(const mq_linear_desc* d);
+
+/* Bytes of the GEMM weight layout written by mq_pack_w4 / mq_repack_w4 for W[N,K]
+ * (N and K padded up to the 128 x 128 weight tile). */
+size_t mq_w4_layout_bytes(int32_t N, int32_t K);
+
+/*
+ * Static-scale calibration (Sec. 3.1 "single-shot calibration"; Algorithm 1 step 6(b);
+ * Eq. 2: s = max|x| / (2^(b-1) - 1) with b = 8).
+ * For each modality: abs-max over all rows of that modality and all K channels of the
+ * values the quantizer will see -- X after the block Hadamard rotation when rot_block
+ * != 0 -- divided by 127.  A modality with no rows, or whose maximum is 0, gets 1.0f.
+ *   X          bf16 [T,K], leading dimension ldx
+ *   amax_state device uint32[2] owned by the caller: running abs-max bit patterns
+ *              (index 0 text, 1 visual).  accumulate = 0 resets it first; accumulate = 1
+ *              folds this batch into what earlier calls left, so several calibration
+ *              batches give one scale.
+ *   s_vis_out, s_txt_out  device float[1] each, rewritten by every call.
+ */
+int mq_calibrate_static_scales(const void* X, int32_t T, int32_t K, int64_t ldx,
+                               const mq_segments* seg, int32_t rot_block, int32_t accumulate,
+                               uint32_t* amax_state, float* s_vis_out, float* s_txt_out,
+                               void* stream);
+
+/*
+ * Weight quantization and packing (Eq. 2 with b = 4, z = 0; Algorithm 1 outputs
+ * per-channel weight scales; plain round-to-nearest stands in for GPTQ).
+ *   s_w[n] = max_k |W[n,k]| / 7 (1.0f for an all-zero row);
+ *   q[n,k] = clamp(round_half_even(W[n,k] / s_w[n]), -8, 7).
+ *   W       float32 [N,K], leading dimension ldw
+ *   packed  optional (may be NULL) canonical layout uint8 [N, K/2]:
+ *           byte j of row n = (q[n,2j] & 15) | ((q[n,2j+1] & 15) << 4)
+ *   s_w     float32 [N]
+ *   gemm_layout optional (may be NULL) opaque layout consumed by mq_w4a8_msq_linear,
+ *           mq_w4_layout_bytes(N,K) bytes, 128-byte aligned; a pure permutation of the
+ *           canonical nibbles, zero-padded to whole 128 x 128 tiles.
+ * group_size must be 0 (per output channel); other values MQ_ERR_UNSUPPORTED.
+ */
+int mq_pack_w4(const float* W, int32_t N, int32_t K, int64_t ldw, int32_t group_size,
+               uint8_t* packed, float* s_w, void* gemm_layout, void* stream);
+
+/* Canonical [N,K/2] bytes -> GEMM weight layout (same permutation as mq_pack_w4). */
+int mq_repack_w4(const uint8_t* packed, int32_t N, int32_t K, void* gemm_layout, void* stream);
+
+/* Debug inverse: int8 codes q[N,K] (leading dimension ldq) from the canonical bytes
+ * (packed != NULL) or from the GEMM layout (packed == NULL, gemm_layout != NULL). */
+int mq_unpack_w4(const uint8_t* packed, const void* gemm_layout, int32_t N, int32_t K,
+                 int8_t* q_out, int64_t ldq, void* stream);
+
+/*
+ * Attention-Invariant Flexible Switching, token reorder (Sec. 3.1; App. A.2:
+ * AIFS(1..L) = (m..n, 1..m-1, n+1..L); App. A.4 for pads).
+ * direction 0 (gather): builds perm = [indices of visual-or-pad tokens in order,
+ *   then indices of text tokens in order], inv_perm, *n_first_out = size of the first
+ *   block, and X_out[i,:] = X[perm[i],:].
+ * direction 1 (scatter back): reads the given perm and writes X_out[perm[i],:] = X[i,:]
+ *   (is_visual, is_pad, inv_perm, n_first_out are ignored and may be NULL).
+ *   X, X_out   bf16 [L,D] (ldx, ldo); X == X_out is rejected.  Either both NULL
+ *              (index-only call) or both non-NULL.
+ *   is_visual  uint8 [L]; is_pad uint8 [L] or NULL
+ *   perm, inv_perm int32 [L]; n_first_out int32 [1]
+ */
+int mq_aifs_reorder(const void* X, void* X_out, int32_t L, int32_t D, int64_t ldx, int64_t ldo,
+                    const uint8_t* is_visual, const uint8_t* is_pad, int32_t* perm,
+                    int32_t* inv_perm, int32_t* n_first_out, int32_t direction, void* stream);
+
+/*
+ * Causal-mask and position remap for the reordered sequence (Eq. 5; App. A.2: rotary
+ * embeddings keep the ORIGINAL token index; App. A.4: nobody attends to pads).
+ *   pos_ids_out[i] = pos_ids[perm[i]]  (pos_ids NULL = 0,1,2,...)
+ *   seg_end_out[2] = {n_first, L}, seg_mod_out[2] = {MQ_VISUAL, MQ_TEXT}  (may be NULL)
+ *   dense_mask_out optional uint8 [L,L], 1 = row i may attend column j:
+ *       perm[j] <= perm[i] and not pad[perm[j]]  (a pad row keeps its own diagonal).
+ *       Rejected with MQ_ERR_UNSUPPORTED for L > 16384.
+ *   n_first    device int32[1] as written by mq_aifs_reorder (needed for seg_*_out).
+ */
+int mq_attn_mask_remap(const int32_t* perm, const int32_t* pos_ids, const uint8_t* is_pad,
+                       const int32_t* n_first, int32_t L, int32_t* pos_ids_out,
+                       int32_t* seg_end_out, uint8_t* seg_mod_out, uint8_t* dense_mask_out,
+                       void* stream);
+
+/*
+ * Fused online Hadamard rotation + MSQ int8 quantizer (Fig. 4(a): the transform in
+ * front of the down-projection; App. A.3: H_2, H_{2^n} = H_2 (x) H_{2^(n-1)}, applied
+ * here block-diagonally over consecutive blocks of rot_block channels, normalised by
+ * 1/sqrt(rot_block); Eq. 2 / Eq. 3 for the quantizer).
+ *   r = X . blockdiag(H)  in float32: butterflies with strides 1,2,4,...,rot_block/2 in
+ *       that order, then one multiply by float32(1/sqrt(rot_block));
+ *   Q[t,k] = sat_int8(round_half_even(r[t,k] * (1.0f / s_mod(t)))).
+ *   X bf16 [T,K] (ldx);  Q int8 [T,K] (ldq, multiple of 16)
+ *   s_vis, s_txt  host floats, finite and > 0
+ *   rotated_out   optional float32 [T,K] (leading dimension K) dump of r, NULL normally.
+ */
+int mq_fwht_quant_i8(const void* X, int32_t T, int32_t K, int64_t ldx, const mq_segments* seg,
+                     float s_vis, float s_txt, int32_t rot_block, int8_t* Q, int64_t ldq,
+                     float* rotated_out, void* stream);
+
+/*
+ * The W4A8 MSQ linear (Sec. 3.1 MSQ + Fig. 4(a) + Eq. 2):
+ *   Qx  = mq_fwht_quant_i8(X)            (skipped when MQ_FLAG_X_IS_INT8)
+ *   acc[t,n] = sum_k Qx[t,k] * q_w[n,k]  (int32, exact)
+ *   Y[t,n] = float(acc) * (s_mod(t) * s_w[n]) (+ bias[n]), rounded to bf16 (or float32).
+ *   X        bf16 [T,K] or, with MQ_FLAG_X_IS_INT8, int8 [T,K]; leading dimension ldx
+ *   W_layout GEMM weight layout from mq_pack_w4 / mq_repack_w4
+ *   s_w      float32 [N];  bias float32 [N] or NULL
+ *   Y        bf16 (or float32) [T,N], leading dimension ldy
+ *   acc_out  optional int32 [T,N] (leading dimension N) dump of the accumulators
+ *   ws       workspace of at least mq_workspace_bytes(d) bytes, 256-byte aligned
+ * T = 0 is a successful no-op.
+ */
+int mq_w4a8_msq_linear(const mq_linear_desc* d, const void* X, int64_t ldx,
+                       const mq_segments* seg, float s_vis, float s_txt, const void* W_layout,
+                       const float* s_w, const float* bias, void* Y, int64_t ldy,
+                       int32_t* acc_out, void* ws, size_t ws_bytes, void* stream);
+
+/* Waits for `stream`, then returns the status word kernels left in the workspace
+ * (MQ_OK or MQ_ERR_TIMEOUT) and, if site_out != NULL (host), where the wait gave up. */
+int mq_last_device_status(void* ws, void* stream, int32_t* site_out);
+
+/* Clears the status word (enqueued on `stream`). */
+int mq_reset_device_status(void* ws, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MQ_H_ */

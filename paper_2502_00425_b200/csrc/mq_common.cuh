@@ -1,0 +1,87 @@
+// Shared device/host helpers of the MSQ W4A8 kernels (sm_100a only).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "mq.h"
+
+namespace mq {
+
+// ---- workspace layout -------------------------------------------------------------
+// [0,256)   status block: int32 status, int32 site, reserved
+// [256, ..) int8 activation codes (when X arrives as bf16), then split-K accumulators
+constexpr size_t kStatusBytes = 256;
+
+struct SegTable {
+  int n_seg;
+  const int32_t* seg_end;
+  const uint8_t* seg_mod;
+};
+
+__host__ __device__ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Modality of row t, looked up cooperatively by one warp (all 32 lanes must call).
+// Row t belongs to the first segment whose exclusive end exceeds t; text otherwise.
+__device__ __forceinline__ int warp_row_modality(const SegTable& seg, int t) {
+  const int lane = threadIdx.x & 31;
+  for (int base = 0; base < seg.n_seg; base += 32) {
+    const int i = base + lane;
+    const bool hit = (i < seg.n_seg) && (t < seg.seg_end[i]);
+    const unsigned m = __ballot_sync(0xffffffffu, hit);
+    if (m) {
+      const int first = base + __ffs(m) - 1;
+      return seg.seg_mod[first] ? MQ_VISUAL : MQ_TEXT;
+    }
+  }
+  return MQ_TEXT;
+}
+
+// Same lookup by a single thread (used where one thread owns one row / column).
+__device__ __forceinline__ int thread_row_modality(const SegTable& seg, int t) {
+  for (int i = 0; i < seg.n_seg; ++i)
+    if (t < seg.seg_end[i]) return seg.seg_mod[i] ? MQ_VISUAL : MQ_TEXT;
+  return MQ_TEXT;
+}
+
+inline int cuda_status(cudaError_t e) { return e == cudaSuccess ? MQ_OK : MQ_ERR_CUDA; }
+
+// host launchers implemented in the .cu files -----------------------------------------
+int launch_fwht_quant(const void* X, int T, int K, int64_t ldx, SegTable seg, float s_vis,
+                      float s_txt, int rot_block, int8_t* Q, int64_t ldq, float* rotated_out,
+                      cudaStream_t st);
+int launch_calibrate(const void* X, int T, int K, int64_t ldx, SegTable seg, int rot_block,
+                     int accumulate, uint32_t* amax_state, float* s_vis_out, float* s_txt_out,
+                     cudaStream_t st);
+int launch_pack_w4(const float* W, int N, int K, int64_t ldw, uint8_t* packed, float* s_w,
+                   void* layout, cudaStream_t st);
+int launch_repack_w4(const uint8_t* packed, int N, int K, void* layout, cudaStream_t st);
+int launch_unpack_w4(const uint8_t* packed, const void* layout, int N, int K, int8_t* q,
+                     int64_t ldq, cudaStream_t st);
+int launch_aifs_reorder(const void* X, void* X_out, int L, int D, int64_t ldx, int64_t ldo,
+                        const uint8_t* is_visual, const uint8_t* is_pad, int32_t* perm,
+                        int32_t* inv_perm, int32_t* n_first_out, int direction, cudaStream_t st);
+int launch_mask_remap(const int32_t* perm, const int32_t* pos_ids, const uint8_t* is_pad,
+                      const int32_t* n_first, int L, int32_t* pos_out, int32_t* seg_end_out,
+                      uint8_t* seg_mod_out, uint8_t* dense, cudaStream_t st);
+
+struct GemmArgs {
+  int T, K, N;
+  const int8_t* Qx;
+  int64_t ldq;
+  SegTable seg;
+  float s_vis, s_txt;
+  const void* W_layout;
+  const float* s_w;
+  const float* bias;
+  void* Y;
+  int64_t ldy;
+  int y_is_f32;
+  int32_t* acc_out;
+  int32_t* status;     // device int32[2]: status, site
+  int32_t* splitk_acc; // device int32 [T,N] scratch (small-T path) or nullptr
+};
+int launch_gemm(const GemmArgs& a, cudaStream_t st);
+size_t gemm_splitk_bytes(int T, int K, int N);
+
+}  // namespace mq

@@ -1,0 +1,211 @@
+// K1: fused online block-Hadamard rotation + modality-specific static int8 quantizer,
+// and the calibration reduce that shares its front end.
+//
+// Method: Fig. 4(a) (online fast Hadamard transform in front of the down-projection
+// quantizer), App. A.3 (H_2 and the Kronecker recursion), Eq. 2 / Eq. 3 (static
+// per-modality scale, round-to-nearest, clamp).
+//
+// Mapping.  A warp owns 1024 consecutive channels of one row per pass.  A rotation block
+// of n = 32 * TPB channels is held by TPB adjacent lanes, each lane keeping four 16-byte
+// chunks (8 bf16 each): chunk c = i * TPB + j for lane-in-block j and i = 0..3.  With the
+// element index written as  e = r + 8 * (j + TPB * i)  the butterfly strides 1,2,4 act on
+// r (registers), strides 8 .. 4n/32 act on j (warp shuffles) and the last two strides act
+// on i (registers), so the stages run in increasing stride order -- the same rounding
+// sequence as a textbook in-place transform -- with only log2(TPB) shuffle stages.
+// Every global access is a full 16-byte (load) or 8-byte (store) vector and every 32-byte
+// sector touched is used completely; the kernel is bounded by HBM traffic of 3 bytes per
+// element (2 read + 1 written).
+#include "mq_common.cuh"
+
+namespace mq {
+namespace {
+
+constexpr int kWarpsPerCta = 8;
+constexpr int kWarpTile = 1024;  // channels per warp pass
+
+enum Mode { kQuant = 0, kQuantDump = 1, kAbsMax = 2 };
+
+__device__ __forceinline__ uint32_t pack_sat_s8x4(int q0, int q1, int q2, int q3) {
+  // cvt.pack.sat.s8.s32.b32 d, a, b, c : d = { c[15:0], sat8(a), sat8(b) } (b in the low byte)
+  uint32_t hi, out;
+  asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(hi) : "r"(q3), "r"(q2), "r"(0));
+  asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(out) : "r"(q1), "r"(q0), "r"(hi));
+  return out;
+}
+
+template <int LOG_TPB, bool ROT, int MODE>
+__global__ void __launch_bounds__(kWarpsPerCta * 32)
+fwht_quant_kernel(const uint16_t* __restrict__ X, int T, int K, int64_t ldx, SegTable seg,
+                  float inv_vis, float inv_txt, float c_n, int8_t* __restrict__ Q, int64_t ldq,
+                  float* __restrict__ rotated_out, uint32_t* __restrict__ amax_state,
+                  int tiles_per_row, long long n_warp_tiles) {
+  constexpr int TPB = 1 << LOG_TPB;
+  const int lane = threadIdx.x & 31;
+  const int warp = threadIdx.x >> 5;
+  const long long wt = (long long)blockIdx.x * kWarpsPerCta + warp;
+  if (wt >= n_warp_tiles) return;
+  const int row = (int)(wt / tiles_per_row);
+  const int tile = (int)(wt % tiles_per_row);
+  const int j = lane & (TPB - 1);
+  const int blk = lane >> LOG_TPB;
+  const int blk_start = tile * kWarpTile + blk * (32 * TPB);
+
+  float v[4][8];
+  const uint16_t* xrow = X + (int64_t)row * ldx;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int off = blk_start + (i * TPB + j) * 8;
+    uint4 w = make_uint4(0u, 0u, 0u, 0u);
+    if (off < K) w = __ldg(reinterpret_cast<const uint4*>(xrow + off));
+    const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+    for (int p = 0; p < 4; ++p) {
+      v[i][2 * p] = __uint_as_float(ww[p] << 16);
+      v[i][2 * p + 1] = __uint_as_float(ww[p] & 0xffff0000u);
+    }
+  }
+
+  if (ROT) {
+    // strides 1, 2, 4: inside each 8-element chunk
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+#pragma unroll
+      for (int h = 1; h < 8; h <<= 1) {
+#pragma unroll
+        for (int r = 0; r < 8; ++r) {
+          if ((r & h) == 0) {
+            const float a = v[i][r], b = v[i][r + h];
+            v[i][r] = __fadd_rn(a, b);
+            v[i][r + h] = __fsub_rn(a, b);
+          }
+        }
+      }
+    }
+    // strides 8 * 2^b for b < log2(TPB): partner lane j ^ 2^b
+#pragma unroll
+    for (int b = 0; b < LOG_TPB; ++b) {
+      const float sgn = ((j >> b) & 1) ? -1.0f : 1.0f;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+#pragma unroll
+        for (int r = 0; r < 8; ++r) {
+          const float p = __shfl_xor_sync(0xffffffffu, v[i][r], 1 << b);
+          // lower element: own + partner; upper element: partner - own (one rounding)
+          v[i][r] = __fmaf_rn(v[i][r], sgn, p);
+        }
+      }
+    }
+    // strides 8 * TPB and 16 * TPB: across the four chunks of this lane
+#pragma unroll
+    for (int r = 0; r < 8; ++r) {
+      float a0 = v[0][r], a1 = v[1][r], a2 = v[2][r], a3 = v[3][r];
+      float b0 = __fadd_rn(a0, a1), b1 = __fsub_rn(a0, a1);
+      float b2 = __fadd_rn(a2, a3), b3 = __fsub_rn(a2, a3);
+      v[0][r] = __fmul_rn(__fadd_rn(b0, b2), c_n);
+      v[1][r] = __fmul_rn(__fadd_rn(b1, b3), c_n);
+      v[2][r] = __fmul_rn(__fsub_rn(b0, b2), c_n);
+      v[3][r] = __fmul_rn(__fsub_rn(b1, b3), c_n);
+    }
+  }
+
+  const int mod = warp_row_modality(seg, row);
+
+  if (MODE == kAbsMax) {
+    float m = 0.0f;
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int r = 0; r < 8; ++r) m = fmaxf(m, fabsf(v[i][r]));  // fmaxf drops NaN
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if (lane == 0 && m > 0.0f) atomicMax(&amax_state[mod], __float_as_uint(m));
+    return;
+  }
+
+  const float inv = (mod == MQ_VISUAL) ? inv_vis : inv_txt;
+  int8_t* qrow = Q + (int64_t)row * ldq;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int off = blk_start + (i * TPB + j) * 8;
+    if (off >= K) continue;
+    if (MODE == kQuantDump) {
+      float4* dst = reinterpret_cast<float4*>(rotated_out + (int64_t)row * K + off);
+      dst[0] = make_float4(v[i][0], v[i][1], v[i][2], v[i][3]);
+      dst[1] = make_float4(v[i][4], v[i][5], v[i][6], v[i][7]);
+    }
+    int q[8];
+#pragma unroll
+    for (int r = 0; r < 8; ++r) q[r] = __float2int_rn(__fmul_rn(v[i][r], inv));  // NaN -> 0, saturating
+    uint2 o;
+    o.x = pack_sat_s8x4(q[0], q[1], q[2], q[3]);
+    o.y = pack_sat_s8x4(q[4], q[5], q[6], q[7]);
+    *reinterpret_cast<uint2*>(qrow + off) = o;
+  }
+}
+
+__global__ void calib_reset_kernel(uint32_t* amax_state) {
+  if (threadIdx.x < 2) amax_state[threadIdx.x] = 0u;
+}
+
+__global__ void calib_finalize_kernel(const uint32_t* amax_state, float* s_vis_out, float* s_txt_out) {
+  if (threadIdx.x == 0) {
+    const float mt = __uint_as_float(amax_state[MQ_TEXT]);
+    const float mv = __uint_as_float(amax_state[MQ_VISUAL]);
+    *s_txt_out = mt > 0.0f ? __fdiv_rn(mt, 127.0f) : 1.0f;
+    *s_vis_out = mv > 0.0f ? __fdiv_rn(mv, 127.0f) : 1.0f;
+  }
+}
+
+template <int MODE>
+int dispatch(const void* X, int T, int K, int64_t ldx, SegTable seg, float inv_vis, float inv_txt,
+             int rot_block, int8_t* Q, int64_t ldq, float* rotated_out, uint32_t* amax_state,
+             cudaStream_t st) {
+  if (T == 0 || K == 0) return MQ_OK;
+  const int tiles_per_row = (K + kWarpTile - 1) / kWarpTile;
+  const long long n_warp_tiles = (long long)T * tiles_per_row;
+  const long long ctas = (n_warp_tiles + kWarpsPerCta - 1) / kWarpsPerCta;
+  if (ctas > 0x7fffffffLL) return MQ_ERR_UNSUPPORTED;
+  const dim3 grid((unsigned)ctas), block(kWarpsPerCta * 32);
+  const float c_n = rot_block ? (float)(1.0 / sqrt((double)rot_block)) : 1.0f;
+  const uint16_t* x = static_cast<const uint16_t*>(X);
+#define MQ_LAUNCH(LOG_TPB, ROT)                                                              \
+  fwht_quant_kernel<LOG_TPB, ROT, MODE><<<grid, block, 0, st>>>(                             \
+      x, T, K, ldx, seg, inv_vis, inv_txt, c_n, Q, ldq, rotated_out, amax_state, tiles_per_row, \
+      n_warp_tiles)
+  switch (rot_block) {
+    case 0: MQ_LAUNCH(2, false); break;
+    case 32: MQ_LAUNCH(0, true); break;
+    case 64: MQ_LAUNCH(1, true); break;
+    case 128: MQ_LAUNCH(2, true); break;
+    case 256: MQ_LAUNCH(3, true); break;
+    case 512: MQ_LAUNCH(4, true); break;
+    case 1024: MQ_LAUNCH(5, true); break;
+    default: return MQ_ERR_UNSUPPORTED;
+  }
+#undef MQ_LAUNCH
+  return cuda_status(cudaGetLastError());
+}
+
+}  // namespace
+
+int launch_fwht_quant(const void* X, int T, int K, int64_t ldx, SegTable seg, float s_vis,
+                      float s_txt, int rot_block, int8_t* Q, int64_t ldq, float* rotated_out,
+                      cudaStream_t st) {
+  const float inv_vis = 1.0f / s_vis, inv_txt = 1.0f / s_txt;
+  if (rotated_out)
+    return dispatch<kQuantDump>(X, T, K, ldx, seg, inv_vis, inv_txt, rot_block, Q, ldq, rotated_out,
+                                nullptr, st);
+  return dispatch<kQuant>(X, T, K, ldx, seg, inv_vis, inv_txt, rot_block, Q, ldq, nullptr, nullptr, st);
+}
+
+int launch_calibrate(const void* X, int T, int K, int64_t ldx, SegTable seg, int rot_block,
+                     int accumulate, uint32_t* amax_state, float* s_vis_out, float* s_txt_out,
+                     cudaStream_t st) {
+  if (!accumulate) calib_reset_kernel<<<1, 32, 0, st>>>(amax_state);
+  int rc = dispatch<kAbsMax>(X, T, K, ldx, seg, 1.0f, 1.0f, rot_block, nullptr, 0, nullptr, amax_state, st);
+  if (rc != MQ_OK) return rc;
+  calib_finalize_kernel<<<1, 32, 0, st>>>(amax_state, s_vis_out, s_txt_out);
+  return cuda_status(cudaGetLastError());
+}
+
+}  // namespace mq

@@ -1,0 +1,605 @@
+// K2: W4A8 integer GEMM with the MSQ dequant epilogue, written for sm_100a.
+//
+// Method: Eq. 2 (uniform quantizer; the integer product of the codes times both scales
+// reconstructs the real product), Eq. 3 (one static activation scale per modality, looked
+// up per token row), Algorithm 1 (per-output-channel weight scales).
+//   acc[t,n] = sum_k Qx[t,k] * q_w[n,k]      (int8 x int4 -> int32, exact)
+//   Y[t,n]   = float(acc) * (s_mod(t) * s_w[n]) (+ bias[n])
+//
+// Design (differs from a conventional "unpack B into shared memory" GEMM on purpose).
+// On B200 a 128-row tcgen05 MMA reads its shared-memory operands at close to the
+// shared-memory bandwidth of the SM, so re-writing unpacked weights to shared memory
+// would make shared memory, not the tensor pipe, the limit.  Here the product is
+// computed transposed, D[n,t] = sum_k W[n,k] X[t,k]:
+//   * the WEIGHTS are the MMA's A operand and live in TENSOR MEMORY: four warps read the
+//     packed int4 tile from shared memory (staged there by a bulk async copy), expand each
+//     32-bit word into eight int8 values with two logic operations, and write them with
+//     tcgen05.st -- the expanded weights never touch shared memory;
+//   * the int8 ACTIVATIONS are the B operand, TMA-loaded (128-byte swizzle, K-major)
+//     straight from the quantizer's output;
+//   * accumulators (128 channels x up to 256 tokens, int32) live in tensor memory and are
+//     double-buffered when the token tile is <= 192 so the epilogue of one tile overlaps
+//     the main loop of the next;
+//   * the epilogue thread that owns channel n holds s_w[n] and bias[n] in registers and
+//     gets the per-token scale from a small shared-memory table built from the segment
+//     table; consecutive lanes write consecutive channels of one token row.
+// The nibble-to-int8 expansion leaves each code in the HIGH nibble of its byte, i.e. the
+// MMA sees 16*q_w; the accumulator is therefore exactly 16x the true one (|16 acc| <=
+// 128*8*16*K < 2^31 for K <= 131071) and the epilogue shifts it back, exactly.
+//
+// Warp roles (384 threads): warp 0 activation TMA producer, warp 1 MMA issuer, warp 2
+// tensor-memory allocator, warp 3 weight bulk-copy producer, warps 4-7 weight expanders
+// (one per 32-lane quarter of tensor memory), warps 8-11 epilogue.
+//
+// Every wait on an mbarrier is bounded: after ~2 s without progress the waiting thread
+// records MQ_ERR_TIMEOUT and its site in the status word, raises a CTA-wide abort flag,
+// and all roles drain (outstanding copies are awaited, tensor memory is freed).
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "mq_common.cuh"
+
+namespace mq {
+namespace {
+
+constexpr int kThreads = 384;
+constexpr int kTileN = MQ_W_TILE_N;    // channels per CTA tile (MMA M)
+constexpr int kBlockK = MQ_W_TILE_K;   // K per pipeline stage
+constexpr int kWTileBytes = 8192;      // packed int4 tile 128 x 128
+constexpr int kMaxActStages = 8;
+constexpr int kMaxWStages = 24;
+constexpr int kMaxAStages = 8;
+constexpr unsigned long long kTimeoutNs = 2000000000ull;
+constexpr int kSmemBudget = 220 * 1024;
+
+struct KernelParams {
+  int T, K, N;
+  int TN;          // token tile (MMA N), multiple of 16, 16..256
+  int n_tn;        // channel tiles
+  int n_tt;        // token tiles
+  int ksplit;      // K splits (1 = direct epilogue)
+  int kb_total;    // K blocks
+  int num_d;       // accumulator buffers (1 or 2)
+  int d_stride;    // tensor-memory columns between accumulator buffers
+  int a_base;      // first tensor-memory column of the weight stages
+  int num_a;       // weight stages in tensor memory
+  int act_stages;  // activation stages in shared memory
+  int w_stages;    // packed-weight stages in shared memory
+  SegTable seg;
+  float s_vis, s_txt;
+  const uint8_t* W_layout;
+  const float* s_w;
+  const float* bias;
+  void* Y;
+  int64_t ldy;
+  int y_is_f32;
+  int32_t* acc_out;
+  int32_t* splitk_acc;
+  int32_t* status;
+};
+
+struct __align__(8) Barriers {
+  uint64_t act_full[kMaxActStages], act_empty[kMaxActStages];
+  uint64_t w_full[kMaxWStages], w_empty[kMaxWStages];
+  uint64_t a_ready[kMaxAStages], a_free[kMaxAStages];
+  uint64_t d_full[2], d_empty[2];
+  uint64_t drain;
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+// ------------------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ unsigned long long globaltimer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+
+// Bounded wait.  Returns false if the CTA is aborting (this wait or another one expired).
+__device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, Barriers* sh,
+                                            int32_t* status, int site) {
+  const unsigned long long t0 = globaltimer_ns();
+  unsigned spins = 0;
+  while (true) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((++spins & 63u) == 0u) {
+      if (*reinterpret_cast<volatile int*>(&sh->abort_flag)) return false;
+      if (globaltimer_ns() - t0 > kTimeoutNs) {
+        *reinterpret_cast<volatile int*>(&sh->abort_flag) = 1;
+        if (atomicCAS(status, MQ_OK, MQ_ERR_TIMEOUT) == MQ_OK) status[1] = site;
+        __threadfence();
+        return false;
+      }
+    }
+  }
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, Barriers* sh,
+                                          int32_t* status, int site) {
+  if (mbar_try_wait(bar, parity)) return true;
+  return mbar_wait_slow(bar, parity, sh, status, site);
+}
+
+__device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* tmap, int x, int y,
+                                            uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(smem_u32(smem_dst)), "l"(tmap), "r"(smem_u32(bar)), "r"(x), "r"(y)
+      : "memory");
+}
+__device__ __forceinline__ void bulk_load_1d(void* smem_dst, const void* gsrc, uint32_t bytes,
+                                             uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+      ::"r"(smem_u32(smem_dst)), "l"(gsrc), "r"(bytes), "r"(smem_u32(bar))
+      : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_alloc(uint32_t* smem_dst, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_dst)),
+               "r"(ncols)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+
+// D[tmem] (+)= A[tmem] * B[smem], int8 x int8 -> int32, one CTA.
+__device__ __forceinline__ void mma_i8_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::i8 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// Arrive on an mbarrier once all tcgen05 operations issued so far by this thread are done.
+__device__ __forceinline__ void tc_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+               : "memory");
+}
+
+__device__ __forceinline__ void tmem_st_x32(uint32_t taddr, const uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+      "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+      "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+      "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_ld_x16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Warp-uniform verdict of a bounded wait, so that .sync.aligned instructions stay converged.
+__device__ __forceinline__ bool warp_all(bool ok) { return __all_sync(0xffffffffu, ok) != 0; }
+
+// K-major, 128-byte-swizzled shared-memory operand: rows of 128 bytes, 8-row groups 1024 B apart.
+__device__ __forceinline__ uint64_t make_b_desc(uint32_t smem_addr) {
+  return (uint64_t)((smem_addr >> 4) & 0x3FFFu) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+// kind::i8: D = s32 (bits 4-5 = 2), A = B = signed 8-bit (bits 7-9, 10-12 = 1), both K-major,
+// N >> 3 at bits 17-22, M >> 4 at bits 24-28.
+__device__ __forceinline__ uint32_t make_idesc(int n) {
+  return (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileN >> 4) << 24);
+}
+
+struct TileCoord {
+  int tn, tt, kb0, kb1;
+};
+__device__ __forceinline__ TileCoord decode_tile(const KernelParams& p, int tile) {
+  TileCoord c;
+  c.tn = tile % p.n_tn;
+  const int rest = tile / p.n_tn;
+  c.tt = rest % p.n_tt;
+  const int ks = rest / p.n_tt;
+  const int per = (p.kb_total + p.ksplit - 1) / p.ksplit;
+  c.kb0 = ks * per;
+  c.kb1 = min(p.kb_total, c.kb0 + per);
+  return c;
+}
+
+// ------------------------------------------------------------------------------ the kernel
+__global__ void __launch_bounds__(kThreads, 1)
+w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const KernelParams p) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  // carve: activation stages (1024-aligned), weight stages, barriers, token scales
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int act_stage_bytes = p.TN * kBlockK;
+  uint8_t* act_smem = smem;
+  uint8_t* w_smem = act_smem + (size_t)p.act_stages * act_stage_bytes;
+  Barriers* sh = reinterpret_cast<Barriers*>(w_smem + (size_t)p.w_stages * kWTileBytes);
+  float* s_tok = reinterpret_cast<float*>(sh + 1);  // [4 epilogue warps][256]
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const int total_tiles = p.n_tn * p.n_tt * p.ksplit;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < p.act_stages; ++i) { mbar_init(&sh->act_full[i], 1); mbar_init(&sh->act_empty[i], 1); }
+    for (int i = 0; i < p.w_stages; ++i) { mbar_init(&sh->w_full[i], 1); mbar_init(&sh->w_empty[i], 128); }
+    for (int i = 0; i < p.num_a; ++i) { mbar_init(&sh->a_ready[i], 128); mbar_init(&sh->a_free[i], 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&sh->d_full[i], 1); mbar_init(&sh->d_empty[i], 128); }
+    mbar_init(&sh->drain, 1);
+    sh->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 2) {
+    tmem_alloc(&sh->tmem_base, 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&sh->tmem_base);
+
+  if (warp == 0) {
+    // ---------------- activation TMA producer
+    if (lane == 0) {
+      int it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        const TileCoord c = decode_tile(p, tile);
+        for (int kb = c.kb0; kb < c.kb1; ++kb, ++it) {
+          const int s = it % p.act_stages;
+          const uint32_t round = it / p.act_stages;
+          if (round > 0 && !(ok = mbar_wait(&sh->act_empty[s], (round - 1) & 1, sh, p.status, 1))) break;
+          mbar_arrive_expect_tx(&sh->act_full[s], act_stage_bytes);
+          tma_load_2d(act_smem + (size_t)s * act_stage_bytes, &tmap_act, kb * kBlockK, c.tt * p.TN,
+                      &sh->act_full[s]);
+        }
+      }
+      if (!ok) {  // drain: wait for copies that are still landing in our shared memory
+        for (int back = 1; back <= p.act_stages && back <= it; ++back) {
+          const int j = it - back;
+          mbar_wait(&sh->act_full[j % p.act_stages], (j / p.act_stages) & 1, sh, p.status, 90);
+        }
+      }
+    }
+  } else if (warp == 3) {
+    // ---------------- packed-weight bulk-copy producer
+    if (lane == 0) {
+      int it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        const TileCoord c = decode_tile(p, tile);
+        const uint8_t* wsrc = p.W_layout + ((size_t)c.tn * p.kb_total) * kWTileBytes;
+        for (int kb = c.kb0; kb < c.kb1; ++kb, ++it) {
+          const int s = it % p.w_stages;
+          const uint32_t round = it / p.w_stages;
+          if (round > 0 && !(ok = mbar_wait(&sh->w_empty[s], (round - 1) & 1, sh, p.status, 2))) break;
+          mbar_arrive_expect_tx(&sh->w_full[s], kWTileBytes);
+          bulk_load_1d(w_smem + (size_t)s * kWTileBytes, wsrc + (size_t)kb * kWTileBytes, kWTileBytes,
+                       &sh->w_full[s]);
+        }
+      }
+      if (!ok) {
+        for (int back = 1; back <= p.w_stages && back <= it; ++back) {
+          const int j = it - back;
+          mbar_wait(&sh->w_full[j % p.w_stages], (j / p.w_stages) & 1, sh, p.status, 91);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc = make_idesc(p.TN);
+      int it = 0, tile_it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tile_it) {
+        const TileCoord c = decode_tile(p, tile);
+        const int d = tile_it % p.num_d;
+        const uint32_t d_round = tile_it / p.num_d;
+        if (d_round > 0 && !(ok = mbar_wait(&sh->d_empty[d], (d_round - 1) & 1, sh, p.status, 3))) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(d * p.d_stride);
+        for (int kb = c.kb0; kb < c.kb1; ++kb, ++it) {
+          const int sa = it % p.act_stages, aa = it % p.num_a;
+          if (!(ok = mbar_wait(&sh->act_full[sa], (it / p.act_stages) & 1, sh, p.status, 4))) break;
+          if (!(ok = mbar_wait(&sh->a_ready[aa], (it / p.num_a) & 1, sh, p.status, 5))) break;
+          tc_fence_after();
+          const uint64_t bdesc = make_b_desc(smem_u32(act_smem + (size_t)sa * act_stage_bytes));
+          const uint32_t a_tmem = tmem_base + (uint32_t)(p.a_base + aa * 32);
+#pragma unroll
+          for (int s = 0; s < 4; ++s)
+            mma_i8_ts(d_tmem, a_tmem + s * 8, bdesc + (uint64_t)(s * 2), idesc, (kb > c.kb0 || s > 0) ? 1u : 0u);
+          tc_commit(&sh->act_empty[sa]);
+          tc_commit(&sh->a_free[aa]);
+        }
+        if (ok) tc_commit(&sh->d_full[d]);
+      }
+      if (!ok) {  // let every MMA already issued finish before tensor memory is freed
+        tc_commit(&sh->drain);
+        mbar_wait(&sh->drain, 0, sh, p.status, 92);
+      }
+    }
+  } else if (warp >= 4 && warp < 8) {
+    // ---------------- weight expanders: packed int4 (smem) -> int8 x16 (tensor memory)
+    const int q = warp & 3;
+    const int r = q * 32 + lane;  // channel row inside the tile == tensor-memory lane
+    int it = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+      const TileCoord c = decode_tile(p, tile);
+      for (int kb = c.kb0; kb < c.kb1; ++kb, ++it) {
+        const int sw = it % p.w_stages, aa = it % p.num_a;
+        if (!(ok = warp_all(mbar_wait(&sh->w_full[sw], (it / p.w_stages) & 1, sh, p.status, 6)))) break;
+        const uint4* src = reinterpret_cast<const uint4*>(w_smem + (size_t)sw * kWTileBytes) + r;
+        uint32_t regs[32];
+#pragma unroll
+        for (int jj = 0; jj < 4; ++jj) {
+          const uint4 w = src[jj * 128];
+          const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            regs[jj * 8 + 2 * i] = (ww[i] << 4) & 0xF0F0F0F0u;   // codes k0..k0+3, each x16
+            regs[jj * 8 + 2 * i + 1] = ww[i] & 0xF0F0F0F0u;      // codes k0+4..k0+7, each x16
+          }
+        }
+        mbar_arrive(&sh->w_empty[sw]);
+        const uint32_t a_round = it / p.num_a;
+        if (a_round > 0 && !(ok = warp_all(mbar_wait(&sh->a_free[aa], (a_round - 1) & 1, sh, p.status, 7)))) break;
+        tc_fence_after();
+        tmem_st_x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(p.a_base + aa * 32), regs);
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(&sh->a_ready[aa]);
+      }
+    }
+  } else if (warp >= 8) {
+    // ---------------- epilogue: tensor memory -> dequant -> global
+    const int q = warp & 3;
+    float* stok = s_tok + q * 256;  // private to this warp: no cross-warp barrier to strand on abort
+    int tile_it = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tile_it) {
+      const TileCoord c = decode_tile(p, tile);
+      const int t0 = c.tt * p.TN;
+      __syncwarp();
+      for (int j = lane; j < p.TN; j += 32) {
+        const int t = t0 + j;
+        stok[j] = (t < p.T && thread_row_modality(p.seg, t) == MQ_VISUAL) ? p.s_vis : p.s_txt;
+      }
+      __syncwarp();
+      const int d = tile_it % p.num_d;
+      if (!(ok = warp_all(mbar_wait(&sh->d_full[d], (tile_it / p.num_d) & 1, sh, p.status, 8)))) break;
+      tc_fence_after();
+      const int n = c.tn * kTileN + q * 32 + lane;
+      const bool n_ok = n < p.N;
+      const float sw = n_ok ? p.s_w[n] : 0.0f;
+      const float bs = (n_ok && p.bias) ? p.bias[n] : 0.0f;
+      const uint32_t d_tmem = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(d * p.d_stride);
+      for (int cc = 0; cc < p.TN; cc += 16) {
+        uint32_t v[16];
+        tmem_ld_x16(d_tmem + cc, v);
+        tmem_wait_ld();
+        if (n_ok) {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const int t = t0 + cc + j;
+            if (t >= p.T) break;
+            const int acc = ((int)v[j]) >> 4;  // the MMA saw 16 * q_w
+            const size_t o = (size_t)t * p.N + n;
+            if (p.ksplit > 1) {
+              atomicAdd(&p.splitk_acc[o], acc);
+            } else {
+              if (p.acc_out) p.acc_out[o] = acc;
+              float y = __fmul_rn((float)acc, __fmul_rn(stok[cc + j], sw));
+              if (p.bias) y = __fadd_rn(y, bs);
+              const size_t oy = (size_t)t * p.ldy + n;
+              if (p.y_is_f32) static_cast<float*>(p.Y)[oy] = y;
+              else static_cast<__nv_bfloat16*>(p.Y)[oy] = __float2bfloat16_rn(y);
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(&sh->d_empty[d]);
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 2) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+// Split-K finalize: exact int32 partial sums -> dequantized output.
+__global__ void splitk_finalize_kernel(const int32_t* __restrict__ acc, int T, int N, SegTable seg, float s_vis,
+                                       float s_txt, const float* __restrict__ s_w, const float* __restrict__ bias,
+                                       void* Y, int64_t ldy, int y_is_f32, int32_t* __restrict__ acc_out) {
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= (int64_t)T * N) return;
+  const int t = (int)(idx / N), n = (int)(idx % N);
+  const int a = acc[idx];
+  if (acc_out) acc_out[idx] = a;
+  const float st = thread_row_modality(seg, t) == MQ_VISUAL ? s_vis : s_txt;
+  float y = __fmul_rn((float)a, __fmul_rn(st, s_w[n]));
+  if (bias) y = __fadd_rn(y, bias[n]);
+  const size_t oy = (size_t)t * ldy + n;
+  if (y_is_f32) static_cast<float*>(Y)[oy] = y;
+  else static_cast<__nv_bfloat16*>(Y)[oy] = __float2bfloat16_rn(y);
+}
+
+// ------------------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  return fn;
+}
+
+struct Plan {
+  int TN, n_tt, n_tn, ksplit, num_d, d_stride, a_base, num_a, act_stages, w_stages, grid;
+  size_t smem;
+};
+
+int sm_count() {
+  static int n = 0;
+  if (!n) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+      n = 148;
+  }
+  return n;
+}
+
+Plan make_plan(int T, int K, int N) {
+  Plan pl{};
+  const int sms = sm_count();
+  pl.n_tn = (N + kTileN - 1) / kTileN;
+  const int kb_total = (K + kBlockK - 1) / kBlockK;
+  // token tile: as few tiles as possible, each as even as possible, multiple of 16
+  int n_tt = (T + 255) / 256;
+  int TN = (((T + n_tt - 1) / n_tt) + 15) / 16 * 16;
+  // several tiles per CTA: prefer <= 192 tokens so two accumulators fit and the epilogue overlaps
+  if ((long long)pl.n_tn * n_tt > sms && TN > 192) {
+    n_tt = (T + 191) / 192;
+    TN = (((T + n_tt - 1) / n_tt) + 15) / 16 * 16;
+  }
+  pl.TN = TN;
+  pl.n_tt = n_tt;
+  pl.d_stride = TN <= 128 ? 128 : (TN <= 192 ? 192 : 256);
+  pl.num_d = pl.d_stride <= 192 ? 2 : 1;
+  pl.a_base = pl.num_d * pl.d_stride;
+  pl.num_a = (512 - pl.a_base) / 32;
+  if (pl.num_a > kMaxAStages) pl.num_a = kMaxAStages;
+  // split K when the tiles alone cannot fill the machine (small T: weight streaming)
+  const long long tiles = (long long)pl.n_tn * n_tt;
+  int ksplit = 1;
+  if (tiles * 2 <= sms) {
+    ksplit = (int)(sms / tiles);
+    const int max_split = kb_total / 4 > 0 ? kb_total / 4 : 1;  // keep >= 4 K blocks per CTA
+    if (ksplit > max_split) ksplit = max_split;
+    if (ksplit < 1) ksplit = 1;
+    const int per = (kb_total + ksplit - 1) / ksplit;
+    ksplit = (kb_total + per - 1) / per;  // no empty split
+  }
+  pl.ksplit = ksplit;
+  const int act_stage = TN * kBlockK;
+  const size_t fixed = 1024 + sizeof(Barriers) + 4 * 256 * sizeof(float);
+  int act_stages = TN <= 64 ? 8 : (TN <= 128 ? 6 : 4);
+  int w_stages = (int)((kSmemBudget - fixed - (size_t)act_stages * act_stage) / kWTileBytes);
+  if (w_stages > kMaxWStages) w_stages = kMaxWStages;
+  if (TN > 128 && w_stages > 8) w_stages = 8;
+  pl.act_stages = act_stages;
+  pl.w_stages = w_stages;
+  pl.smem = fixed + (size_t)act_stages * act_stage + (size_t)w_stages * kWTileBytes;
+  const long long total = tiles * ksplit;
+  pl.grid = (int)(total < sms ? total : sms);
+  return pl;
+}
+
+}  // namespace
+
+size_t gemm_splitk_bytes(int T, int K, int N) {
+  if (T <= 0 || K <= 0 || N <= 0) return 0;
+  const Plan pl = make_plan(T, K, N);
+  return pl.ksplit > 1 ? (size_t)T * N * sizeof(int32_t) : 0;
+}
+
+int launch_gemm(const GemmArgs& a, cudaStream_t st) {
+  if (a.T == 0 || a.N == 0) return MQ_OK;
+  const Plan pl = make_plan(a.T, a.K, a.N);
+  EncodeTiledFn encode = get_encode_fn();
+  if (!encode) return MQ_ERR_CUDA;
+
+  CUtensorMap tmap;
+  const cuuint64_t dims[2] = {(cuuint64_t)a.K, (cuuint64_t)a.T};
+  const cuuint64_t strides[1] = {(cuuint64_t)a.ldq};
+  const cuuint32_t box[2] = {(cuuint32_t)kBlockK, (cuuint32_t)pl.TN};
+  const cuuint32_t estr[2] = {1, 1};
+  if (encode(&tmap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t*>(a.Qx), dims, strides, box, estr,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return MQ_ERR_CUDA;
+
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(w4a8_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 2048) !=
+        cudaSuccess)
+      return MQ_ERR_CUDA;
+    attr_set = true;
+  }
+
+  KernelParams p{};
+  p.T = a.T; p.K = a.K; p.N = a.N;
+  p.TN = pl.TN; p.n_tn = pl.n_tn; p.n_tt = pl.n_tt; p.ksplit = pl.ksplit;
+  p.kb_total = (a.K + kBlockK - 1) / kBlockK;
+  p.num_d = pl.num_d; p.d_stride = pl.d_stride; p.a_base = pl.a_base; p.num_a = pl.num_a;
+  p.act_stages = pl.act_stages; p.w_stages = pl.w_stages;
+  p.seg = a.seg; p.s_vis = a.s_vis; p.s_txt = a.s_txt;
+  p.W_layout = static_cast<const uint8_t*>(a.W_layout);
+  p.s_w = a.s_w; p.bias = a.bias; p.Y = a.Y; p.ldy = a.ldy; p.y_is_f32 = a.y_is_f32;
+  p.acc_out = a.acc_out; p.splitk_acc = a.splitk_acc; p.status = a.status;
+
+  if (pl.ksplit > 1) {
+    if (!a.splitk_acc) return MQ_ERR_WORKSPACE;
+    if (cudaMemsetAsync(a.splitk_acc, 0, (size_t)a.T * a.N * sizeof(int32_t), st) != cudaSuccess) return MQ_ERR_CUDA;
+  }
+  w4a8_gemm_kernel<<<pl.grid, kThreads, pl.smem, st>>>(tmap, p);
+  if (cudaGetLastError() != cudaSuccess) return MQ_ERR_CUDA;
+  if (pl.ksplit > 1) {
+    const int64_t n = (int64_t)a.T * a.N;
+    splitk_finalize_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(a.splitk_acc, a.T, a.N, a.seg, a.s_vis,
+                                                                       a.s_txt, a.s_w, a.bias, a.Y, a.ldy,
+                                                                       a.y_is_f32, a.acc_out);
+    if (cudaGetLastError() != cudaSuccess) return MQ_ERR_CUDA;
+  }
+  return MQ_OK;
+}
+
+}  // namespace mq

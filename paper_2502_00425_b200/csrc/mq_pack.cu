@@ -1,0 +1,171 @@
+// K0b: per-output-channel symmetric int4 round-to-nearest weight quantizer and the two
+// storage layouts (offline, untimed).
+//
+// Method: Eq. 2 with b = 4 and zero-point 0; Algorithm 1 lists per-channel weight scales
+// among the outputs.  s_w[n] = max_k |W[n,k]| / 7, q = clamp(rne(W / s_w), -8, 7).
+//
+// GEMM weight layout.  W is cut into tiles of 128 output channels x 128 input channels
+// (zero-padded at the edges).  Tile (tn, kb) is one contiguous 8 KB block at
+// ((tn * KB + kb) * 8192); inside it, 16-byte piece (jj, r) at (jj * 128 + r) * 16 holds
+// the 32 codes k = kb*128 + jj*32 .. +31 of channel tn*128 + r: 32-bit word i of the piece
+// carries codes k0 = jj*32 + i*8 .. +7 with code k0+b in the LOW nibble of byte b and code
+// k0+4+b in the HIGH nibble of byte b.  A thread of the GEMM that owns channel r then reads
+// its four pieces with conflict-free 16-byte shared-memory loads and turns one word into
+// eight consecutive int8 values with two logic operations (see mq_gemm.cu).
+#include "mq_common.cuh"
+
+namespace mq {
+namespace {
+
+__device__ __forceinline__ int rtn_int4(float w, float s) {
+  int q = __float2int_rn(__fdiv_rn(w, s));
+  return max(-8, min(7, q));
+}
+
+__global__ void row_scale_kernel(const float* __restrict__ W, int N, int K, int64_t ldw,
+                                 float* __restrict__ s_w) {
+  const int n = blockIdx.x;
+  if (n >= N) return;
+  float m = 0.0f;
+  for (int k = threadIdx.x; k < K; k += blockDim.x) m = fmaxf(m, fabsf(W[(int64_t)n * ldw + k]));
+  __shared__ float red[32];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = m;
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    m = threadIdx.x < (blockDim.x >> 5) ? red[threadIdx.x] : 0.0f;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if (threadIdx.x == 0) s_w[n] = m > 0.0f ? __fdiv_rn(m, 7.0f) : 1.0f;
+  }
+}
+
+__global__ void pack_canonical_kernel(const float* __restrict__ W, int N, int K, int64_t ldw,
+                                      const float* __restrict__ s_w, uint8_t* __restrict__ packed) {
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int half = K / 2;
+  if (idx >= (int64_t)N * half) return;
+  const int n = (int)(idx / half), j = (int)(idx % half);
+  const float s = s_w[n];
+  const int q0 = rtn_int4(W[(int64_t)n * ldw + 2 * j], s);
+  const int q1 = rtn_int4(W[(int64_t)n * ldw + 2 * j + 1], s);
+  packed[idx] = (uint8_t)((q0 & 15) | ((q1 & 15) << 4));
+}
+
+// One thread per 32-bit word of the GEMM layout.
+struct WordCoord {
+  int n, k0;
+};
+__device__ __forceinline__ WordCoord layout_word_coord(int64_t word, int KB) {
+  // word index = ((tn * KB + kb) * 4 + jj) * 512 + r * 4 + i
+  const int i = (int)(word & 3);
+  const int r = (int)((word >> 2) & 127);
+  const int64_t rest = word >> 9;
+  const int jj = (int)(rest & 3);
+  const int64_t tile = rest >> 2;
+  const int kb = (int)(tile % KB);
+  const int tn = (int)(tile / KB);
+  return {tn * MQ_W_TILE_N + r, kb * MQ_W_TILE_K + jj * 32 + i * 8};
+}
+
+__global__ void pack_layout_kernel(const float* __restrict__ W, int N, int K, int64_t ldw,
+                                   const float* __restrict__ s_w, uint32_t* __restrict__ layout,
+                                   int KB, int64_t n_words) {
+  const int64_t word = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (word >= n_words) return;
+  const WordCoord c = layout_word_coord(word, KB);
+  uint32_t out = 0;
+  if (c.n < N) {
+    const float s = s_w[c.n];
+#pragma unroll
+    for (int b = 0; b < 4; ++b) {
+      const int klo = c.k0 + b, khi = c.k0 + 4 + b;
+      const int qlo = klo < K ? rtn_int4(W[(int64_t)c.n * ldw + klo], s) : 0;
+      const int qhi = khi < K ? rtn_int4(W[(int64_t)c.n * ldw + khi], s) : 0;
+      out |= (uint32_t)((qlo & 15) | ((qhi & 15) << 4)) << (8 * b);
+    }
+  }
+  layout[word] = out;
+}
+
+__device__ __forceinline__ int canon_nibble(const uint8_t* packed, int half, int n, int k) {
+  return (packed[(int64_t)n * half + (k >> 1)] >> (4 * (k & 1))) & 15;
+}
+
+__global__ void repack_kernel(const uint8_t* __restrict__ packed, int N, int K,
+                              uint32_t* __restrict__ layout, int KB, int64_t n_words) {
+  const int64_t word = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (word >= n_words) return;
+  const WordCoord c = layout_word_coord(word, KB);
+  uint32_t out = 0;
+  if (c.n < N) {
+#pragma unroll
+    for (int b = 0; b < 4; ++b) {
+      const int klo = c.k0 + b, khi = c.k0 + 4 + b;
+      const int qlo = klo < K ? canon_nibble(packed, K / 2, c.n, klo) : 0;
+      const int qhi = khi < K ? canon_nibble(packed, K / 2, c.n, khi) : 0;
+      out |= (uint32_t)(qlo | (qhi << 4)) << (8 * b);
+    }
+  }
+  layout[word] = out;
+}
+
+__global__ void unpack_kernel(const uint8_t* __restrict__ packed, const uint8_t* __restrict__ layout,
+                              int N, int K, int KB, int8_t* __restrict__ q, int64_t ldq) {
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= (int64_t)N * K) return;
+  const int n = (int)(idx / K), k = (int)(idx % K);
+  int nib;
+  if (packed) {
+    nib = canon_nibble(packed, K / 2, n, k);
+  } else {
+    const int tn = n / MQ_W_TILE_N, r = n % MQ_W_TILE_N, kb = k / MQ_W_TILE_K, kk = k % MQ_W_TILE_K;
+    const int jj = kk / 32, c = kk % 32, i = c / 8, e = c % 8;
+    const int64_t byte = (((int64_t)tn * KB + kb) * 4 + jj) * 2048 + r * 16 + i * 4 + (e & 3);
+    nib = (layout[byte] >> (e >= 4 ? 4 : 0)) & 15;
+  }
+  q[(int64_t)n * ldq + k] = (int8_t)(nib >= 8 ? nib - 16 : nib);
+}
+
+inline int64_t layout_words(int N, int K) {
+  const int64_t TN = (N + MQ_W_TILE_N - 1) / MQ_W_TILE_N, KB = (K + MQ_W_TILE_K - 1) / MQ_W_TILE_K;
+  return TN * KB * 2048;
+}
+
+}  // namespace
+
+int launch_pack_w4(const float* W, int N, int K, int64_t ldw, uint8_t* packed, float* s_w,
+                   void* layout, cudaStream_t st) {
+  if (N == 0 || K == 0) return MQ_OK;
+  row_scale_kernel<<<N, 256, 0, st>>>(W, N, K, ldw, s_w);
+  if (packed) {
+    const int64_t n = (int64_t)N * (K / 2);
+    pack_canonical_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(W, N, K, ldw, s_w, packed);
+  }
+  if (layout) {
+    const int64_t nw = layout_words(N, K);
+    pack_layout_kernel<<<(unsigned)((nw + 255) / 256), 256, 0, st>>>(
+        W, N, K, ldw, s_w, static_cast<uint32_t*>(layout), (K + MQ_W_TILE_K - 1) / MQ_W_TILE_K, nw);
+  }
+  return cuda_status(cudaGetLastError());
+}
+
+int launch_repack_w4(const uint8_t* packed, int N, int K, void* layout, cudaStream_t st) {
+  if (N == 0 || K == 0) return MQ_OK;
+  const int64_t nw = layout_words(N, K);
+  repack_kernel<<<(unsigned)((nw + 255) / 256), 256, 0, st>>>(
+      packed, N, K, static_cast<uint32_t*>(layout), (K + MQ_W_TILE_K - 1) / MQ_W_TILE_K, nw);
+  return cuda_status(cudaGetLastError());
+}
+
+int launch_unpack_w4(const uint8_t* packed, const void* layout, int N, int K, int8_t* q,
+                     int64_t ldq, cudaStream_t st) {
+  if (N == 0 || K == 0) return MQ_OK;
+  const int64_t n = (int64_t)N * K;
+  unpack_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(
+      packed, static_cast<const uint8_t*>(layout), N, K, (K + MQ_W_TILE_K - 1) / MQ_W_TILE_K, q, ldq);
+  return cuda_status(cudaGetLastError());
+}
+
+}  // namespace mq

@@ -1,0 +1,130 @@
+"""Host-side checks that need no GPU: the shared library loads, exports every symbol the
+header declares, and rejects bad arguments before touching the device."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+from paper_2502_00425_b200 import binding as B
+from paper_2502_00425_b200 import build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build_library()
+    return B.load()
+
+
+def test_header_symbols_are_exported(lib):
+    hdr = open(os.path.join(ROOT, "include", "mq.h")).read()
+    declared = set(re.findall(r"\b(mq_[a-z0-9_]+)\s*\(", hdr))
+    assert {"mq_calibrate_static_scales", "mq_pack_w4", "mq_aifs_reorder", "mq_fwht_quant_i8",
+            "mq_w4a8_msq_linear", "mq_attn_mask_remap"} <= declared
+    for name in declared:
+        assert hasattr(lib, name), name
+    assert declared == set(B.EXPORTED)
+    assert lib.mq_version() == 1
+
+
+def test_status_strings(lib):
+    assert B.status_string(0) == "MQ_OK"
+    assert B.status_string(B.MQ_ERR_ALIGNMENT) == "MQ_ERR_ALIGNMENT"
+    assert B.status_string(-99) == "MQ_ERR_UNKNOWN"
+
+
+def test_size_queries(lib):
+    assert B.mq_w4_layout_bytes(128, 128) == 8192
+    assert B.mq_w4_layout_bytes(3584, 18944) == 28 * 148 * 8192
+    assert B.mq_w4_layout_bytes(16, 32) == 8192                     # padded to one tile
+    assert B.mq_w4_layout_bytes(0, 32) == 0
+    big = B.mq_workspace_bytes(1088, 18944, 3584, 128)
+    assert big >= 256 + 1088 * 18944
+    assert B.mq_workspace_bytes(1088, 18944, 3584, 0, B.MQ_FLAG_X_IS_INT8) == 256
+    assert B.mq_workspace_bytes(8, 4096, 256) >= 256 + 8 * 4096 + 8 * 256 * 4   # split-K scratch
+    assert B.mq_workspace_bytes(8, 100, 256) == 0                   # K % 32
+    assert B.mq_workspace_bytes(8, 128, 100) == 0                   # N % 16
+    assert B.mq_workspace_bytes(8, 128, 128, 48) == 0               # rotation block not a power of two
+
+
+def _desc(T=8, K=128, N=128, rot=0, group=0, flags=0):
+    return B.mq_linear_desc(T, K, N, rot, group, flags)
+
+
+def test_linear_argument_validation(lib):
+    A = 0x10000  # fake, aligned "device" address: validation must fail before it is used
+    seg = B.mq_segments(0, None, None)
+
+    def call(d, x=A, ldx=128, s_v=1.0, s_t=1.0, w=A, s_w=A, y=A, ldy=128, ws=A, ws_bytes=1 << 30):
+        return lib.mq_w4a8_msq_linear(C.byref(d), x, ldx, C.byref(seg), s_v, s_t, w, s_w, None, y, ldy, None, ws,
+                                      ws_bytes, None)
+
+    assert lib.mq_w4a8_msq_linear(None, A, 128, None, 1.0, 1.0, A, A, None, A, 128, None, A, 1 << 30, None) \
+        == B.MQ_ERR_INVALID_ARG
+    assert call(_desc(K=100)) == B.MQ_ERR_INVALID_ARG
+    assert call(_desc(N=100)) == B.MQ_ERR_INVALID_ARG
+    assert call(_desc(T=-1)) == B.MQ_ERR_INVALID_ARG
+    assert call(_desc(group=128)) == B.MQ_ERR_UNSUPPORTED
+    assert call(_desc(rot=16)) == B.MQ_ERR_UNSUPPORTED
+    assert call(_desc(rot=96)) == B.MQ_ERR_INVALID_ARG
+    assert call(_desc(K=384, rot=256), ldx=384) == B.MQ_ERR_INVALID_ARG      # rotation block must divide K
+    assert call(_desc(flags=8)) == B.MQ_ERR_INVALID_ARG
+    assert call(_desc(rot=128, flags=B.MQ_FLAG_X_IS_INT8)) == B.MQ_ERR_INVALID_ARG
+    assert call(_desc(K=1 << 20), ldx=1 << 20) == B.MQ_ERR_UNSUPPORTED
+    assert call(_desc(), s_v=0.0) == B.MQ_ERR_INVALID_ARG
+    assert call(_desc(), s_t=float("inf")) == B.MQ_ERR_INVALID_ARG
+    assert call(_desc(), s_t=float("nan")) == B.MQ_ERR_INVALID_ARG
+    assert call(_desc(), x=None) == B.MQ_ERR_INVALID_ARG
+    assert call(_desc(), ldx=64) == B.MQ_ERR_INVALID_ARG
+    assert call(_desc(), x=A + 2) == B.MQ_ERR_ALIGNMENT
+    assert call(_desc(), ldx=132) == B.MQ_ERR_ALIGNMENT
+    assert call(_desc(), w=A + 64) == B.MQ_ERR_ALIGNMENT
+    assert call(_desc(), ws=None) == B.MQ_ERR_WORKSPACE
+    assert call(_desc(), ws=A + 16) == B.MQ_ERR_ALIGNMENT
+    assert call(_desc(), ws_bytes=100) == B.MQ_ERR_WORKSPACE
+    assert call(_desc(T=0)) == B.MQ_OK                                        # empty input: no-op
+    bad_seg = B.mq_segments(-1, None, None)
+    assert lib.mq_w4a8_msq_linear(C.byref(_desc()), A, 128, C.byref(bad_seg), 1.0, 1.0, A, A, None, A, 128, None, A,
+                                  1 << 30, None) == B.MQ_ERR_INVALID_ARG
+    bad_seg = B.mq_segments(2, None, None)
+    assert lib.mq_w4a8_msq_linear(C.byref(_desc()), A, 128, C.byref(bad_seg), 1.0, 1.0, A, A, None, A, 128, None, A,
+                                  1 << 30, None) == B.MQ_ERR_INVALID_ARG
+
+
+def test_other_entry_points_validate(lib):
+    A = 0x10000
+    seg = B.mq_segments(0, None, None)
+    f = lib.mq_fwht_quant_i8
+    assert f(A, 4, 100, 100, C.byref(seg), 1.0, 1.0, 0, A, 112, None, None) == B.MQ_ERR_INVALID_ARG
+    assert f(A, 4, 128, 128, C.byref(seg), -1.0, 1.0, 0, A, 128, None, None) == B.MQ_ERR_INVALID_ARG
+    assert f(A, 4, 128, 128, C.byref(seg), 1.0, 1.0, 2048, A, 128, None, None) == B.MQ_ERR_UNSUPPORTED
+    assert f(A, 4, 128, 128, C.byref(seg), 1.0, 1.0, 0, A + 1, 128, None, None) == B.MQ_ERR_ALIGNMENT
+    assert f(A, 4, 128, 128, C.byref(seg), 1.0, 1.0, 0, A, 136, None, None) == B.MQ_ERR_ALIGNMENT
+    assert f(None, 4, 128, 128, C.byref(seg), 1.0, 1.0, 0, A, 128, None, None) == B.MQ_ERR_INVALID_ARG
+    c = lib.mq_calibrate_static_scales
+    assert c(A, 4, 128, 128, C.byref(seg), 0, 0, None, A, A, None) == B.MQ_ERR_INVALID_ARG
+    assert c(A, 4, 128, 128, C.byref(seg), 24, 0, A, A, A, None) == B.MQ_ERR_INVALID_ARG
+    p = lib.mq_pack_w4
+    assert p(A, 128, 128, 128, 128, None, A, None, None) == B.MQ_ERR_UNSUPPORTED
+    assert p(A, 128, 100, 100, 0, None, A, None, None) == B.MQ_ERR_INVALID_ARG
+    assert p(A, 128, 128, 128, 0, None, None, None, None) == B.MQ_ERR_INVALID_ARG
+    assert p(A, 128, 128, 128, 0, None, A, A + 16, None) == B.MQ_ERR_ALIGNMENT
+    r = lib.mq_aifs_reorder
+    assert r(A, A, 4, 8, 8, 8, A, None, A, A, A, 0, None) == B.MQ_ERR_INVALID_ARG      # in place
+    assert r(A, None, 4, 8, 8, 8, A, None, A, A, A, 0, None) == B.MQ_ERR_INVALID_ARG
+    assert r(A, A + 64, 4, 12, 12, 12, A, None, A, A, A, 0, None) == B.MQ_ERR_ALIGNMENT
+    assert r(A, A + 64, 4, 8, 8, 8, A, None, A, A, A, 2, None) == B.MQ_ERR_INVALID_ARG
+    assert r(A, A + 64, 4, 8, 8, 8, None, None, A, A, A, 0, None) == B.MQ_ERR_INVALID_ARG
+    m = lib.mq_attn_mask_remap
+    assert m(A, None, None, None, 4, A, A, A, None, None) == B.MQ_ERR_INVALID_ARG       # seg out needs n_first
+    assert m(A, None, None, A, 20000, A, None, None, A, None) == B.MQ_ERR_UNSUPPORTED
+    assert m(None, None, None, A, 4, A, None, None, None, None) == B.MQ_ERR_INVALID_ARG
+    assert lib.mq_last_device_status(None, None, None) == B.MQ_ERR_INVALID_ARG
+
+
+def test_binding_refuses_cpu_tensors():
+    import torch
+    with pytest.raises(ValueError):
+        B._ptr(torch.zeros(4))
