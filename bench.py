@@ -1,0 +1,399 @@
+#!/usr/bin/env python
+"""Benchmark of the W4A8 MSQ linear hot path on B200.
+
+    python bench.py --gpus N --steps K --warmup W [--impl reference]
+
+A step is one pass of the whole hot path over one batch shaped like the paper's prefill
+workload (Qwen2-7B-shaped down-projection, T = 1024 visual + 64 text tokens, K = 18944,
+N = 3584, online 128-block Hadamard rotation): AIFS reorder of the [L, 3584] hidden rows,
+position / segment remap, fused rotation + MSQ int8 quantizer, W4A8 tensor-core GEMM with the
+dequant epilogue.  Calibration and weight packing are offline and untimed.  Inputs are
+seeded synthetic tensors; several independent buffer sets are cycled so that every step
+reads its operands from HBM rather than L2.
+
+Prints ONE JSON line (rank 0).  `value` is device-resident throughput in TOPS (2*T*K*N
+integer operations per step over all ranks / slowest rank's time); `e2e` is the same metric
+through the C ABI with host buffers (H2D of the activations, D2H of the output inside the
+timed region); `roofline` describes the dominant kernel (the GEMM) against the measured
+tensor peak; `cpu_baseline` is the CPU oracle timed on this machine's host cores.
+With --impl reference the oracle itself is the timed program.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "w4a8_msq_linear_prefill_throughput"
+UNIT = "TOPS"
+WORKLOAD = "config2: Qwen2-7B-shaped down_proj, T=1088 (1024 visual + 64 text), K=18944, N=3584, rot_block=128"
+T_VIS, T_TXT, K_DIM, N_DIM, ROT, HIDDEN = 1024, 64, 18944, 3584, 128, 3584
+SPANS = [(0, 16), (1, 512), (0, 16), (1, 512), (0, 32)]  # original (interleaved) token order
+
+
+def ops_per_step(T=T_VIS + T_TXT):
+    return 2.0 * T * K_DIM * N_DIM
+
+
+def read_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_burst": p["bf16_tflops"],
+                "bf16_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_burst": 1590.0, "bf16_sustained": 1400.0, "source": "fallback"}
+
+
+# ------------------------------------------------------------------------------------------ clocks
+class ClockSampler:
+    """Polls SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.01):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        self.period = period_s
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _poll(self):
+        nv = self.nv
+        names = {"hw_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8),
+                 "hw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40),
+                 "sw_thermal_slowdown": getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20),
+                 "sw_power_cap": getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4)}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for k, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def start(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._poll, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+        if self.nv is not None and not self.samples:
+            try:
+                self.samples.append(self.nv.nvmlDeviceGetClockInfo(self.h, self.nv.NVML_CLOCK_SM))
+            except Exception:
+                pass
+        return {"sm_mhz": float(np.median(self.samples)) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# ------------------------------------------------------------------------------------------ oracle arm
+def oracle_sample_rows():
+    """Bounded sample of the workload for the CPU arms: 192 visual rows + all 64 text rows."""
+    return np.concatenate([np.arange(0, 192), np.arange(T_VIS, T_VIS + T_TXT)])
+
+
+def time_oracle(case, qw, s_w, s_v, s_t, rows, repeats):
+    from oracle import mq_oracle as O
+    from paper_2502_00425_b200 import synth
+    seg = synth.segments_from_row_modality(case.seg.row_modality(case.T)[rows])
+    x = case.x[rows]
+    times = []
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        O.linear_w4a8_msq(x, seg.seg_end, seg.seg_mod, s_v, s_t, case.rot_block, qw, s_w)
+        times.append(time.perf_counter() - t0)
+    return times
+
+
+def host_threads():
+    try:
+        return len(os.sched_getaffinity(0))
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def run_reference(args, info):
+    """The CPU oracle as the timed program (rank 0 only)."""
+    if not info.is_main:
+        return
+    from oracle import mq_oracle as O
+    from paper_2502_00425_b200 import synth
+    case = synth.config2()
+    qw, s_w = O.quantize_weight_int4(case.w)
+    s_v, s_t = O.calibrate_static_scales(case.x_calib, case.seg_calib.seg_end, case.seg_calib.seg_mod, ROT)
+    rows = oracle_sample_rows()
+    time_oracle(case, qw, s_w, s_v, s_t, rows, args.warmup)
+    times = time_oracle(case, qw, s_w, s_v, s_t, rows, args.steps)
+    total = float(np.sum(times))
+    value = ops_per_step(len(rows)) * args.steps / total / 1e12
+    sample = f"{len(rows)} of 1088 rows (192 visual + 64 text), all K and N, per step"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8xint4->int32",
+            "data": "synthetic", "config": {"workload": WORKLOAD, "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": host_threads(), "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------ our arm
+class BufferSet:
+    """One independent copy of every device buffer a step touches."""
+
+    def __init__(self, B, torch, dev, case, is_vis, emb_bits, w_layout_src, s_w):
+        T, K, N = case.T, case.K, case.N
+        L = T
+        self.x = torch.from_numpy(case.x_bits.astype(np.int16)).to(dev).view(torch.bfloat16)
+        self.layout = w_layout_src.clone()
+        self.s_w = s_w
+        self.ws = B.new_workspace(T, K, N, ROT)
+        self.y = torch.empty((T, N), dtype=torch.bfloat16, device=dev)
+        self.qx = torch.empty((T, K), dtype=torch.int8, device=dev)
+        self.ws_gemm = B.new_workspace(T, K, N, 0, B.MQ_FLAG_X_IS_INT8)
+        self.emb = torch.from_numpy(emb_bits.astype(np.int16)).to(dev).view(torch.bfloat16)
+        self.emb_u = torch.empty_like(self.emb)
+        self.is_vis = torch.from_numpy(is_vis).to(dev)
+        self.perm = torch.empty(L, dtype=torch.int32, device=dev)
+        self.inv = torch.empty(L, dtype=torch.int32, device=dev)
+        self.n_first = torch.empty(1, dtype=torch.int32, device=dev)
+        self.pos = torch.empty(L, dtype=torch.int32, device=dev)
+        self.seg_end = torch.empty(2, dtype=torch.int32, device=dev)
+        self.seg_mod = torch.empty(2, dtype=torch.uint8, device=dev)
+        self.seg = B.Segments(self.seg_end, self.seg_mod)
+
+    def bytes(self):
+        return sum(t.numel() * t.element_size() for t in (self.x, self.layout, self.ws, self.y, self.emb, self.emb_u))
+
+
+LAUNCHES_PER_STEP = 5  # index scan, row gather, remap, rotation+quantizer, GEMM
+
+
+def run_ours(args, info):
+    import torch
+    from paper_2502_00425_b200 import binding as B
+    from paper_2502_00425_b200 import dist as D
+    from paper_2502_00425_b200 import synth
+
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the product path has no CPU fallback")
+    B.load(build_if_missing=True)
+    torch.cuda.set_device(info.local_rank)
+    dev = torch.device("cuda", info.local_rank)
+    D.init(info)
+    peaks = read_peaks()
+
+    case = synth.config2(seed=D.batch_seed(1, info.rank))
+    is_vis = synth.interleaved_modality(SPANS)
+    assert is_vis.sum() == T_VIS and len(is_vis) == case.T
+    emb_bits = synth.to_bf16_bits(synth.embedding_rows(7 + info.rank, case.T, HIDDEN, is_vis))
+
+    # ---- offline, untimed: calibration and weight packing (on the GPU, through the C ABI)
+    xc = torch.from_numpy(synth.to_bf16_bits(case.x_calib).astype(np.int16)).to(dev).view(torch.bfloat16)
+    state = torch.zeros(2, dtype=torch.int32, device=dev)
+    sv, st = torch.zeros(1, device=dev), torch.zeros(1, device=dev)
+    B.mq_calibrate_static_scales(xc, B.Segments.from_host(case.seg_calib.seg_end, case.seg_calib.seg_mod, dev), ROT,
+                                 state, sv, st)
+    s_vis, s_txt = float(sv.item()), float(st.item())
+    w = torch.from_numpy(case.w).to(dev)
+    s_w = torch.empty(case.N, dtype=torch.float32, device=dev)
+    layout = torch.empty(B.mq_w4_layout_bytes(case.N, case.K), dtype=torch.uint8, device=dev)
+    B.mq_pack_w4(w, None, s_w, layout)
+    del w, xc
+
+    n_sets = args.buffer_sets
+    sets = [BufferSet(B, torch, dev, case, is_vis, emb_bits, layout, s_w) for _ in range(n_sets)]
+    footprint = sum(s.bytes() for s in sets)
+
+    def step(s):
+        B.mq_aifs_reorder(s.emb, s.emb_u, s.is_vis, None, s.perm, s.inv, s.n_first, 0)
+        B.mq_attn_mask_remap(s.perm, None, None, s.n_first, s.pos, s.seg_end, s.seg_mod)
+        B.mq_w4a8_msq_linear(s.x, s.seg, s_vis, s_txt, s.layout, s.s_w, s.y, s.ws, case.N, rot_block=ROT)
+
+    # ---- CUDA graphs: one per buffer set, so that the host only replays
+    graphs = None
+    launch_mode = "eager"
+    if not args.no_graph:
+        try:
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                for s in sets:
+                    step(s)
+            torch.cuda.current_stream().wait_stream(side)
+            torch.cuda.synchronize()
+            graphs = []
+            for s in sets:
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g):
+                    step(s)
+                graphs.append(g)
+            launch_mode = "cuda_graph"
+        except Exception as e:  # capture unavailable: time eager launches instead
+            graphs = None
+            launch_mode = "eager (graph capture failed: %s)" % type(e).__name__
+            torch.cuda.synchronize()
+
+    def run_step(i):
+        if graphs is not None:
+            graphs[i % n_sets].replay()
+        else:
+            step(sets[i % n_sets])
+
+    for i in range(max(args.warmup, 3)):
+        run_step(i)
+    torch.cuda.synchronize()
+
+    # ---- timed region: exactly K steps, device-resident inputs
+    sampler = ClockSampler(info.local_rank)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    D.barrier(dev)
+    torch.cuda.synchronize()
+    sampler.start()
+    e0.record()
+    for i in range(args.steps):
+        run_step(i)
+    e1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    D.barrier(dev)
+    secs = e0.elapsed_time(e1) * 1e-3
+    value_ops, t_max = D.aggregate_throughput(ops_per_step() * args.steps, secs, dev)
+
+    # ---- per-kernel durations, live, with events between the launches (eager, same buffers)
+    ksteps = min(args.steps, 200)
+    names = ["aifs_reorder", "mask_remap", "fwht_quant", "gemm"]
+    acc = {n: 0.0 for n in names}
+    for i in range(ksteps + 3):
+        s = sets[i % n_sets]
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(5)]
+        ev[0].record()
+        B.mq_aifs_reorder(s.emb, s.emb_u, s.is_vis, None, s.perm, s.inv, s.n_first, 0)
+        ev[1].record()
+        B.mq_attn_mask_remap(s.perm, None, None, s.n_first, s.pos, s.seg_end, s.seg_mod)
+        ev[2].record()
+        B.mq_fwht_quant_i8(s.x, s.seg, s_vis, s_txt, ROT, s.qx, None)
+        ev[3].record()
+        B.mq_w4a8_msq_linear(s.qx, s.seg, s_vis, s_txt, s.layout, s.s_w, s.y, s.ws_gemm, case.N)
+        ev[4].record()
+        torch.cuda.synchronize()
+        if i >= 3:
+            for j, n in enumerate(names):
+                acc[n] += ev[j].elapsed_time(ev[j + 1]) * 1e-3
+    kern = {n: acc[n] / ksteps for n in names}
+    status = B.mq_last_device_status(sets[0].ws)
+
+    # ---- end to end through the C ABI with host buffers
+    x_host = torch.from_numpy(case.x_bits.astype(np.int16)).view(torch.bfloat16).pin_memory()
+    y_host = torch.empty((case.T, case.N), dtype=torch.bfloat16).pin_memory()
+    e2e_steps = max(3, min(args.steps, 50))
+
+    def e2e_step(i):
+        s = sets[i % n_sets]
+        s.x.copy_(x_host, non_blocking=True)
+        step(s)
+        y_host.copy_(s.y, non_blocking=True)
+
+    for i in range(3):
+        e2e_step(i)
+    torch.cuda.synchronize()
+    D.barrier(dev)
+    e0.record()
+    for i in range(e2e_steps):
+        e2e_step(i)
+    e1.record()
+    torch.cuda.synchronize()
+    D.barrier(dev)
+    e2e_ops, _ = D.aggregate_throughput(ops_per_step() * e2e_steps, e0.elapsed_time(e1) * 1e-3, dev)
+
+    # ---- CPU baseline: the oracle on this host (rank 0, N = 1 only)
+    cpu = None
+    if info.is_main and info.world == 1 and not args.no_cpu_baseline:
+        from oracle import mq_oracle as O
+        qw, sw_ref = O.quantize_weight_int4(case.w)
+        o_v, o_t = O.calibrate_static_scales(case.x_calib, case.seg_calib.seg_end, case.seg_calib.seg_mod, ROT)
+        rows = np.arange(case.T)
+        times = time_oracle(case, qw, sw_ref, o_v, o_t, rows, 3)
+        cpu = {"value": ops_per_step() / float(np.median(times)) / 1e12, "unit": UNIT, "cores": host_threads(),
+               "kind": "oracle", "sample": "the full config-2 workload (1088 rows), median of 3 passes",
+               "seconds_per_pass": float(np.median(times))}
+
+    if info.is_main:
+        gemm_tops = ops_per_step() / kern["gemm"] / 1e12
+        timed_s = t_max
+        sustained = timed_s > 1.0
+        peak = 2.0 * (peaks["bf16_sustained"] if sustained else peaks["bf16_burst"])
+        quant_bytes = case.T * case.K * 3
+        line = {
+            "metric": METRIC, "value": value_ops / 1e12, "unit": UNIT, "n_gpus": info.world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": 1e3 * t_max / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "int8xint4->int32", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "launch": launch_mode,
+                       "l2": "inputs larger than L2: %d buffer sets, %.0f MB cycled" % (n_sets, footprint / 1e6),
+                       "step": "aifs_reorder + mask_remap + fwht_quant_i8 + w4a8 gemm",
+                       "tokens_per_s": (T_VIS + T_TXT) * args.steps * info.world / t_max},
+            "clocks": clocks,
+            "e2e": {"value": e2e_ops / 1e12, "unit": UNIT, "h2d_bytes_per_step": case.T * case.K * 2,
+                    "d2h_bytes_per_step": case.T * case.N * 2, "steps": e2e_steps},
+            "gpu_launches": LAUNCHES_PER_STEP * args.steps,
+            "roofline": {"bound": "tensor", "kernel": "w4a8_gemm_kernel", "achieved": gemm_tops, "peak": peak,
+                         "unit": "TOP/s", "frac": gemm_tops / peak,
+                         "peak_kind": "2 x measured bf16 %s (%s)" % ("sustained" if sustained else "burst",
+                                                                      peaks["source"]),
+                         "traffic": None, "avg_kernel_us": kern["gemm"] * 1e6},
+            "kernels_us": {n: kern[n] * 1e6 for n in names},
+            "fwht_quant_hbm": {"achieved_gbs": quant_bytes / kern["fwht_quant"] / 1e9, "peak_gbs": peaks["hbm_gbs"],
+                               "frac": quant_bytes / kern["fwht_quant"] / 1e9 / peaks["hbm_gbs"]},
+            "device_status": list(status),
+            "cpu_baseline": cpu,
+        }
+        print(json.dumps(line), flush=True)
+    D.shutdown()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--buffer-sets", type=int, default=4)
+    ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.steps is None:
+        args.steps = 5 if args.impl == "reference" else 2000
+    if args.impl == "reference":
+        args.warmup = min(args.warmup, 3)
+    from paper_2502_00425_b200 import dist as D
+    info = D.rank_info_from_env()
+    if args.impl == "reference":
+        run_reference(args, info)
+    else:
+        run_ours(args, info)
+
+
+if __name__ == "__main__":
+    main()
