@@ -59,6 +59,9 @@ extern "C" {
 #define MQ_FLAG_X_IS_INT8 1u /* X is already int8 codes [T,K]; skip rotation + quantization */
 #define MQ_FLAG_Y_IS_F32 2u  /* write Y as float32 instead of bfloat16 */
 
+/* Size of the library-owned scratch array behind mq_w4a8_msq_linear_noalloc (4 MiB). */
+#define MQ_NOALLOC_WS_BYTES 4194304
+
 /* Rows of the weight tile and columns of the K block of the GEMM weight layout. */
 #define MQ_W_TILE_N 128
 #define MQ_W_TILE_K 128
@@ -198,6 +201,39 @@ int mq_w4a8_msq_linear(const mq_linear_desc* d, const void* X, int64_t ldx,
                        const mq_segments* seg, float s_vis, float s_txt, const void* W_layout,
                        const float* s_w, const float* bias, void* Y, int64_t ldy,
                        int32_t* acc_out, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * mq_w4a8_msq_linear for callers that cannot supply a workspace.  (The paper has no
+ * counterpart: this is an integration aid, not a step of the method.)
+ *
+ * The computation, the arguments and the results are those of mq_w4a8_msq_linear; only
+ * the scratch differs.  Instead of a caller-owned workspace the call uses a fixed
+ * MQ_NOALLOC_WS_BYTES array that is part of the library's device image.  It exists for
+ * code that is handed only its inputs and outputs and may not, or cannot, allocate: a
+ * plugin inside another runtime's inference loop, a decode step that must not risk the
+ * device-wide lock or implicit synchronisation of an allocation, or a process whose device
+ * memory is already owned in full by another pool.  The call performs no cudaMalloc, no
+ * cudaFree and calls no allocating library routine.
+ *
+ *  - Limit: mq_workspace_bytes(d) must not exceed MQ_NOALLOC_WS_BYTES, otherwise
+ *    MQ_ERR_WORKSPACE is returned and nothing is enqueued.  That covers decode-shaped
+ *    problems (for example T = 128, K = 13696, N = 4096); prefill-sized ones need
+ *    mq_w4a8_msq_linear.  The array occupies that much memory on every device the
+ *    library is used on, until the process exits.
+ *  - Set-up: the first call on each device looks up the array's device address (with that
+ *    device current).  Make that first call outside any stream capture.
+ *  - Sharing: every call on a device uses the same array, which keeps what the previous
+ *    call left; the call re-initialises what has to start from zero.  Two calls that
+ *    overlap on the GPU (different streams without an ordering between them) race on it:
+ *    keep all calls on one stream or order them with events.
+ *  - status_out: optional device int32[2] owned by the caller; receives {status, site} as
+ *    mq_last_device_status would report them (MQ_OK / MQ_ERR_TIMEOUT), stream-ordered
+ *    after the kernels.  Pass NULL to skip it.
+ */
+int mq_w4a8_msq_linear_noalloc(const mq_linear_desc* d, const void* X, int64_t ldx,
+                               const mq_segments* seg, float s_vis, float s_txt,
+                               const void* W_layout, const float* s_w, const float* bias, void* Y,
+                               int64_t ldy, int32_t* acc_out, int32_t* status_out, void* stream);
 
 /* Waits for `stream`, then returns the status word kernels left in the workspace
  * (MQ_OK or MQ_ERR_TIMEOUT) and, if site_out != NULL (host), where the wait gave up. */

@@ -22,6 +22,7 @@ MQ_ERR_TIMEOUT = -5
 MQ_ERR_WORKSPACE = -6
 MQ_FLAG_X_IS_INT8 = 1
 MQ_FLAG_Y_IS_F32 = 2
+MQ_NOALLOC_WS_BYTES = 4 << 20
 TEXT, VISUAL = 0, 1
 
 _LIB_NAME = "libmq.so"
@@ -75,6 +76,7 @@ def load(build_if_missing: bool = False):
         "mq_attn_mask_remap": (C.c_int, [vp, vp, vp, vp, i32, vp, vp, vp, vp, vp]),
         "mq_fwht_quant_i8": (C.c_int, [vp, i32, i32, i64, segp, f32, f32, i32, vp, i64, vp, vp]),
         "mq_w4a8_msq_linear": (C.c_int, [descp, vp, i64, segp, f32, f32, vp, vp, vp, vp, i64, vp, vp, sz, vp]),
+        "mq_w4a8_msq_linear_noalloc": (C.c_int, [descp, vp, i64, segp, f32, f32, vp, vp, vp, vp, i64, vp, vp, vp]),
         "mq_last_device_status": (C.c_int, [vp, vp, C.POINTER(C.c_int32)]),
         "mq_reset_device_status": (C.c_int, [vp, vp]),
     }
@@ -88,7 +90,7 @@ def load(build_if_missing: bool = False):
 
 EXPORTED = ["mq_version", "mq_status_string", "mq_workspace_bytes", "mq_w4_layout_bytes",
             "mq_calibrate_static_scales", "mq_pack_w4", "mq_repack_w4", "mq_unpack_w4", "mq_aifs_reorder",
-            "mq_attn_mask_remap", "mq_fwht_quant_i8", "mq_w4a8_msq_linear", "mq_last_device_status",
+            "mq_attn_mask_remap", "mq_fwht_quant_i8", "mq_w4a8_msq_linear", "mq_w4a8_msq_linear_noalloc", "mq_last_device_status",
             "mq_reset_device_status"]
 
 
@@ -225,6 +227,29 @@ def mq_w4a8_msq_linear(x, seg: Segments, s_vis, s_txt, w_layout, s_w, y, ws, N, 
     _check(load().mq_w4a8_msq_linear(C.byref(d), _ptr(x), _ld(x), seg.ref(), float(s_vis), float(s_txt),
                                      _ptr(w_layout), _ptr(s_w), _ptr(bias), _ptr(y), _ld(y), _ptr(acc_out),
                                      _ptr(ws), ws.numel(), _stream()), "mq_w4a8_msq_linear")
+
+
+def mq_w4a8_msq_linear_noalloc(x, seg: Segments, s_vis, s_txt, w_layout, s_w, y, N, rot_block=0, bias=None,
+                               acc_out=None, status_out=None):
+    """mq_w4a8_msq_linear without a workspace argument: the scratch is a fixed 4 MiB array
+    inside the library, for callers that are not in a position to allocate one (see
+    include/mq.h).  Problems whose workspace would exceed MQ_NOALLOC_WS_BYTES raise
+    MqError(MQ_ERR_WORKSPACE).  status_out: optional device int32[2] for {status, site}."""
+    T, K = x.shape
+    flags = 0
+    if x.dtype == torch.int8:
+        flags |= MQ_FLAG_X_IS_INT8
+    else:
+        assert x.dtype == torch.bfloat16
+    if y.dtype == torch.float32:
+        flags |= MQ_FLAG_Y_IS_F32
+    else:
+        assert y.dtype == torch.bfloat16
+    d = mq_linear_desc(T, K, N, rot_block, 0, flags)
+    _check(load().mq_w4a8_msq_linear_noalloc(C.byref(d), _ptr(x), _ld(x), seg.ref(), float(s_vis), float(s_txt),
+                                             _ptr(w_layout), _ptr(s_w), _ptr(bias), _ptr(y), _ld(y),
+                                             _ptr(acc_out), _ptr(status_out), _stream()),
+           "mq_w4a8_msq_linear_noalloc")
 
 
 def mq_last_device_status(ws):
