@@ -42,15 +42,15 @@
 namespace mq {
 namespace {
 
-constexpr int kThreads = 384;
+constexpr int kMaxGroups = 4;                       // expander warp groups (4 warps each)
+constexpr int kMaxThreads = (8 + 4 * kMaxGroups) * 32;
 constexpr int kTileN = MQ_W_TILE_N;    // channels per CTA tile (MMA M)
 constexpr int kBlockK = MQ_W_TILE_K;   // K per pipeline stage
 constexpr int kWTileBytes = 8192;      // packed int4 tile 128 x 128
-constexpr int kMaxActStages = 8;
-constexpr int kMaxWStages = 24;
-constexpr int kMaxAStages = 8;
+constexpr int kMaxStages = 8;    // main ring: activation tiles in shared memory
+constexpr int kMaxWStages = 16;  // packed-weight tiles in shared memory
 constexpr unsigned long long kTimeoutNs = 2000000000ull;
-constexpr int kSmemBudget = 220 * 1024;
+constexpr int kSmemBudget = 226 * 1024;  // of the 227 KB a CTA may use
 
 struct KernelParams {
   int T, K, N;
@@ -62,9 +62,10 @@ struct KernelParams {
   int num_d;       // accumulator buffers (1 or 2)
   int d_stride;    // tensor-memory columns between accumulator buffers
   int a_base;      // first tensor-memory column of the weight stages
-  int num_a;       // weight stages in tensor memory
-  int act_stages;  // activation stages in shared memory
+  int num_a;       // expanded-weight slots in tensor memory (<= stages)
+  int stages;      // main ring: activation stages in shared memory
   int w_stages;    // packed-weight stages in shared memory
+  int groups;      // expander warp groups; group g expands the K blocks with it % groups == g
   SegTable seg;
   float s_vis, s_txt;
   const uint8_t* W_layout;
@@ -79,9 +80,11 @@ struct KernelParams {
 };
 
 struct __align__(8) Barriers {
-  uint64_t act_full[kMaxActStages], act_empty[kMaxActStages];
+  // main ring, one entry per K block in flight.  full: the activation tile has landed (TMA
+  // transaction bytes) AND the four expander warps have written the weight slot (4 arrivals);
+  // done: the MMAs that read the stage have completed (one tcgen05.commit).
+  uint64_t full[kMaxStages], done[kMaxStages];
   uint64_t w_full[kMaxWStages], w_empty[kMaxWStages];
-  uint64_t a_ready[kMaxAStages], a_free[kMaxAStages];
   uint64_t d_full[2], d_empty[2];
   uint64_t drain;
   uint32_t tmem_base;
@@ -141,6 +144,16 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, Barrie
                                           int32_t* status, int site) {
   if (mbar_try_wait(bar, parity)) return true;
   return mbar_wait_slow(bar, parity, sh, status, site);
+}
+
+// Wait used while a CTA winds down after an abort: ignores the abort flag, gives up quietly
+// after `limit_ns` (asynchronous copies and MMAs already issued get that long to finish).
+__device__ __noinline__ void mbar_wait_drain(uint64_t* bar, uint32_t parity, unsigned long long limit_ns) {
+  const unsigned long long t0 = globaltimer_ns();
+  unsigned spins = 0;
+  while (!mbar_try_wait(bar, parity)) {
+    if ((++spins & 15u) == 0u && globaltimer_ns() - t0 > limit_ns) return;
+  }
 }
 
 __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* tmap, int x, int y,
@@ -241,14 +254,14 @@ __device__ __forceinline__ TileCoord decode_tile(const KernelParams& p, int tile
 }
 
 // ------------------------------------------------------------------------------ the kernel
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kMaxThreads, 1)
 w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const KernelParams p) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   // carve: activation stages (1024-aligned), weight stages, barriers, token scales
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int act_stage_bytes = p.TN * kBlockK;
   uint8_t* act_smem = smem;
-  uint8_t* w_smem = act_smem + (size_t)p.act_stages * act_stage_bytes;
+  uint8_t* w_smem = act_smem + (size_t)p.stages * act_stage_bytes;
   Barriers* sh = reinterpret_cast<Barriers*>(w_smem + (size_t)p.w_stages * kWTileBytes);
   float* s_tok = reinterpret_cast<float*>(sh + 1);  // [4 epilogue warps][256]
 
@@ -257,10 +270,9 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const KernelParam
   const int total_tiles = p.n_tn * p.n_tt * p.ksplit;
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < p.act_stages; ++i) { mbar_init(&sh->act_full[i], 1); mbar_init(&sh->act_empty[i], 1); }
-    for (int i = 0; i < p.w_stages; ++i) { mbar_init(&sh->w_full[i], 1); mbar_init(&sh->w_empty[i], 128); }
-    for (int i = 0; i < p.num_a; ++i) { mbar_init(&sh->a_ready[i], 128); mbar_init(&sh->a_free[i], 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(&sh->d_full[i], 1); mbar_init(&sh->d_empty[i], 128); }
+    for (int i = 0; i < p.stages; ++i) { mbar_init(&sh->full[i], 1 + 4); mbar_init(&sh->done[i], 1); }
+    for (int i = 0; i < p.w_stages; ++i) { mbar_init(&sh->w_full[i], 1); mbar_init(&sh->w_empty[i], 4); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&sh->d_full[i], 1); mbar_init(&sh->d_empty[i], 4); }
     mbar_init(&sh->drain, 1);
     sh->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -274,126 +286,156 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const KernelParam
   tc_fence_after();
   const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&sh->tmem_base);
 
+  // Ring positions are kept as (stage, phase) pairs that advance by increment-and-wrap: the
+  // issuing roles are latency-bound, and an integer division per K block would cost more
+  // cycles than the MMAs of that block.  For the same reason the MMA warp waits on ONE
+  // barrier and signals ONE per K block, and runs converged with a single lane issuing.
   if (warp == 0) {
     // ---------------- activation TMA producer
     if (lane == 0) {
-      int it = 0;
-      bool ok = true;
+      int it = 0, s = 0;
+      uint32_t ph = 0;
+      bool wrapped = false, ok = true;
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
         const TileCoord c = decode_tile(p, tile);
+        const int row0 = c.tt * p.TN;
         for (int kb = c.kb0; kb < c.kb1; ++kb, ++it) {
-          const int s = it % p.act_stages;
-          const uint32_t round = it / p.act_stages;
-          if (round > 0 && !(ok = mbar_wait(&sh->act_empty[s], (round - 1) & 1, sh, p.status, 1))) break;
-          mbar_arrive_expect_tx(&sh->act_full[s], act_stage_bytes);
-          tma_load_2d(act_smem + (size_t)s * act_stage_bytes, &tmap_act, kb * kBlockK, c.tt * p.TN,
-                      &sh->act_full[s]);
+          if (wrapped && !(ok = mbar_wait(&sh->done[s], ph ^ 1u, sh, p.status, 1))) break;
+          mbar_arrive_expect_tx(&sh->full[s], act_stage_bytes);
+          tma_load_2d(act_smem + (size_t)s * act_stage_bytes, &tmap_act, kb * kBlockK, row0, &sh->full[s]);
+          if (++s == p.stages) { s = 0; ph ^= 1u; wrapped = true; }
         }
       }
-      if (!ok) {  // drain: wait for copies that are still landing in our shared memory
-        for (int back = 1; back <= p.act_stages && back <= it; ++back) {
+      if (!ok) {
+        // drain: the copies still landing in our shared memory complete their transaction
+        // bytes on `full`, whose phase may never complete once the expanders have stopped;
+        // the bounded wait below gives them time to land before the CTA exits.
+        for (int back = 1; back <= p.stages && back <= it; ++back) {
           const int j = it - back;
-          mbar_wait(&sh->act_full[j % p.act_stages], (j / p.act_stages) & 1, sh, p.status, 90);
+          mbar_wait_drain(&sh->full[j % p.stages], (j / p.stages) & 1, 20000ull);
         }
       }
     }
   } else if (warp == 3) {
     // ---------------- packed-weight bulk-copy producer
     if (lane == 0) {
-      int it = 0;
-      bool ok = true;
+      int it = 0, s = 0;
+      uint32_t ph = 0;
+      bool wrapped = false, ok = true;
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
         const TileCoord c = decode_tile(p, tile);
-        const uint8_t* wsrc = p.W_layout + ((size_t)c.tn * p.kb_total) * kWTileBytes;
-        for (int kb = c.kb0; kb < c.kb1; ++kb, ++it) {
-          const int s = it % p.w_stages;
-          const uint32_t round = it / p.w_stages;
-          if (round > 0 && !(ok = mbar_wait(&sh->w_empty[s], (round - 1) & 1, sh, p.status, 2))) break;
+        const uint8_t* wsrc = p.W_layout + ((size_t)c.tn * p.kb_total + c.kb0) * kWTileBytes;
+        for (int kb = c.kb0; kb < c.kb1; ++kb, ++it, wsrc += kWTileBytes) {
+          if (wrapped && !(ok = mbar_wait(&sh->w_empty[s], ph ^ 1u, sh, p.status, 2))) break;
           mbar_arrive_expect_tx(&sh->w_full[s], kWTileBytes);
-          bulk_load_1d(w_smem + (size_t)s * kWTileBytes, wsrc + (size_t)kb * kWTileBytes, kWTileBytes,
-                       &sh->w_full[s]);
+          bulk_load_1d(w_smem + (size_t)s * kWTileBytes, wsrc, kWTileBytes, &sh->w_full[s]);
+          if (++s == p.w_stages) { s = 0; ph ^= 1u; wrapped = true; }
         }
       }
       if (!ok) {
         for (int back = 1; back <= p.w_stages && back <= it; ++back) {
           const int j = it - back;
-          mbar_wait(&sh->w_full[j % p.w_stages], (j / p.w_stages) & 1, sh, p.status, 91);
+          mbar_wait_drain(&sh->w_full[j % p.w_stages], (j / p.w_stages) & 1, 20000ull);
         }
       }
     }
   } else if (warp == 1) {
-    // ---------------- MMA issuer
-    if (lane == 0) {
-      const uint32_t idesc = make_idesc(p.TN);
-      int it = 0, tile_it = 0;
-      bool ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tile_it) {
-        const TileCoord c = decode_tile(p, tile);
-        const int d = tile_it % p.num_d;
-        const uint32_t d_round = tile_it / p.num_d;
-        if (d_round > 0 && !(ok = mbar_wait(&sh->d_empty[d], (d_round - 1) & 1, sh, p.status, 3))) break;
-        tc_fence_after();
-        const uint32_t d_tmem = tmem_base + (uint32_t)(d * p.d_stride);
-        for (int kb = c.kb0; kb < c.kb1; ++kb, ++it) {
-          const int sa = it % p.act_stages, aa = it % p.num_a;
-          if (!(ok = mbar_wait(&sh->act_full[sa], (it / p.act_stages) & 1, sh, p.status, 4))) break;
-          if (!(ok = mbar_wait(&sh->a_ready[aa], (it / p.num_a) & 1, sh, p.status, 5))) break;
-          tc_fence_after();
-          const uint64_t bdesc = make_b_desc(smem_u32(act_smem + (size_t)sa * act_stage_bytes));
-          const uint32_t a_tmem = tmem_base + (uint32_t)(p.a_base + aa * 32);
-#pragma unroll
-          for (int s = 0; s < 4; ++s)
-            mma_i8_ts(d_tmem, a_tmem + s * 8, bdesc + (uint64_t)(s * 2), idesc, (kb > c.kb0 || s > 0) ? 1u : 0u);
-          tc_commit(&sh->act_empty[sa]);
-          tc_commit(&sh->a_free[aa]);
-        }
-        if (ok) tc_commit(&sh->d_full[d]);
-      }
-      if (!ok) {  // let every MMA already issued finish before tensor memory is freed
-        tc_commit(&sh->drain);
-        mbar_wait(&sh->drain, 0, sh, p.status, 92);
-      }
-    }
-  } else if (warp >= 4 && warp < 8) {
-    // ---------------- weight expanders: packed int4 (smem) -> int8 x16 (tensor memory)
-    const int q = warp & 3;
-    const int r = q * 32 + lane;  // channel row inside the tile == tensor-memory lane
-    int it = 0;
-    bool ok = true;
+    // ---------------- MMA issuer (whole warp converged, lane 0 issues)
+    const uint32_t idesc = make_idesc(p.TN);
+    const uint64_t bdesc0 = make_b_desc(smem_u32(act_smem));
+    const uint32_t bdesc_step = (uint32_t)(act_stage_bytes >> 4);
+    int s = 0, a = 0, d = 0;
+    uint32_t ph = 0, ph_d = 0;
+    bool d_wrapped = false, ok = true;
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
       const TileCoord c = decode_tile(p, tile);
-      for (int kb = c.kb0; kb < c.kb1; ++kb, ++it) {
-        const int sw = it % p.w_stages, aa = it % p.num_a;
-        if (!(ok = warp_all(mbar_wait(&sh->w_full[sw], (it / p.w_stages) & 1, sh, p.status, 6)))) break;
-        const uint4* src = reinterpret_cast<const uint4*>(w_smem + (size_t)sw * kWTileBytes) + r;
-        uint32_t regs[32];
-#pragma unroll
-        for (int jj = 0; jj < 4; ++jj) {
-          const uint4 w = src[jj * 128];
-          const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            regs[jj * 8 + 2 * i] = (ww[i] << 4) & 0xF0F0F0F0u;   // codes k0..k0+3, each x16
-            regs[jj * 8 + 2 * i + 1] = ww[i] & 0xF0F0F0F0u;      // codes k0+4..k0+7, each x16
-          }
-        }
-        mbar_arrive(&sh->w_empty[sw]);
-        const uint32_t a_round = it / p.num_a;
-        if (a_round > 0 && !(ok = warp_all(mbar_wait(&sh->a_free[aa], (a_round - 1) & 1, sh, p.status, 7)))) break;
+      if (d_wrapped && !(ok = warp_all(mbar_wait(&sh->d_empty[d], ph_d ^ 1u, sh, p.status, 3)))) break;
+      tc_fence_after();
+      const uint32_t d_tmem = tmem_base + (uint32_t)(d * p.d_stride);
+      uint32_t accumulate = 0;
+      for (int kb = c.kb0; kb < c.kb1; ++kb) {
+        if (!(ok = warp_all(mbar_wait(&sh->full[s], ph, sh, p.status, 4)))) break;
         tc_fence_after();
-        tmem_st_x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(p.a_base + aa * 32), regs);
-        tmem_wait_st();
-        tc_fence_before();
-        mbar_arrive(&sh->a_ready[aa]);
+        if (lane == 0) {
+          const uint64_t bdesc = bdesc0 + (uint64_t)((uint32_t)s * bdesc_step);
+          const uint32_t a_tmem = tmem_base + (uint32_t)(p.a_base + a * 32);
+#pragma unroll
+          for (int k4 = 0; k4 < 4; ++k4)
+            mma_i8_ts(d_tmem, a_tmem + k4 * 8, bdesc + (uint64_t)(k4 * 2), idesc, (accumulate | (uint32_t)k4));
+          tc_commit(&sh->done[s]);
+        }
+        accumulate = 1;
+        if (++s == p.stages) { s = 0; ph ^= 1u; }
+        if (++a == p.num_a) a = 0;
       }
+      if (ok && lane == 0) tc_commit(&sh->d_full[d]);
+      if (++d == p.num_d) { d = 0; ph_d ^= 1u; d_wrapped = true; }
     }
-  } else if (warp >= 8) {
+    if (!ok && lane == 0) {  // let every MMA already issued finish before tensor memory is freed
+      tc_commit(&sh->drain);
+      mbar_wait_drain(&sh->drain, 0, 2000000ull);
+    }
+  } else if (warp >= 4 && warp < 4 + 4 * p.groups) {
+    // ---------------- weight expanders: packed int4 (smem) -> int8 x16 (tensor memory)
+    // Group g of four warps takes the K blocks g, g + groups, g + 2 groups, ... of this CTA's
+    // stream, so the latency of one block's chain (wait, load, expand, tcgen05.st, wait::st)
+    // overlaps with the other groups' blocks.  Needs groups <= w_stages and groups <= num_a
+    // <= stages.  Block `it` uses weight slot it % num_a, free once the MMAs of block
+    // it - num_a are done, i.e. once done[(it - num_a) % stages] has completed that round.
+    const int q = warp & 3;
+    const int grp = (warp - 4) >> 2;
+    const int r = q * 32 + lane;  // channel row inside the tile == tensor-memory lane
+    int total_it = 0;
+    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+      const TileCoord c = decode_tile(p, tile);
+      total_it += c.kb1 - c.kb0;
+    }
+    int sw = grp, a = grp, s = grp;
+    uint32_t ph_w = 0, ph = 0;
+    bool ok = true;
+    for (int it = grp; it < total_it && ok; it += p.groups) {
+      if (!(ok = warp_all(mbar_wait(&sh->w_full[sw], ph_w, sh, p.status, 6)))) break;
+      const uint4* src = reinterpret_cast<const uint4*>(w_smem + (size_t)sw * kWTileBytes) + r;
+      uint32_t regs[32];
+#pragma unroll
+      for (int jj = 0; jj < 4; ++jj) {
+        const uint4 w = src[jj * 128];
+        const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          regs[jj * 8 + 2 * i] = (ww[i] << 4) & 0xF0F0F0F0u;   // codes k0..k0+3, each x16
+          regs[jj * 8 + 2 * i + 1] = ww[i] & 0xF0F0F0F0u;      // codes k0+4..k0+7, each x16
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sh->w_empty[sw]);
+      if (it >= p.num_a) {
+        // stage and parity of block it - num_a, derived from those of block it
+        const int fs = s >= p.num_a ? s - p.num_a : s - p.num_a + p.stages;
+        const uint32_t fph = s >= p.num_a ? ph : ph ^ 1u;
+        if (!(ok = warp_all(mbar_wait(&sh->done[fs], fph, sh, p.status, 7)))) break;
+      }
+      tc_fence_after();
+      tmem_st_x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(p.a_base + a * 32), regs);
+      tmem_wait_st();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sh->full[s]);
+      sw += p.groups;
+      if (sw >= p.w_stages) { sw -= p.w_stages; ph_w ^= 1u; }
+      s += p.groups;
+      if (s >= p.stages) { s -= p.stages; ph ^= 1u; }
+      a += p.groups;
+      if (a >= p.num_a) a -= p.num_a;
+    }
+  } else if (warp >= 4 + 4 * p.groups) {
     // ---------------- epilogue: tensor memory -> dequant -> global
     const int q = warp & 3;
     float* stok = s_tok + q * 256;  // private to this warp: no cross-warp barrier to strand on abort
-    int tile_it = 0;
+    int d = 0;
+    uint32_t ph_d = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tile_it) {
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
       const TileCoord c = decode_tile(p, tile);
       const int t0 = c.tt * p.TN;
       __syncwarp();
@@ -402,8 +444,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const KernelParam
         stok[j] = (t < p.T && thread_row_modality(p.seg, t) == MQ_VISUAL) ? p.s_vis : p.s_txt;
       }
       __syncwarp();
-      const int d = tile_it % p.num_d;
-      if (!(ok = warp_all(mbar_wait(&sh->d_full[d], (tile_it / p.num_d) & 1, sh, p.status, 8)))) break;
+      if (!(ok = warp_all(mbar_wait(&sh->d_full[d], ph_d, sh, p.status, 8)))) break;
       tc_fence_after();
       const int n = c.tn * kTileN + q * 32 + lane;
       const bool n_ok = n < p.N;
@@ -435,7 +476,9 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const KernelParam
         }
       }
       tc_fence_before();
-      mbar_arrive(&sh->d_empty[d]);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sh->d_empty[d]);
+      if (++d == p.num_d) { d = 0; ph_d ^= 1u; }
     }
   }
 
@@ -482,7 +525,7 @@ EncodeTiledFn get_encode_fn() {
 }
 
 struct Plan {
-  int TN, n_tt, n_tn, ksplit, num_d, d_stride, a_base, num_a, act_stages, w_stages, grid;
+  int TN, n_tt, n_tn, ksplit, num_d, d_stride, a_base, num_a, stages, w_stages, grid, groups;
   size_t smem;
 };
 
@@ -516,7 +559,7 @@ Plan make_plan(int T, int K, int N) {
   pl.num_d = pl.d_stride <= 192 ? 2 : 1;
   pl.a_base = pl.num_d * pl.d_stride;
   pl.num_a = (512 - pl.a_base) / 32;
-  if (pl.num_a > kMaxAStages) pl.num_a = kMaxAStages;
+  if (pl.num_a > kMaxStages) pl.num_a = kMaxStages;
   // split K when the tiles alone cannot fill the machine (small T: weight streaming)
   const long long tiles = (long long)pl.n_tn * n_tt;
   int ksplit = 1;
@@ -529,15 +572,22 @@ Plan make_plan(int T, int K, int N) {
     ksplit = (kb_total + per - 1) / per;  // no empty split
   }
   pl.ksplit = ksplit;
+  // shared memory: as many activation stages as fit beside a minimum of 4 weight stages, then
+  // the rest to the weight ring
   const int act_stage = TN * kBlockK;
   const size_t fixed = 1024 + sizeof(Barriers) + 4 * 256 * sizeof(float);
-  int act_stages = TN <= 64 ? 8 : (TN <= 128 ? 6 : 4);
-  int w_stages = (int)((kSmemBudget - fixed - (size_t)act_stages * act_stage) / kWTileBytes);
+  int stages = (int)((kSmemBudget - fixed - 4 * (size_t)kWTileBytes) / act_stage);
+  if (stages > kMaxStages) stages = kMaxStages;
+  if (stages < pl.num_a) pl.num_a = stages;
+  int w_stages = (int)((kSmemBudget - fixed - (size_t)stages * act_stage) / kWTileBytes);
   if (w_stages > kMaxWStages) w_stages = kMaxWStages;
-  if (TN > 128 && w_stages > 8) w_stages = 8;
-  pl.act_stages = act_stages;
+  pl.stages = stages;
   pl.w_stages = w_stages;
-  pl.smem = fixed + (size_t)act_stages * act_stage + (size_t)w_stages * kWTileBytes;
+  pl.smem = fixed + (size_t)stages * act_stage + (size_t)w_stages * kWTileBytes;
+  pl.groups = 1;
+  if (pl.groups > pl.num_a) pl.groups = pl.num_a;
+  if (pl.groups > pl.w_stages) pl.groups = pl.w_stages;
+  if (pl.groups < 1) pl.groups = 1;
   const long long total = tiles * ksplit;
   pl.grid = (int)(total < sms ? total : sms);
   return pl;
@@ -569,7 +619,7 @@ int launch_gemm(const GemmArgs& a, cudaStream_t st) {
 
   static bool attr_set = false;
   if (!attr_set) {
-    if (cudaFuncSetAttribute(w4a8_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 2048) !=
+    if (cudaFuncSetAttribute(w4a8_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget) !=
         cudaSuccess)
       return MQ_ERR_CUDA;
     attr_set = true;
@@ -580,7 +630,7 @@ int launch_gemm(const GemmArgs& a, cudaStream_t st) {
   p.TN = pl.TN; p.n_tn = pl.n_tn; p.n_tt = pl.n_tt; p.ksplit = pl.ksplit;
   p.kb_total = (a.K + kBlockK - 1) / kBlockK;
   p.num_d = pl.num_d; p.d_stride = pl.d_stride; p.a_base = pl.a_base; p.num_a = pl.num_a;
-  p.act_stages = pl.act_stages; p.w_stages = pl.w_stages;
+  p.stages = pl.stages; p.w_stages = pl.w_stages; p.groups = pl.groups;
   p.seg = a.seg; p.s_vis = a.s_vis; p.s_txt = a.s_txt;
   p.W_layout = static_cast<const uint8_t*>(a.W_layout);
   p.s_w = a.s_w; p.bias = a.bias; p.Y = a.Y; p.ldy = a.ldy; p.y_is_f32 = a.y_is_f32;
@@ -590,7 +640,7 @@ int launch_gemm(const GemmArgs& a, cudaStream_t st) {
     if (!a.splitk_acc) return MQ_ERR_WORKSPACE;
     if (cudaMemsetAsync(a.splitk_acc, 0, (size_t)a.T * a.N * sizeof(int32_t), st) != cudaSuccess) return MQ_ERR_CUDA;
   }
-  w4a8_gemm_kernel<<<pl.grid, kThreads, pl.smem, st>>>(tmap, p);
+  w4a8_gemm_kernel<<<pl.grid, (8 + 4 * pl.groups) * 32, pl.smem, st>>>(tmap, p);
   if (cudaGetLastError() != cudaSuccess) return MQ_ERR_CUDA;
   if (pl.ksplit > 1) {
     const int64_t n = (int64_t)a.T * a.N;
