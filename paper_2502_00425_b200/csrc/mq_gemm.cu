@@ -42,7 +42,7 @@
 namespace mq {
 namespace {
 
-constexpr int kMaxGroups = 4;                       // expander warp groups (4 warps each)
+constexpr int kMaxGroups = 2;                       // expander warp groups (4 warps each)
 constexpr int kMaxThreads = (8 + 4 * kMaxGroups) * 32;
 constexpr int kTileN = MQ_W_TILE_N;    // channels per CTA tile (MMA M)
 constexpr int kBlockK = MQ_W_TILE_K;   // K per pipeline stage
@@ -59,6 +59,8 @@ struct KernelParams {
   int n_tt;        // token tiles
   int ksplit;      // K splits (1 = direct epilogue)
   int kb_total;    // K blocks
+  int kb_per_split;        // K blocks per split (the last split may have fewer)
+  int step_tn, step_tt, step_ks;  // the grid stride written in (n_tn, n_tt) mixed radix
   int num_d;       // accumulator buffers (1 or 2)
   int d_stride;    // tensor-memory columns between accumulator buffers
   int a_base;      // first tensor-memory column of the weight stages
@@ -79,7 +81,7 @@ struct KernelParams {
   int32_t* status;
 };
 
-struct __align__(8) Barriers {
+struct __align__(16) Barriers {
   // main ring, one entry per K block in flight.  full: the activation tile has landed (TMA
   // transaction bytes) AND the four expander warps have written the weight slot (4 arrivals);
   // done: the MMAs that read the stage have completed (one tcgen05.commit).
@@ -225,6 +227,17 @@ __device__ __forceinline__ void tmem_ld_x16(uint32_t taddr, uint32_t (&r)[16]) {
 }
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
+// True in exactly one lane of a converged warp.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "elect.sync _|p, 0xffffffff;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(pred));
+  return pred != 0;
+}
+
 // Warp-uniform verdict of a bounded wait, so that .sync.aligned instructions stay converged.
 __device__ __forceinline__ bool warp_all(bool ok) { return __all_sync(0xffffffffu, ok) != 0; }
 
@@ -238,19 +251,123 @@ __device__ __forceinline__ uint32_t make_idesc(int n) {
   return (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileN >> 4) << 24);
 }
 
-struct TileCoord {
-  int tn, tt, kb0, kb1;
+// Tile t of the launch is (channel tile, token tile, K split) = (t % n_tn, (t / n_tn) % n_tt,
+// t / (n_tn * n_tt)); CTA b owns tiles b, b + grid, b + 2 grid, ...  The first one is decoded
+// with divisions once; each further one is reached by adding the (host-decomposed) grid
+// stride digit by digit, because a division per tile sits on the MMA warp's critical path.
+struct TileIter {
+  int tn, tt, ks;
+  __device__ __forceinline__ void init(const KernelParams& p, int tile) {
+    tn = tile % p.n_tn;
+    const int rest = tile / p.n_tn;
+    tt = rest % p.n_tt;
+    ks = rest / p.n_tt;
+  }
+  __device__ __forceinline__ bool valid(const KernelParams& p) const { return ks < p.ksplit; }
+  __device__ __forceinline__ void next(const KernelParams& p) {
+    tn += p.step_tn;
+    int carry = tn >= p.n_tn ? 1 : 0;
+    tn -= carry * p.n_tn;
+    tt += p.step_tt + carry;
+    carry = tt >= p.n_tt ? 1 : 0;
+    tt -= carry * p.n_tt;
+    ks += p.step_ks + carry;
+  }
+  __device__ __forceinline__ int kb0(const KernelParams& p) const { return ks * p.kb_per_split; }
+  __device__ __forceinline__ int kb1(const KernelParams& p) const { return min(p.kb_total, kb0(p) + p.kb_per_split); }
 };
-__device__ __forceinline__ TileCoord decode_tile(const KernelParams& p, int tile) {
-  TileCoord c;
-  c.tn = tile % p.n_tn;
-  const int rest = tile / p.n_tn;
-  c.tt = rest % p.n_tt;
-  const int ks = rest / p.n_tt;
-  const int per = (p.kb_total + p.ksplit - 1) / p.ksplit;
-  c.kb0 = ks * per;
-  c.kb1 = min(p.kb_total, c.kb0 + per);
-  return c;
+
+// ------------------------------------------------------------------------------ epilogue
+// What the epilogue does with an accumulator is fixed per launch.  The product configurations
+// (bf16 output, with or without bias, and the split-K partial sums) are compiled separately so
+// that their per-element code has no branches; the debug outputs (accumulator dump, float32
+// output) share one generic variant that tests its flags at run time.
+enum : int { kEpiSplitK = 1, kEpiAcc = 2, kEpiF32 = 4, kEpiBias = 8, kEpiGeneric = 16, kEpiStaged = 32 };
+
+// 16 token columns of one channel (this lane's n): dequantize and store, or add into the
+// split-K sums.  `nvalid` (1..16) masks the ragged end of the token range.
+template <int MODE>
+__device__ __forceinline__ void epilogue_chunk(const KernelParams& p, const uint32_t (&v)[16], int t_first,
+                                               int nvalid, int n, bool n_ok, float sw, float bs,
+                                               const float* stok, __nv_bfloat16* stage) {
+  if (!(MODE & kEpiStaged) && !n_ok) return;
+  if (MODE & kEpiSplitK) {
+    int32_t* dst = p.splitk_acc + (size_t)t_first * p.N + n;
+#pragma unroll
+    for (int j = 0; j < 16; ++j)
+      if (j < nvalid) atomicAdd(dst + (size_t)j * p.N, ((int)v[j]) >> 4);  // the MMA saw 16 * q_w
+    return;
+  }
+  if (MODE & kEpiGeneric) {
+#pragma unroll 1
+    for (int j = 0; j < nvalid; ++j) {
+      const int acc = ((int)v[j]) >> 4;
+      const size_t t = (size_t)(t_first + j);
+      if (p.acc_out) p.acc_out[t * p.N + n] = acc;
+      float y = __fmul_rn((float)acc, __fmul_rn(stok[j], sw));
+      if (p.bias) y = __fadd_rn(y, bs);
+      if (p.y_is_f32) static_cast<float*>(p.Y)[t * p.ldy + n] = y;
+      else static_cast<__nv_bfloat16*>(p.Y)[t * p.ldy + n] = __float2bfloat16_rn(y);
+    }
+    return;
+  }
+  int32_t* acc_dst = (MODE & kEpiAcc) ? p.acc_out + (size_t)t_first * p.N + n : nullptr;
+  float* y32 = static_cast<float*>(p.Y) + (size_t)t_first * p.ldy + n;
+  __nv_bfloat16* y16 = static_cast<__nv_bfloat16*>(p.Y) + (size_t)t_first * p.ldy + n;
+  float y[16];
+#pragma unroll
+  for (int j = 0; j < 16; ++j) {
+    y[j] = __fmul_rn((float)(((int)v[j]) >> 4), __fmul_rn(stok[j], sw));  // the MMA saw 16 * q_w
+    if (MODE & kEpiBias) y[j] = __fadd_rn(y[j], bs);
+  }
+  if (MODE & kEpiStaged) {
+    // bf16 output: transpose the 16 x 32 (token x channel) block through this warp's staging
+    // buffer so that every lane stores 16 bytes (8 channels of one token) instead of 2.
+    const int lane = threadIdx.x & 31;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) stage[j * 32 + lane] = __float2bfloat16_rn(y[j]);
+    __syncwarp();
+    const int n8 = n - lane + (lane & 3) * 8;  // first of this lane's 8 channels
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const int row = (lane >> 2) + 8 * h;
+      if (row < nvalid && n8 < p.N) {
+        const uint4 val = *reinterpret_cast<const uint4*>(stage + row * 32 + (lane & 3) * 8);
+        *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.Y) + (size_t)(t_first + row) * p.ldy + n8) = val;
+      }
+    }
+    __syncwarp();
+    return;
+  }
+#pragma unroll
+  for (int j = 0; j < 16; ++j) {
+    if (j < nvalid) {
+      if (MODE & kEpiAcc) acc_dst[(size_t)j * p.N] = ((int)v[j]) >> 4;
+      if (MODE & kEpiF32) y32[(size_t)j * p.ldy] = y[j];
+      else y16[(size_t)j * p.ldy] = __float2bfloat16_rn(y[j]);
+    }
+  }
+}
+
+// One accumulator tile of this warp's 32 channels.  Two register buffers: the tensor-memory
+// load of the next 16 columns is in flight while the current 16 are converted and stored.
+template <int MODE>
+__device__ __forceinline__ void epilogue_tile(const KernelParams& p, uint32_t d_tmem, int t0, int n, bool n_ok,
+                                              float sw, float bs, const float* stok, __nv_bfloat16* stage) {
+  const int ncols = min(p.TN, p.T - t0);  // valid token columns of this tile (> 0)
+  uint32_t va[16], vb[16];
+  tmem_ld_x16(d_tmem, va);
+  for (int cc = 0; cc < ncols; cc += 32) {
+    tmem_wait_ld();
+    const bool has_b = cc + 16 < ncols;
+    if (has_b) tmem_ld_x16(d_tmem + cc + 16, vb);
+    epilogue_chunk<MODE>(p, va, t0 + cc, min(16, ncols - cc), n, n_ok, sw, bs, stok + cc, stage);
+    if (has_b) {
+      tmem_wait_ld();
+      if (cc + 32 < ncols) tmem_ld_x16(d_tmem + cc + 32, va);
+      epilogue_chunk<MODE>(p, vb, t0 + cc + 16, min(16, ncols - cc - 16), n, n_ok, sw, bs, stok + cc + 16, stage);
+    }
+  }
 }
 
 // ------------------------------------------------------------------------------ the kernel
@@ -263,13 +380,15 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const KernelParam
   uint8_t* act_smem = smem;
   uint8_t* w_smem = act_smem + (size_t)p.stages * act_stage_bytes;
   Barriers* sh = reinterpret_cast<Barriers*>(w_smem + (size_t)p.w_stages * kWTileBytes);
-  float* s_tok = reinterpret_cast<float*>(sh + 1);  // [4 epilogue warps][256]
+  float* s_tok = reinterpret_cast<float*>(sh + 1);  // [4 epilogue warps][256], then bf16 staging [4][16 x 32]
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const int total_tiles = p.n_tn * p.n_tt * p.ksplit;
+  TileIter first;
+  first.init(p, blockIdx.x);  // the divisions overlap with barrier set-up and the TMEM allocation
 
   if (threadIdx.x == 0) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmap_act)) : "memory");
     for (int i = 0; i < p.stages; ++i) { mbar_init(&sh->full[i], 1 + 4); mbar_init(&sh->done[i], 1); }
     for (int i = 0; i < p.w_stages; ++i) { mbar_init(&sh->w_full[i], 1); mbar_init(&sh->w_empty[i], 4); }
     for (int i = 0; i < 2; ++i) { mbar_init(&sh->d_full[i], 1); mbar_init(&sh->d_empty[i], 4); }
@@ -296,10 +415,9 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const KernelParam
       int it = 0, s = 0;
       uint32_t ph = 0;
       bool wrapped = false, ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-        const TileCoord c = decode_tile(p, tile);
+      for (TileIter c = first; c.valid(p) && ok; c.next(p)) {
         const int row0 = c.tt * p.TN;
-        for (int kb = c.kb0; kb < c.kb1; ++kb, ++it) {
+        for (int kb = c.kb0(p), kb_end = c.kb1(p); kb < kb_end; ++kb, ++it) {
           if (wrapped && !(ok = mbar_wait(&sh->done[s], ph ^ 1u, sh, p.status, 1))) break;
           mbar_arrive_expect_tx(&sh->full[s], act_stage_bytes);
           tma_load_2d(act_smem + (size_t)s * act_stage_bytes, &tmap_act, kb * kBlockK, row0, &sh->full[s]);
@@ -322,10 +440,9 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const KernelParam
       int it = 0, s = 0;
       uint32_t ph = 0;
       bool wrapped = false, ok = true;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-        const TileCoord c = decode_tile(p, tile);
-        const uint8_t* wsrc = p.W_layout + ((size_t)c.tn * p.kb_total + c.kb0) * kWTileBytes;
-        for (int kb = c.kb0; kb < c.kb1; ++kb, ++it, wsrc += kWTileBytes) {
+      for (TileIter c = first; c.valid(p) && ok; c.next(p)) {
+        const uint8_t* wsrc = p.W_layout + ((size_t)c.tn * p.kb_total + c.kb0(p)) * kWTileBytes;
+        for (int kb = c.kb0(p), kb_end = c.kb1(p); kb < kb_end; ++kb, ++it, wsrc += kWTileBytes) {
           if (wrapped && !(ok = mbar_wait(&sh->w_empty[s], ph ^ 1u, sh, p.status, 2))) break;
           mbar_arrive_expect_tx(&sh->w_full[s], kWTileBytes);
           bulk_load_1d(w_smem + (size_t)s * kWTileBytes, wsrc, kWTileBytes, &sh->w_full[s]);
@@ -347,18 +464,18 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const KernelParam
     int s = 0, a = 0, d = 0;
     uint32_t ph = 0, ph_d = 0;
     bool d_wrapped = false, ok = true;
-    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-      const TileCoord c = decode_tile(p, tile);
+    for (TileIter c = first; c.valid(p) && ok; c.next(p)) {
       if (d_wrapped && !(ok = warp_all(mbar_wait(&sh->d_empty[d], ph_d ^ 1u, sh, p.status, 3)))) break;
       tc_fence_after();
       const uint32_t d_tmem = tmem_base + (uint32_t)(d * p.d_stride);
       uint32_t accumulate = 0;
-      for (int kb = c.kb0; kb < c.kb1; ++kb) {
+      for (int kb = c.kb0(p), kb_end = c.kb1(p); kb < kb_end; ++kb) {
         if (!(ok = warp_all(mbar_wait(&sh->full[s], ph, sh, p.status, 4)))) break;
         tc_fence_after();
-        if (lane == 0) {
-          const uint64_t bdesc = bdesc0 + (uint64_t)((uint32_t)s * bdesc_step);
-          const uint32_t a_tmem = tmem_base + (uint32_t)(p.a_base + a * 32);
+        // operands are computed by the whole (converged) warp so that they stay warp-uniform
+        const uint64_t bdesc = bdesc0 + (uint64_t)((uint32_t)s * bdesc_step);
+        const uint32_t a_tmem = tmem_base + (uint32_t)(p.a_base + a * 32);
+        if (elect_one()) {
 #pragma unroll
           for (int k4 = 0; k4 < 4; ++k4)
             mma_i8_ts(d_tmem, a_tmem + k4 * 8, bdesc + (uint64_t)(k4 * 2), idesc, (accumulate | (uint32_t)k4));
@@ -386,10 +503,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const KernelParam
     const int grp = (warp - 4) >> 2;
     const int r = q * 32 + lane;  // channel row inside the tile == tensor-memory lane
     int total_it = 0;
-    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
-      const TileCoord c = decode_tile(p, tile);
-      total_it += c.kb1 - c.kb0;
-    }
+    for (TileIter c = first; c.valid(p); c.next(p)) total_it += c.kb1(p) - c.kb0(p);
     int sw = grp, a = grp, s = grp;
     uint32_t ph_w = 0, ph = 0;
     bool ok = true;
@@ -432,11 +546,14 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const KernelParam
     // ---------------- epilogue: tensor memory -> dequant -> global
     const int q = warp & 3;
     float* stok = s_tok + q * 256;  // private to this warp: no cross-warp barrier to strand on abort
+    __nv_bfloat16* stage = reinterpret_cast<__nv_bfloat16*>(s_tok + 4 * 256) + q * (16 * 32);
+    // bf16 rows whose pitch keeps 16-byte stores aligned take the staged path
+    const bool plain = !p.acc_out && !p.y_is_f32 && (p.ldy % 8) == 0;
+    const int epi_mode = p.ksplit > 1 ? kEpiSplitK : (plain ? (kEpiStaged | (p.bias ? kEpiBias : 0)) : kEpiGeneric);
     int d = 0;
     uint32_t ph_d = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-      const TileCoord c = decode_tile(p, tile);
+    for (TileIter c = first; c.valid(p) && ok; c.next(p)) {
       const int t0 = c.tt * p.TN;
       __syncwarp();
       for (int j = lane; j < p.TN; j += 32) {
@@ -451,29 +568,11 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const KernelParam
       const float sw = n_ok ? p.s_w[n] : 0.0f;
       const float bs = (n_ok && p.bias) ? p.bias[n] : 0.0f;
       const uint32_t d_tmem = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(d * p.d_stride);
-      for (int cc = 0; cc < p.TN; cc += 16) {
-        uint32_t v[16];
-        tmem_ld_x16(d_tmem + cc, v);
-        tmem_wait_ld();
-        if (n_ok) {
-#pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            const int t = t0 + cc + j;
-            if (t >= p.T) break;
-            const int acc = ((int)v[j]) >> 4;  // the MMA saw 16 * q_w
-            const size_t o = (size_t)t * p.N + n;
-            if (p.ksplit > 1) {
-              atomicAdd(&p.splitk_acc[o], acc);
-            } else {
-              if (p.acc_out) p.acc_out[o] = acc;
-              float y = __fmul_rn((float)acc, __fmul_rn(stok[cc + j], sw));
-              if (p.bias) y = __fadd_rn(y, bs);
-              const size_t oy = (size_t)t * p.ldy + n;
-              if (p.y_is_f32) static_cast<float*>(p.Y)[oy] = y;
-              else static_cast<__nv_bfloat16*>(p.Y)[oy] = __float2bfloat16_rn(y);
-            }
-          }
-        }
+      switch (epi_mode) {
+#define MQ_EPI_CASE(M) case M: epilogue_tile<M>(p, d_tmem, t0, n, n_ok, sw, bs, stok, stage); break;
+        MQ_EPI_CASE(kEpiStaged) MQ_EPI_CASE(kEpiStaged | kEpiBias) MQ_EPI_CASE(kEpiSplitK)
+#undef MQ_EPI_CASE
+        default: epilogue_tile<kEpiGeneric>(p, d_tmem, t0, n, n_ok, sw, bs, stok, stage); break;
       }
       tc_fence_before();
       __syncwarp();
@@ -575,7 +674,7 @@ Plan make_plan(int T, int K, int N) {
   // shared memory: as many activation stages as fit beside a minimum of 4 weight stages, then
   // the rest to the weight ring
   const int act_stage = TN * kBlockK;
-  const size_t fixed = 1024 + sizeof(Barriers) + 4 * 256 * sizeof(float);
+  const size_t fixed = 1024 + sizeof(Barriers) + 4 * 256 * sizeof(float) + 4 * 16 * 32 * 2;
   int stages = (int)((kSmemBudget - fixed - 4 * (size_t)kWTileBytes) / act_stage);
   if (stages > kMaxStages) stages = kMaxStages;
   if (stages < pl.num_a) pl.num_a = stages;
@@ -584,7 +683,7 @@ Plan make_plan(int T, int K, int N) {
   pl.stages = stages;
   pl.w_stages = w_stages;
   pl.smem = fixed + (size_t)stages * act_stage + (size_t)w_stages * kWTileBytes;
-  pl.groups = 1;
+  pl.groups = 2;
   if (pl.groups > pl.num_a) pl.groups = pl.num_a;
   if (pl.groups > pl.w_stages) pl.groups = pl.w_stages;
   if (pl.groups < 1) pl.groups = 1;
@@ -629,6 +728,10 @@ int launch_gemm(const GemmArgs& a, cudaStream_t st) {
   p.T = a.T; p.K = a.K; p.N = a.N;
   p.TN = pl.TN; p.n_tn = pl.n_tn; p.n_tt = pl.n_tt; p.ksplit = pl.ksplit;
   p.kb_total = (a.K + kBlockK - 1) / kBlockK;
+  p.kb_per_split = (p.kb_total + pl.ksplit - 1) / pl.ksplit;
+  p.step_tn = pl.grid % pl.n_tn;
+  p.step_tt = (pl.grid / pl.n_tn) % pl.n_tt;
+  p.step_ks = (pl.grid / pl.n_tn) / pl.n_tt;
   p.num_d = pl.num_d; p.d_stride = pl.d_stride; p.a_base = pl.a_base; p.num_a = pl.num_a;
   p.stages = pl.stages; p.w_stages = pl.w_stages; p.groups = pl.groups;
   p.seg = a.seg; p.s_vis = a.s_vis; p.s_txt = a.s_txt;
