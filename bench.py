@@ -257,9 +257,12 @@ def run_ours(args, info):
         if events is not None:
             events[len(kernels)].record()
 
-    # ---- CUDA graphs: one per buffer set, so that the host only replays.  Timing events that
-    # are recorded as graph nodes ("external" events) bracket every kernel inside the graphs.
-    graphs, set_events = None, None
+    # ---- CUDA graphs: one per buffer set, so that the host only replays.  A second family of
+    # graphs of the same step carries timing events recorded as graph nodes ("external" events)
+    # around every kernel; it is replayed after the timed region for the per-kernel durations
+    # (event nodes between kernels would keep them from overlapping their launch with the
+    # predecessor's tail, so the timed graphs have none).
+    graphs, ev_graphs, set_events = None, None, None
     launch_mode = "eager"
     if not args.no_graph:
         try:
@@ -279,11 +282,18 @@ def run_ours(args, info):
             for i, s in enumerate(sets):
                 g = torch.cuda.CUDAGraph()
                 with torch.cuda.graph(g):
-                    step(s, set_events[i] if set_events else None)
+                    step(s)
                 graphs.append(g)
+            if set_events is not None:
+                ev_graphs = []
+                for i, s in enumerate(sets):
+                    g = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(g):
+                        step(s, set_events[i])
+                    ev_graphs.append(g)
             launch_mode = "cuda_graph"
         except Exception as e:  # capture unavailable: time eager launches instead
-            graphs, set_events = None, None
+            graphs, ev_graphs, set_events = None, None, None
             launch_mode = "eager (graph capture failed: %s)" % type(e).__name__
             torch.cuda.synchronize()
 
@@ -313,13 +323,22 @@ def run_ours(args, info):
     secs = e0.elapsed_time(e1) * 1e-3
     value_ops, t_max = D.aggregate_throughput(ops_per_step() * args.steps, secs, dev)
 
-    # ---- per-kernel durations.  (1) From inside the timed region: the event nodes of each
-    # graph hold the timestamps of its last replay, i.e. of the last n_sets timed steps.
+    # ---- per-kernel durations.  (1) Inside the step: the same K steps replayed from the graphs
+    # that carry event nodes; samples are read every n_sets steps (one per buffer set).
     in_step = None
-    if set_events is not None and args.steps >= n_sets:
+    if ev_graphs is not None:
         try:
-            in_step = {n: float(np.mean([ev[j].elapsed_time(ev[j + 1]) for ev in set_events])) * 1e-3
-                       for j, n in enumerate(names)}
+            acc = {n: [] for n in names}
+            for i in range(min(args.steps, 200)):
+                ev_graphs[i % n_sets].replay()
+                if i % n_sets == n_sets - 1:
+                    torch.cuda.synchronize()
+                    for ev in set_events:
+                        for j, n in enumerate(names):
+                            acc[n].append(ev[j].elapsed_time(ev[j + 1]) * 1e-3)
+            torch.cuda.synchronize()
+            if all(acc[n] for n in names):
+                in_step = {n: float(np.mean(acc[n])) for n in names}
         except Exception:
             in_step = None
     # (2) Each kernel alone, launched back to back over the rotating buffer sets (one graph of
@@ -348,7 +367,7 @@ def run_ours(args, info):
         e1.record()
         torch.cuda.synchronize()
         kern[n] = e0.elapsed_time(e1) * 1e-3 / (reps * n_sets)
-    timing_kind = "CUDA event nodes around the kernel inside the timed graphs (last %d steps)" % n_sets
+    timing_kind = "CUDA event nodes around the kernel inside graphs of the whole step, replayed after the timed region"
     if in_step is None:
         in_step = dict(kern)
         timing_kind = "kernel alone, launched back to back over the rotating buffer sets"

@@ -82,6 +82,8 @@ aifs_perm_kernel(const uint8_t* __restrict__ is_visual, const uint8_t* __restric
 __global__ void row_move_kernel(const uint4* __restrict__ X, uint4* __restrict__ Y, int L, int vec_per_row,
                                 int64_t ldx_vec, int64_t ldo_vec, const int32_t* __restrict__ perm,
                                 int direction) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= (int64_t)L * vec_per_row) return;
   const int i = (int)(idx / vec_per_row), c = (int)(idx % vec_per_row);
@@ -91,10 +93,74 @@ __global__ void row_move_kernel(const uint4* __restrict__ X, uint4* __restrict__
   Y[(int64_t)dst * ldo_vec + c] = __ldg(&X[(int64_t)src * ldx_vec + c]);
 }
 
+// Index build and row gather in one launch, for sequences short enough that every CTA can
+// afford to count the modality flags itself (L bytes from L2 per CTA).  A CTA owns the source
+// rows [r0, r1): it counts the first-block tokens before r0 and in the whole sequence, which
+// fixes the destination of each of its rows (stable partition), writes perm / inv_perm for
+// them and copies the rows with 16-byte vectors.
+constexpr int kFusedThreads = 256;
+constexpr int kFusedMaxL = 16384;
+
+__global__ void __launch_bounds__(kFusedThreads)
+aifs_fused_gather_kernel(const uint4* __restrict__ X, uint4* __restrict__ Y, int L, int vec_per_row,
+                         int64_t ldx_vec, int64_t ldo_vec, const uint8_t* __restrict__ is_visual,
+                         const uint8_t* __restrict__ is_pad, int32_t* __restrict__ perm,
+                         int32_t* __restrict__ inv_perm, int32_t* __restrict__ n_first_out, int rows_per_cta) {
+  __shared__ int red_before[kFusedThreads / 32], red_total[kFusedThreads / 32];
+  __shared__ int s_before, s_total;
+  __shared__ int s_dst[64];
+  pdl_launch_dependents();
+  pdl_wait();
+  const int r0 = blockIdx.x * rows_per_cta;
+  const int r1 = min(L, r0 + rows_per_cta);
+  int before = 0, total = 0;
+  for (int i = threadIdx.x; i < L; i += kFusedThreads) {
+    const int f = (is_visual[i] != 0) || (is_pad && is_pad[i] != 0);
+    total += f;
+    before += (i < r0) ? f : 0;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    before += __shfl_xor_sync(0xffffffffu, before, o);
+    total += __shfl_xor_sync(0xffffffffu, total, o);
+  }
+  if ((threadIdx.x & 31) == 0) {
+    red_before[threadIdx.x >> 5] = before;
+    red_total[threadIdx.x >> 5] = total;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int b = 0, t = 0;
+    for (int w = 0; w < kFusedThreads / 32; ++w) { b += red_before[w]; t += red_total[w]; }
+    // destinations of this CTA's rows (rows_per_cta <= 64): sequential, a handful of rows
+    int fb = b;
+    for (int i = r0; i < r1; ++i) {
+      const int f = (is_visual[i] != 0) || (is_pad && is_pad[i] != 0);
+      const int pos = f ? fb : t + (i - fb);
+      s_dst[i - r0] = pos;
+      perm[pos] = i;
+      if (inv_perm) inv_perm[i] = pos;
+      fb += f;
+    }
+    s_before = b;
+    s_total = t;
+    if (blockIdx.x == 0 && n_first_out) *n_first_out = t;
+  }
+  __syncthreads();
+  if (X == nullptr) return;
+  const int n_vec = (r1 - r0) * vec_per_row;
+  for (int v = threadIdx.x; v < n_vec; v += kFusedThreads) {
+    const int rr = v / vec_per_row, c = v - rr * vec_per_row;
+    Y[(int64_t)s_dst[rr] * ldo_vec + c] = __ldg(&X[(int64_t)(r0 + rr) * ldx_vec + c]);
+  }
+}
+
 __global__ void remap_small_kernel(const int32_t* __restrict__ perm, const int32_t* __restrict__ pos_ids,
                                    const int32_t* __restrict__ n_first, int L,
                                    int32_t* __restrict__ pos_out, int32_t* __restrict__ seg_end_out,
                                    uint8_t* __restrict__ seg_mod_out) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (pos_out && i < L) {
     const int p = perm[i];
@@ -131,13 +197,27 @@ int launch_aifs_reorder(const void* X, void* X_out, int L, int D, int64_t ldx, i
     if (direction == 0 && n_first_out) cudaMemsetAsync(n_first_out, 0, sizeof(int32_t), st);
     return cuda_status(cudaGetLastError());
   }
+  if (direction == 0 && L <= kFusedMaxL) {
+    int sms = 148, dev = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    int rows_per_cta = (L + 4 * sms - 1) / (4 * sms);
+    if (rows_per_cta > 64) rows_per_cta = 64;
+    const int ctas = (L + rows_per_cta - 1) / rows_per_cta;
+    const bool move = X && D > 0;
+    return cuda_status(launch_pdl(aifs_fused_gather_kernel, dim3(ctas), dim3(kFusedThreads), 0, st,
+                                  move ? static_cast<const uint4*>(X) : nullptr, static_cast<uint4*>(X_out), L,
+                                  move ? D / 8 : 0, ldx / 8, ldo / 8, is_visual, is_pad, perm, inv_perm,
+                                  n_first_out, rows_per_cta));
+  }
   if (direction == 0)
     aifs_perm_kernel<<<1, kScanThreads, 0, st>>>(is_visual, is_pad, L, perm, inv_perm, n_first_out);
   if (X && D > 0) {
     const int vec = D / 8;
     const int64_t n = (int64_t)L * vec;
-    row_move_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(
-        static_cast<const uint4*>(X), static_cast<uint4*>(X_out), L, vec, ldx / 8, ldo / 8, perm, direction);
+    if (launch_pdl(row_move_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), 0, st,
+                   static_cast<const uint4*>(X), static_cast<uint4*>(X_out), L, vec, ldx / 8, ldo / 8,
+                   static_cast<const int32_t*>(perm), direction) != cudaSuccess)
+      return MQ_ERR_CUDA;
   }
   return cuda_status(cudaGetLastError());
 }
@@ -146,7 +226,9 @@ int launch_mask_remap(const int32_t* perm, const int32_t* pos_ids, const uint8_t
                       const int32_t* n_first, int L, int32_t* pos_out, int32_t* seg_end_out,
                       uint8_t* seg_mod_out, uint8_t* dense, cudaStream_t st) {
   const int blocks = L > 0 ? (L + 255) / 256 : 1;
-  remap_small_kernel<<<blocks, 256, 0, st>>>(perm, pos_ids, n_first, L, pos_out, seg_end_out, seg_mod_out);
+  if (launch_pdl(remap_small_kernel, dim3(blocks), dim3(256), 0, st, perm, pos_ids, n_first, L, pos_out, seg_end_out,
+                 seg_mod_out) != cudaSuccess)
+    return MQ_ERR_CUDA;
   if (dense && L > 0) {
     dim3 grid((L + 255) / 256, L);
     dense_mask_kernel<<<grid, 256, 0, st>>>(perm, is_pad, L, dense);

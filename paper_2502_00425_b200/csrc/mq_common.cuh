@@ -46,6 +46,34 @@ __device__ __forceinline__ int thread_row_modality(const SegTable& seg, int t) {
 
 inline int cuda_status(cudaError_t e) { return e == cudaSuccess ? MQ_OK : MQ_ERR_CUDA; }
 
+// ---- programmatic dependent launch ----------------------------------------------------
+// The hot-path kernels follow one another on a stream, each a few tens of microseconds long,
+// so the launch latency between them is a visible share of a step.  They are launched with
+// programmatic stream serialization: a kernel lets its successor start launching at once
+// (pdl_launch_dependents at its top), and every such kernel executes pdl_wait -- which returns
+// once the preceding kernel has completed and its writes are visible -- after its private
+// set-up and BEFORE it reads or writes any global memory other than its parameters.  Because
+// every kernel of the chain waits before it exits, completion is transitive along the chain.
+// On a launch without the attribute both instructions do nothing.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                              Args&&... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // host launchers implemented in the .cu files -----------------------------------------
 int launch_fwht_quant(const void* X, int T, int K, int64_t ldx, SegTable seg, float s_vis,
                       float s_txt, int rot_block, int8_t* Q, int64_t ldq, float* rotated_out,

@@ -40,6 +40,8 @@ fwht_quant_kernel(const uint16_t* __restrict__ X, int T, int K, int64_t ldx, Seg
                   float* __restrict__ rotated_out, uint32_t* __restrict__ amax_state,
                   int tiles_per_row, long long n_warp_tiles) {
   constexpr int TPB = 1 << LOG_TPB;
+  pdl_launch_dependents();
+  pdl_wait();
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
   const long long wt = (long long)blockIdx.x * kWarpsPerCta + warp;
@@ -169,9 +171,8 @@ int dispatch(const void* X, int T, int K, int64_t ldx, SegTable seg, float inv_v
   const float c_n = rot_block ? (float)(1.0 / sqrt((double)rot_block)) : 1.0f;
   const uint16_t* x = static_cast<const uint16_t*>(X);
 #define MQ_LAUNCH(LOG_TPB, ROT)                                                              \
-  fwht_quant_kernel<LOG_TPB, ROT, MODE><<<grid, block, 0, st>>>(                             \
-      x, T, K, ldx, seg, inv_vis, inv_txt, c_n, Q, ldq, rotated_out, amax_state, tiles_per_row, \
-      n_warp_tiles)
+  launch_pdl(fwht_quant_kernel<LOG_TPB, ROT, MODE>, grid, block, 0, st, x, T, K, ldx, seg, inv_vis, inv_txt, c_n, \
+             Q, ldq, rotated_out, amax_state, tiles_per_row, n_warp_tiles)
   switch (rot_block) {
     case 0: MQ_LAUNCH(2, false); break;
     case 32: MQ_LAUNCH(0, true); break;

@@ -400,10 +400,14 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const KernelParam
     tmem_alloc(&sh->tmem_base, 512);
     tmem_relinquish();
   }
+  pdl_launch_dependents();
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&sh->tmem_base);
+  // everything above touched only this CTA's shared and tensor memory; from here on the
+  // roles read what the preceding kernel wrote (the int8 codes, the segment table)
+  pdl_wait();
 
   // Ring positions are kept as (stage, phase) pairs that advance by increment-and-wrap: the
   // issuing roles are latency-bound, and an integer division per K block would cost more
@@ -593,6 +597,8 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const KernelParam
 __global__ void splitk_finalize_kernel(const int32_t* __restrict__ acc, int T, int N, SegTable seg, float s_vis,
                                        float s_txt, const float* __restrict__ s_w, const float* __restrict__ bias,
                                        void* Y, int64_t ldy, int y_is_f32, int32_t* __restrict__ acc_out) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= (int64_t)T * N) return;
   const int t = (int)(idx / N), n = (int)(idx % N);
@@ -743,14 +749,14 @@ int launch_gemm(const GemmArgs& a, cudaStream_t st) {
     if (!a.splitk_acc) return MQ_ERR_WORKSPACE;
     if (cudaMemsetAsync(a.splitk_acc, 0, (size_t)a.T * a.N * sizeof(int32_t), st) != cudaSuccess) return MQ_ERR_CUDA;
   }
-  w4a8_gemm_kernel<<<pl.grid, (8 + 4 * pl.groups) * 32, pl.smem, st>>>(tmap, p);
-  if (cudaGetLastError() != cudaSuccess) return MQ_ERR_CUDA;
+  if (launch_pdl(w4a8_gemm_kernel, dim3(pl.grid), dim3((8 + 4 * pl.groups) * 32), pl.smem, st, tmap, p) != cudaSuccess)
+    return MQ_ERR_CUDA;
   if (pl.ksplit > 1) {
     const int64_t n = (int64_t)a.T * a.N;
-    splitk_finalize_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(a.splitk_acc, a.T, a.N, a.seg, a.s_vis,
-                                                                       a.s_txt, a.s_w, a.bias, a.Y, a.ldy,
-                                                                       a.y_is_f32, a.acc_out);
-    if (cudaGetLastError() != cudaSuccess) return MQ_ERR_CUDA;
+    if (launch_pdl(splitk_finalize_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), 0, st,
+                   static_cast<const int32_t*>(a.splitk_acc), a.T, a.N, a.seg, a.s_vis, a.s_txt, a.s_w, a.bias, a.Y,
+                   a.ldy, a.y_is_f32, a.acc_out) != cudaSuccess)
+      return MQ_ERR_CUDA;
   }
   return MQ_OK;
 }

@@ -144,7 +144,7 @@ def _aifs_case(is_vis, is_pad, D, seed):
     return perm, n_first, pad_d, p_ref
 
 
-@pytest.mark.parametrize("name", ["c3", "c4", "tiny", "all_text", "all_visual", "long"])
+@pytest.mark.parametrize("name", ["c3", "c4", "tiny", "all_text", "all_visual", "long", "very_long"])
 def test_aifs_reorder_and_remap(name):
     rng = np.random.default_rng(7)
     is_pad = None
@@ -159,6 +159,8 @@ def test_aifs_reorder_and_remap(name):
         is_vis, D = np.zeros(37, np.uint8), 8
     elif name == "all_visual":
         is_vis, D = np.ones(1025, np.uint8), 8
+    elif name == "very_long":      # beyond the single-launch limit: separate index-scan and row-move kernels
+        is_vis, D = (rng.random(20000) < 0.4).astype(np.uint8), 8
     else:
         is_vis, D = (rng.random(5000) < 0.7).astype(np.uint8), 16
         is_pad = np.zeros(5000, np.uint8)
@@ -180,6 +182,18 @@ def test_aifs_reorder_and_remap(name):
     pos_iota = torch.empty(L, dtype=torch.int32, device=DEV)
     B.mq_attn_mask_remap(perm, None, pad_d, n_first, pos_iota)
     assert np.array_equal(pos_iota.cpu().numpy(), p_ref)
+
+
+def test_aifs_index_only_call():
+    is_vis = synth.config3_sequence()
+    L = len(is_vis)
+    perm = torch.full((L,), -1, dtype=torch.int32, device=DEV)
+    inv = torch.full((L,), -1, dtype=torch.int32, device=DEV)
+    n_first = torch.full((1,), -1, dtype=torch.int32, device=DEV)
+    B.mq_aifs_reorder(None, None, torch.from_numpy(is_vis).to(DEV), None, perm, inv, n_first, direction=0, L=L)
+    p_ref = O.aifs_perm(is_vis)
+    assert np.array_equal(perm.cpu().numpy(), p_ref) and n_first.item() == int(is_vis.sum())
+    assert np.array_equal(inv.cpu().numpy(), O.inverse_perm(p_ref))
 
 
 # ----------------------------------------------------------------------------- the linear
