@@ -107,7 +107,6 @@ aifs_fused_gather_kernel(const uint4* __restrict__ X, uint4* __restrict__ Y, int
                          const uint8_t* __restrict__ is_pad, int32_t* __restrict__ perm,
                          int32_t* __restrict__ inv_perm, int32_t* __restrict__ n_first_out, int rows_per_cta) {
   __shared__ int red_before[kFusedThreads / 32], red_total[kFusedThreads / 32];
-  __shared__ int s_before, s_total;
   __shared__ int s_dst[64];
   pdl_launch_dependents();
   pdl_wait();
@@ -142,8 +141,6 @@ aifs_fused_gather_kernel(const uint4* __restrict__ X, uint4* __restrict__ Y, int
       if (inv_perm) inv_perm[i] = pos;
       fb += f;
     }
-    s_before = b;
-    s_total = t;
     if (blockIdx.x == 0 && n_first_out) *n_first_out = t;
   }
   __syncthreads();

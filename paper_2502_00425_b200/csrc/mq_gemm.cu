@@ -289,13 +289,15 @@ enum : int { kEpiSplitK = 1, kEpiAcc = 2, kEpiF32 = 4, kEpiBias = 8, kEpiGeneric
 template <int MODE>
 __device__ __forceinline__ void epilogue_chunk(const KernelParams& p, const uint32_t (&v)[16], int t_first,
                                                int nvalid, int n, bool n_ok, float sw, float bs,
-                                               const float* stok, __nv_bfloat16* stage) {
+                                               const float* stok, __nv_bfloat16* stage, int ks) {
   if (!(MODE & kEpiStaged) && !n_ok) return;
   if (MODE & kEpiSplitK) {
-    int32_t* dst = p.splitk_acc + (size_t)t_first * p.N + n;
+    // every K split owns a slice [T,N] of the scratch: plain stores, summed by the finalize
+    // kernel -- no atomics and nothing to clear beforehand
+    int32_t* dst = p.splitk_acc + (size_t)ks * p.T * p.N + (size_t)t_first * p.N + n;
 #pragma unroll
     for (int j = 0; j < 16; ++j)
-      if (j < nvalid) atomicAdd(dst + (size_t)j * p.N, ((int)v[j]) >> 4);  // the MMA saw 16 * q_w
+      if (j < nvalid) dst[(size_t)j * p.N] = ((int)v[j]) >> 4;  // the MMA saw 16 * q_w
     return;
   }
   if (MODE & kEpiGeneric) {
@@ -353,19 +355,21 @@ __device__ __forceinline__ void epilogue_chunk(const KernelParams& p, const uint
 // load of the next 16 columns is in flight while the current 16 are converted and stored.
 template <int MODE>
 __device__ __forceinline__ void epilogue_tile(const KernelParams& p, uint32_t d_tmem, int t0, int n, bool n_ok,
-                                              float sw, float bs, const float* stok, __nv_bfloat16* stage) {
+                                              float sw, float bs, const float* stok, __nv_bfloat16* stage, int ks) {
   const int ncols = min(p.TN, p.T - t0);  // valid token columns of this tile (> 0)
   uint32_t va[16], vb[16];
   tmem_ld_x16(d_tmem, va);
   for (int cc = 0; cc < ncols; cc += 32) {
+    __syncwarp();  // tcgen05.ld / wait::ld are warp-collective; lanes may have left the chunk code early
     tmem_wait_ld();
     const bool has_b = cc + 16 < ncols;
     if (has_b) tmem_ld_x16(d_tmem + cc + 16, vb);
-    epilogue_chunk<MODE>(p, va, t0 + cc, min(16, ncols - cc), n, n_ok, sw, bs, stok + cc, stage);
+    epilogue_chunk<MODE>(p, va, t0 + cc, min(16, ncols - cc), n, n_ok, sw, bs, stok + cc, stage, ks);
     if (has_b) {
+      __syncwarp();
       tmem_wait_ld();
       if (cc + 32 < ncols) tmem_ld_x16(d_tmem + cc + 32, va);
-      epilogue_chunk<MODE>(p, vb, t0 + cc + 16, min(16, ncols - cc - 16), n, n_ok, sw, bs, stok + cc + 16, stage);
+      epilogue_chunk<MODE>(p, vb, t0 + cc + 16, min(16, ncols - cc - 16), n, n_ok, sw, bs, stok + cc + 16, stage, ks);
     }
   }
 }
@@ -573,10 +577,10 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const KernelParam
       const float bs = (n_ok && p.bias) ? p.bias[n] : 0.0f;
       const uint32_t d_tmem = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(d * p.d_stride);
       switch (epi_mode) {
-#define MQ_EPI_CASE(M) case M: epilogue_tile<M>(p, d_tmem, t0, n, n_ok, sw, bs, stok, stage); break;
+#define MQ_EPI_CASE(M) case M: epilogue_tile<M>(p, d_tmem, t0, n, n_ok, sw, bs, stok, stage, c.ks); break;
         MQ_EPI_CASE(kEpiStaged) MQ_EPI_CASE(kEpiStaged | kEpiBias) MQ_EPI_CASE(kEpiSplitK)
 #undef MQ_EPI_CASE
-        default: epilogue_tile<kEpiGeneric>(p, d_tmem, t0, n, n_ok, sw, bs, stok, stage); break;
+        default: epilogue_tile<kEpiGeneric>(p, d_tmem, t0, n, n_ok, sw, bs, stok, stage, c.ks); break;
       }
       tc_fence_before();
       __syncwarp();
@@ -594,7 +598,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const KernelParam
 }
 
 // Split-K finalize: exact int32 partial sums -> dequantized output.
-__global__ void splitk_finalize_kernel(const int32_t* __restrict__ acc, int T, int N, SegTable seg, float s_vis,
+__global__ void splitk_finalize_kernel(const int32_t* __restrict__ acc, int ksplit, int T, int N, SegTable seg, float s_vis,
                                        float s_txt, const float* __restrict__ s_w, const float* __restrict__ bias,
                                        void* Y, int64_t ldy, int y_is_f32, int32_t* __restrict__ acc_out) {
   pdl_launch_dependents();
@@ -602,7 +606,8 @@ __global__ void splitk_finalize_kernel(const int32_t* __restrict__ acc, int T, i
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= (int64_t)T * N) return;
   const int t = (int)(idx / N), n = (int)(idx % N);
-  const int a = acc[idx];
+  int a = 0;
+  for (int ks = 0; ks < ksplit; ++ks) a += acc[(size_t)ks * T * N + idx];  // one slice per K split
   if (acc_out) acc_out[idx] = a;
   const float st = thread_row_modality(seg, t) == MQ_VISUAL ? s_vis : s_txt;
   float y = __fmul_rn((float)a, __fmul_rn(st, s_w[n]));
@@ -703,7 +708,7 @@ Plan make_plan(int T, int K, int N) {
 size_t gemm_splitk_bytes(int T, int K, int N) {
   if (T <= 0 || K <= 0 || N <= 0) return 0;
   const Plan pl = make_plan(T, K, N);
-  return pl.ksplit > 1 ? (size_t)T * N * sizeof(int32_t) : 0;
+  return pl.ksplit > 1 ? (size_t)pl.ksplit * T * N * sizeof(int32_t) : 0;  // one [T,N] slice per K split
 }
 
 int launch_gemm(const GemmArgs& a, cudaStream_t st) {
@@ -745,16 +750,13 @@ int launch_gemm(const GemmArgs& a, cudaStream_t st) {
   p.s_w = a.s_w; p.bias = a.bias; p.Y = a.Y; p.ldy = a.ldy; p.y_is_f32 = a.y_is_f32;
   p.acc_out = a.acc_out; p.splitk_acc = a.splitk_acc; p.status = a.status;
 
-  if (pl.ksplit > 1) {
-    if (!a.splitk_acc) return MQ_ERR_WORKSPACE;
-    if (cudaMemsetAsync(a.splitk_acc, 0, (size_t)a.T * a.N * sizeof(int32_t), st) != cudaSuccess) return MQ_ERR_CUDA;
-  }
+  if (pl.ksplit > 1 && !a.splitk_acc) return MQ_ERR_WORKSPACE;
   if (launch_pdl(w4a8_gemm_kernel, dim3(pl.grid), dim3((8 + 4 * pl.groups) * 32), pl.smem, st, tmap, p) != cudaSuccess)
     return MQ_ERR_CUDA;
   if (pl.ksplit > 1) {
     const int64_t n = (int64_t)a.T * a.N;
     if (launch_pdl(splitk_finalize_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), 0, st,
-                   static_cast<const int32_t*>(a.splitk_acc), a.T, a.N, a.seg, a.s_vis, a.s_txt, a.s_w, a.bias, a.Y,
+                   static_cast<const int32_t*>(a.splitk_acc), pl.ksplit, a.T, a.N, a.seg, a.s_vis, a.s_txt, a.s_w, a.bias, a.Y,
                    a.ldy, a.y_is_f32, a.acc_out) != cudaSuccess)
       return MQ_ERR_CUDA;
   }

@@ -43,7 +43,8 @@ def test_size_queries(lib):
     big = B.mq_workspace_bytes(1088, 18944, 3584, 128)
     assert big >= 256 + 1088 * 18944
     assert B.mq_workspace_bytes(1088, 18944, 3584, 0, B.MQ_FLAG_X_IS_INT8) == 256
-    assert B.mq_workspace_bytes(8, 4096, 256) >= 256 + 8 * 4096 + 8 * 256 * 4   # split-K scratch
+    assert B.mq_workspace_bytes(8, 4096, 256) >= 256 + 8 * 4096 + 2 * 8 * 256 * 4   # split-K slices
+    assert (B.mq_workspace_bytes(8, 4096, 256) - 256 - 8 * 4096) % (8 * 256 * 4) == 0  # whole [T,N] slices
     assert B.mq_workspace_bytes(8, 100, 256) == 0                   # K % 32
     assert B.mq_workspace_bytes(8, 128, 100) == 0                   # N % 16
     assert B.mq_workspace_bytes(8, 128, 128, 48) == 0               # rotation block not a power of two

@@ -251,8 +251,12 @@ def test_config1_full():
     (70, 0, 256, 128, 64),         # no text rows
     (1, 0, 32, 16, 32),            # the smallest legal problem
     (250, 263, 160, 144, 32),      # K not a multiple of the K block; two token tiles
-    (3, 5, 4096, 256, 128),        # small T: split-K path
-    (100, 28, 4096, 512, 1024),    # T = 128, split-K
+    (3, 5, 4096, 256, 128),        # T = 8: streaming variant (tokens as MMA rows), split-K slices
+    (5, 8, 160, 144, 32),          # T = 13: streaming, ragged K block, one half-empty 256-channel tile
+    (0, 27, 1152, 272, 128),       # T = 27: streaming, two channel tiles, the second one ragged
+    (20, 13, 2048, 128, 0),        # T = 33: streaming, tokens in two epilogue warps
+    (100, 28, 4096, 512, 1024),    # T = 128: the largest streaming problem, split-K
+    (100, 29, 1024, 384, 0),       # T = 129: smallest problem of the channel-row variant
 ])
 def test_linear_edge_shapes(T_vis, T_txt, K, N, rot):
     c = synth.small_linear(100 + K + N, T_vis, T_txt, K, N, rot, calib_vis=24, calib_txt=8)

@@ -40,9 +40,10 @@ def test_noalloc_matches_workspace_entry_point_twice_in_a_row():
     from paper_2502_00425_b200 import synth
     from gpu_util import DEV, bf16_to_dev, dev_segments, gpu_calibrate, gpu_linear, gpu_pack
 
-    # two different decode-shaped problems, both on the split-K path, so that the second call
-    # finds the first call's codes and partial sums in the shared array
-    cases = [synth.small_linear(41, 3, 29, 4096, 512, 128, calib_vis=8, calib_txt=24),
+    # two different small problems -- the first large enough to take the split-K path of the
+    # GEMM, the second GEMV-shaped -- so that each call finds the other's codes and partial sums
+    # in the shared array
+    cases = [synth.small_linear(41, 3, 45, 4096, 512, 128, calib_vis=8, calib_txt=24),
              synth.small_linear(42, 0, 8, 2048, 256, 0, calib_vis=8, calib_txt=8)]
     bias = [np.random.default_rng(5).standard_normal(512).astype(np.float32), None]
     prepared = []
