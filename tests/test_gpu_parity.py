@@ -330,6 +330,56 @@ def test_config2_full_size_sampled():
     assert int(acc.abs().max()) <= 128 * 8 * c.K
 
 
+def _check_full_size_sampled(c, tile_rows, n_sample=24):
+    """Full-size linear in the launch configuration a layer would use; the oracle checks every
+    column of a deterministic row sample: rows around every segment boundary, first / last rows
+    of token tiles, the massive-activation rows and an even spread."""
+    s_v, s_t = gpu_calibrate(c.x_calib, c.seg_calib, c.rot_block)
+    o_v, o_t = O.calibrate_static_scales(c.x_calib, c.seg_calib.seg_end, c.seg_calib.seg_mod, c.rot_block)
+    assert (s_v, s_t) == (o_v, o_t)
+    packed, s_w, layout = gpu_pack(c.w)
+    qw, sw_ref = O.quantize_weight_int4(c.w)
+    assert np.array_equal(s_w.cpu().numpy(), sw_ref)
+    rows = {0, c.T - 1} | set(c.meta["massive_rows"])
+    for e in np.asarray(c.seg.seg_end)[:-1].tolist():
+        rows |= {e - 1, e}
+    for t0 in range(0, c.T, tile_rows):
+        rows |= {t0, min(c.T - 1, t0 + tile_rows - 1)}
+    rows = sorted(rows)
+    if len(rows) > n_sample:                     # thin the tile-edge rows, keep boundaries and massive rows
+        keep = set(c.meta["massive_rows"]) | {0, c.T - 1}
+        for e in np.asarray(c.seg.seg_end)[:-1].tolist():
+            keep |= {e - 1, e}
+        rest = [r for r in rows if r not in keep]
+        step = max(1, len(rest) // max(1, n_sample - len(keep)))
+        rows = sorted(keep | set(rest[::step]))
+    rows = np.array(rows)
+    yb, acc, st = gpu_linear(c, s_v, s_t, layout, s_w, None, torch.bfloat16)
+    assert st == (B.MQ_OK, 0)
+    sub_mod = c.seg.row_modality(c.T)[rows]
+    ref = O.linear_w4a8_msq(c.x[rows], *_seg_arrays(sub_mod), s_v, s_t, c.rot_block, qw, sw_ref)
+    assert np.array_equal(acc.cpu().numpy()[rows], ref["acc"])
+    assert np.array_equal(bf16_from_dev(yb)[rows], ref["y_bf16"])
+    nz = np.abs(ref["y64"]) > 0
+    assert _rel(bf16_from_dev(yb)[rows], ref["y64"])[nz].max() <= 1e-2
+    assert int(acc.abs().max()) <= 128 * 8 * c.K
+
+
+@pytest.mark.parametrize("which", ["k_proj", "down_proj"])
+def test_config3_linears_full_size_sampled(which):
+    """Qwen2-7B-shaped block at T = 3360 in AIFS order (3072 visual, 288 text): the narrow
+    k-projection (N = 512) and the rotated down-projection (K = 18944)."""
+    _check_full_size_sampled(synth.config3_linear(which), tile_rows=192)
+
+
+@pytest.mark.parametrize("which", ["q_proj", "down_proj"])
+def test_config4_linears_full_size_sampled(which):
+    """8B-shaped block, batch of 4 sequences flattened to 9728 rows with 8 segments."""
+    c = synth.config4_linear(which)
+    assert c.seg.n_seg == 8
+    _check_full_size_sampled(c, tile_rows=192)
+
+
 def _seg_arrays(row_mod):
     s = synth.segments_from_row_modality(row_mod)
     return s.seg_end, s.seg_mod
