@@ -214,6 +214,62 @@ def decode_sweep(torch, B, dev, peaks, n_sets=6, reps=20):
     return out
 
 
+# ------------------------------------------------------------------------------------------ layer linear suites
+def linear_suite(torch, B, dev, name, T, n_vis_per_seq, n_txt_per_seq, batch, shape, reps=5):
+    """The seven W4A8 MSQ linears of one decoder block (configs 3 and 4, linear-suite mode): every
+    linear gets its own synthetic activations in AIFS order and runs rotation (down_proj only) +
+    quantizer + GEMM through mq_w4a8_msq_linear.  Weight layouts and scales are random valid bytes
+    (timing only; parity of these shapes is covered by the tests).  Reports microseconds per
+    linear and TOPS over the seven."""
+    g = torch.Generator(device="cpu").manual_seed(11)
+    seg_end, seg_mod, e = [], [], 0
+    for _ in range(batch):
+        e += n_vis_per_seq
+        seg_end.append(e)
+        seg_mod.append(1)
+        e += n_txt_per_seq
+        seg_end.append(e)
+        seg_mod.append(0)
+    assert e == T
+    seg = B.Segments.from_host(seg_end, seg_mod, dev)
+    items, total_ops = [], 0.0
+    for lname, K, N, rot in shape.linears():
+        x = (torch.randn((T, K), generator=g, dtype=torch.float32) * 2).to(torch.bfloat16).to(dev)
+        lay = torch.randint(0, 256, (B.mq_w4_layout_bytes(N, K),), dtype=torch.uint8, generator=g).to(dev)
+        s_w = (torch.rand(N, generator=g) * 0.01 + 0.001).to(dev)
+        y = torch.empty((T, N), dtype=torch.bfloat16, device=dev)
+        ws = B.new_workspace(T, K, N, rot)
+        items.append((lname, K, N, rot, x, lay, s_w, y, ws))
+        total_ops += 2.0 * T * K * N
+
+    def run(it):
+        lname, K, N, rot, x, lay, s_w, y, ws = it
+        B.mq_w4a8_msq_linear(x, seg, 0.5, 0.05, lay, s_w, y, ws, N, rot_block=rot)
+
+    per = {}
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for it in items:
+        run(it)
+    torch.cuda.synchronize()
+    for it in items:
+        e0.record()
+        for _ in range(reps):
+            run(it)
+        e1.record()
+        torch.cuda.synchronize()
+        per[it[0]] = e0.elapsed_time(e1) * 1e3 / reps
+    e0.record()
+    for _ in range(reps):
+        for it in items:
+            run(it)
+    e1.record()
+    torch.cuda.synchronize()
+    sec = e0.elapsed_time(e1) * 1e-3 / reps
+    ok = all(B.mq_last_device_status(it[8])[0] == 0 for it in items)
+    return {"workload": name, "T": T, "us_per_linear": per, "us_all_seven": sec * 1e6, "tops": total_ops / sec / 1e12,
+            "tokens_per_s": T / sec, "status_ok": ok}
+
+
 # ------------------------------------------------------------------------------------------ our arm
 class BufferSet:
     """One independent copy of every device buffer a step touches."""
@@ -454,10 +510,16 @@ def run_ours(args, info):
     e2e_ops, _ = D.aggregate_throughput(ops_per_step() * e2e_steps, e0.elapsed_time(e1) * 1e-3, dev)
 
     # ---- decode-shaped sweep (rank 0, N = 1 only): the HBM-bound regime of the same path
-    decode = None
+    decode, suites = None, None
     if info.is_main and info.world == 1 and not args.no_decode:
         del graphs, ev_graphs
         decode = decode_sweep(torch, B, dev, peaks)
+        del sets
+        torch.cuda.empty_cache()
+        suites = [linear_suite(torch, B, dev, "config3: Qwen2-7B-shaped block, 3 x (1024 visual + 96 text) in AIFS order",
+                               3360, 3072, 288, 1, synth.QWEN2_7B),
+                  linear_suite(torch, B, dev, "config4: 8B-shaped block, 4 sequences x (2304 visual + 128 text)",
+                               9728, 2304, 128, 4, synth.LLAMA_8B)]
 
     # ---- CPU baseline: the oracle on this host (rank 0, N = 1 only)
     cpu = None
@@ -506,6 +568,7 @@ def run_ours(args, info):
                                "peak_gbs": peaks["hbm_gbs"],
                                "frac": quant_bytes / kern["fwht_quant"] / 1e9 / peaks["hbm_gbs"]},
             "decode": decode,
+            "layer_linear_suites": suites,
             "device_status": list(status),
             "cpu_baseline": cpu,
         }
