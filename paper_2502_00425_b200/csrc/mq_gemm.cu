@@ -103,6 +103,12 @@ __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
+// Arrive that cannot be issued before `dep` is available in a register.  Used to release a
+// shared-memory stage after reading it: `dep` is computed from every load of the stage, so the
+// loads have returned their data (not merely been issued) when the producer is told to overwrite it.
+__device__ __forceinline__ void mbar_arrive_after(uint64_t* bar, uint32_t dep) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];  // after %1" ::"r"(smem_u32(bar)), "r"(dep) : "memory");
+}
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
                : "memory");
@@ -493,7 +499,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const KernelParam
         if (++s == p.stages) { s = 0; ph ^= 1u; }
         if (++a == p.num_a) a = 0;
       }
-      if (ok && lane == 0) tc_commit(&sh->d_full[d]);
+      if (ok && elect_one()) tc_commit(&sh->d_full[d]);  // the thread that issued the MMAs
       if (++d == p.num_d) { d = 0; ph_d ^= 1u; d_wrapped = true; }
     }
     if (!ok && lane == 0) {  // let every MMA already issued finish before tensor memory is freed
@@ -529,8 +535,9 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const KernelParam
           regs[jj * 8 + 2 * i + 1] = ww[i] & 0xF0F0F0F0u;      // codes k0+4..k0+7, each x16
         }
       }
+      const uint32_t dep = __shfl_xor_sync(0xffffffffu, regs[1] ^ regs[9] ^ regs[17] ^ regs[25], 1);  // all lanes' loads done
       __syncwarp();
-      if (lane == 0) mbar_arrive(&sh->w_empty[sw]);
+      if (lane == 0) mbar_arrive_after(&sh->w_empty[sw], dep);
       if (it >= p.num_a) {
         // stage and parity of block it - num_a, derived from those of block it
         const int fs = s >= p.num_a ? s - p.num_a : s - p.num_a + p.stages;
@@ -596,6 +603,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const KernelParam
     tmem_dealloc(tmem_base, 512);
   }
 }
+
 
 // Split-K finalize: exact int32 partial sums -> dequantized output.
 __global__ void splitk_finalize_kernel(const int32_t* __restrict__ acc, int ksplit, int T, int N, SegTable seg, float s_vis,

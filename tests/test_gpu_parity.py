@@ -284,6 +284,30 @@ def test_linear_clipping_variant():
     _check_linear(c, clipping_expected=True)
 
 
+@pytest.mark.parametrize("T,K,N", [(128, 13696, 512), (8, 4096, 1024), (600, 2048, 640)])
+def test_repeated_launches_give_identical_accumulators(T, K, N):
+    """A race in the producer / expander / MMA pipeline shows as a result that changes from launch
+    to launch.  Exact integer reference (int8 x int4 codes, float64 matmul is exact here), the
+    first launch cold, then back-to-back launches without host synchronisation in between."""
+    g = torch.Generator().manual_seed(T + K + N)
+    x = torch.randint(-127, 128, (T, K), dtype=torch.int8, generator=g)
+    qw = torch.randint(-8, 8, (N, K), dtype=torch.int8, generator=g)
+    packed = ((qw[:, 0::2] & 15) | ((qw[:, 1::2] & 15) << 4)).to(torch.uint8)
+    layout = torch.empty(B.mq_w4_layout_bytes(N, K), dtype=torch.uint8, device=DEV)
+    B.mq_repack_w4(packed.to(DEV), N, K, layout)
+    ref = (x.to(torch.float64) @ qw.to(torch.float64).T).to(torch.int32)
+    xd, ones = x.to(DEV), torch.ones(N, device=DEV)
+    seg = B.Segments.from_host([T // 2, T], [1, 0], DEV)
+    ws = B.new_workspace(T, K, N, 0, B.MQ_FLAG_X_IS_INT8)
+    y = torch.empty((T, N), dtype=torch.float32, device=DEV)
+    accs = [torch.full((T, N), -7, dtype=torch.int32, device=DEV) for _ in range(12)]
+    for a in accs:
+        B.mq_w4a8_msq_linear(xd, seg, 1.0, 1.0, layout, ones, y, ws, N, acc_out=a)
+    assert B.mq_last_device_status(ws) == (B.MQ_OK, 0)
+    for a in accs:
+        assert torch.equal(a.cpu(), ref)
+
+
 def test_zero_rows_is_a_noop():
     c = synth.small_linear(3, 4, 4, 128, 128, 0, calib_vis=4, calib_txt=4)
     packed, s_w, layout = gpu_pack(c.w)
