@@ -161,54 +161,63 @@ def run_reference(args, info):
 
 # ------------------------------------------------------------------------------------------ decode sweep
 def decode_sweep(torch, B, dev, peaks, n_sets=6, reps=20):
-    """Config-5-shaped decode steps: the three linears of a 4096 / 13696 MLP (gate, up: 4096 -> 13696;
+    """Config-5-shaped decode steps: the linears of a 4096 / 13696 SwiGLU MLP (gate, up: 4096 -> 13696;
     down: 13696 -> 4096 behind the 128-block rotation) at T = 1, 8, 32, 128 text tokens.  Each step
-    runs rotation + quantizer + W4A8 product for the three linears; n_sets independent copies of the
-    int4 weights (84 MB each, more than four L2 sizes in all) are cycled so that the weights come from
-    HBM.  Reported per T: microseconds per MLP pass and packed-weight bytes per second."""
+    runs rotation + quantizer + W4A8 product per linear; n_sets independent copies of the int4
+    weights (84 MB each, more than four L2 sizes in all) are cycled so that the weights come from
+    HBM.  Two arrangements are timed: the three linears as three calls, and gate and up stored as
+    one [27392, 4096] weight (they share their input), i.e. two calls.  Reported per T:
+    microseconds per MLP pass and packed-weight bytes per second."""
     hidden, mlp = 4096, 13696
-    shapes = [("gate_proj", hidden, mlp, 0), ("up_proj", hidden, mlp, 0), ("down_proj", mlp, hidden, 128)]
+    arrangements = {"three_calls": [(hidden, mlp, 0), (hidden, mlp, 0), (mlp, hidden, 128)],
+                    "gate_up_fused": [(hidden, 2 * mlp, 0), (mlp, hidden, 128)]}
     g = torch.Generator(device="cpu").manual_seed(4)
-    weights = []
-    for _ in range(n_sets):
-        per_set = []
-        for _, K, N, _ in shapes:
-            lay = torch.randint(0, 256, (B.mq_w4_layout_bytes(N, K),), dtype=torch.uint8, generator=g).to(dev)
-            per_set.append((lay, (torch.rand(N, generator=g) * 0.01 + 0.001).to(dev)))
-        weights.append(per_set)
-    w_bytes = sum(N * K // 2 for _, K, N, _ in shapes)
+    w_bytes = 3 * hidden * mlp // 2
     out = {}
     seg = B.Segments.from_host([], [], dev)  # no visual rows: every token uses the text scale
-    for T in (1, 8, 32, 128):
-        xs = [(torch.randn((T, K), generator=g) * 2).to(torch.bfloat16).to(dev) for _, K, _, _ in shapes]
-        ys = [torch.empty((T, N), dtype=torch.bfloat16, device=dev) for _, _, N, _ in shapes]
-        wss = [B.new_workspace(T, K, N, rot) for _, K, N, rot in shapes]
+    for name, shapes in arrangements.items():
+        weights = []
+        for _ in range(n_sets):
+            per_set = []
+            for K, N, _ in shapes:
+                lay = torch.randint(0, 256, (B.mq_w4_layout_bytes(N, K),), dtype=torch.uint8, generator=g).to(dev)
+                per_set.append((lay, (torch.rand(N, generator=g) * 0.01 + 0.001).to(dev)))
+            weights.append(per_set)
+        res = {}
+        for T in (1, 8, 32, 128):
+            xs = [(torch.randn((T, K), generator=g) * 2).to(torch.bfloat16).to(dev) for K, _, _ in shapes]
+            ys = [torch.empty((T, N), dtype=torch.bfloat16, device=dev) for _, N, _ in shapes]
+            wss = [B.new_workspace(T, K, N, rot) for K, N, rot in shapes]
 
-        def mlp_pass(i):
-            for j, (_, K, N, rot) in enumerate(shapes):
-                lay, s_w = weights[i % n_sets][j]
-                B.mq_w4a8_msq_linear(xs[j], seg, 1.0, 0.05, lay, s_w, ys[j], wss[j], N, rot_block=rot)
+            def mlp_pass(i):
+                for j, (K, N, rot) in enumerate(shapes):
+                    lay, s_w = weights[i % n_sets][j]
+                    B.mq_w4a8_msq_linear(xs[j], seg, 1.0, 0.05, lay, s_w, ys[j], wss[j], N, rot_block=rot)
 
-        for i in range(n_sets):
-            mlp_pass(i)
-        torch.cuda.synchronize()
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph):
             for i in range(n_sets):
                 mlp_pass(i)
-        graph.replay()
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for _ in range(reps):
+            torch.cuda.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                for i in range(n_sets):
+                    mlp_pass(i)
             graph.replay()
-        e1.record()
-        torch.cuda.synchronize()
-        sec = e0.elapsed_time(e1) * 1e-3 / (reps * n_sets)
-        status = [B.mq_last_device_status(w)[0] for w in wss]
-        gbs = w_bytes / sec / 1e9
-        out["T%d" % T] = {"us_per_mlp": sec * 1e6, "weight_gbs": gbs, "frac_of_measured_hbm": gbs / peaks["hbm_gbs"],
-                          "tokens_per_s": T / sec, "status_ok": all(v == 0 for v in status)}
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(reps):
+                graph.replay()
+            e1.record()
+            torch.cuda.synchronize()
+            sec = e0.elapsed_time(e1) * 1e-3 / (reps * n_sets)
+            status = [B.mq_last_device_status(w)[0] for w in wss]
+            gbs = w_bytes / sec / 1e9
+            res["T%d" % T] = {"us_per_mlp": sec * 1e6, "weight_gbs": gbs, "frac_of_measured_hbm": gbs / peaks["hbm_gbs"],
+                              "tokens_per_s": T / sec, "status_ok": all(v == 0 for v in status)}
+            del graph
+        out[name] = res
+        del weights
+        torch.cuda.empty_cache()
     out["workload"] = ("config5: 4096/13696 MLP (gate, up, down with 128-block rotation), %d weight sets of %.0f MB "
                        "cycled" % (n_sets, w_bytes / 1e6))
     return out
@@ -316,8 +325,12 @@ def run_ours(args, info):
     B.load(build_if_missing=True)
     torch.cuda.set_device(info.local_rank)
     dev = torch.device("cuda", info.local_rank)
-    D.init(info)
     peaks = read_peaks()
+    if args.decode_only:
+        if info.is_main:
+            print(json.dumps({"decode": decode_sweep(torch, B, dev, peaks, n_sets=4, reps=2)}), flush=True)
+        return
+    D.init(info)
 
     case = synth.config2(seed=D.batch_seed(1, info.rank))
     is_vis = synth.interleaved_modality(SPANS)
@@ -586,6 +599,8 @@ def main():
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-decode", action="store_true")
+    ap.add_argument("--decode-only", action="store_true",
+                    help="run only the decode-shaped sweep and print it (used for profiler captures)")
     args = ap.parse_args()
     if args.steps is None:
         args.steps = 5 if args.impl == "reference" else 2000
