@@ -421,6 +421,56 @@ def rotate_weight_input_dim(w, n: int) -> np.ndarray:
     return rotate_dense(np.asarray(w, dtype=np.float64), n)
 
 
+# ----------------------------------------------------------------------------- RMS (Sec. 3.2)
+def rms_detect(w, n: int) -> np.ndarray:
+    """Eq. 9 per output channel and rotation block: the first row of the rotated weight,
+    sqrt(n) * mean(w) over the block's n input channels (the equation between Eq. 7 and Eq. 9),
+    exceeds the block's largest original weight -- a channel-mean outlier created by the
+    online transform.  w is the UNROTATED weight [N, K]; returns bool [N, K / n].
+    (The paper's W is [in, out]; its column j is our row.)"""
+    w = np.asarray(w, dtype=np.float64)
+    N, K = w.shape
+    assert K % n == 0
+    blocks = w.reshape(N, K // n, n)
+    return np.sqrt(float(n)) * blocks.mean(axis=2) > blocks.max(axis=2)
+
+
+def rms_split(w_rot, n: int):
+    """Rotation Magnitude Suppression, steps 1 and 2 (Sec. 3.2): the first input channel of
+    every rotation block of the ROTATED weight [N, K] is split off (it is handled by a
+    separate GEMV) and zeroed in the main matrix so that it is not counted twice.
+    Returns (w_main [N, K], w_side [N, K / n])."""
+    w_rot = np.asarray(w_rot)
+    w_main = w_rot.copy()
+    w_side = w_rot[:, ::n].copy()
+    w_main[:, ::n] = 0
+    return w_main, w_side
+
+
+def linear_w4a8_msq_rms(x, seg_end, seg_mod, s_vis, s_txt, rot_block, qw_main, s_w_main, qw_side, s_w_side,
+                        bias=None):
+    """The down-projection with RMS (Sec. 3.2, step 3: add the GEMV's partial output back):
+      y = Q(x~) . Q(HW with the split rows zeroed)^T  +  Q(x~[:, first channel of each block]) . Q(split rows)^T.
+    Both terms use the same int8 activation codes; each weight part has its own per-channel
+    int4 scale.  float32 twin: each term is float(acc) * (s_a * s_w) with the scale product
+    formed first, the terms are added, then the bias."""
+    x = np.asarray(x, dtype=np.float32)
+    T = x.shape[0]
+    r = fwht_blocks(x, rot_block, np.float32)
+    s_rows = row_scales(T, seg_end, seg_mod, s_vis, s_txt)
+    qx = quantize_act_int8(r, s_rows)
+    acc_main = int_gemm(qx, qw_main)
+    acc_side = int_gemm(qx[:, ::rot_block], qw_side)
+    y64 = dequant(acc_main, s_rows, s_w_main, None, np.float64) + dequant(acc_side, s_rows, s_w_side, None, np.float64)
+    y32 = (dequant(acc_main, s_rows, s_w_main, None, np.float32)
+           + dequant(acc_side, s_rows, s_w_side, None, np.float32)).astype(np.float32)
+    if bias is not None:
+        y64 = y64 + np.asarray(bias, dtype=np.float64).reshape(1, -1)
+        y32 = (y32 + np.asarray(bias, dtype=np.float32).reshape(1, -1)).astype(np.float32)
+    return {"qx": qx, "s_rows": s_rows, "acc_main": acc_main, "acc_side": acc_side, "y64": y64, "y32": y32,
+            "y_bf16": bf16_rne(y32)}
+
+
 def quantize_act_int8_dynamic(r):
     """Per-token dynamic A8 (the baseline MSQ replaces, Sec. 1): every row gets
     its own Eq. 2 scale from its own abs-max."""

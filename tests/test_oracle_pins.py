@@ -394,6 +394,59 @@ def test_rms_split_cost_fixture():
         assert (2 * 1 * N) * denom == 2 * K * N
 
 
+def test_rms_detect_is_the_first_row_criterion():
+    # Eq. 9 on hand-made rows (n = 4): sqrt(4) * mean > max  <=>  2 * mean > max
+    w = np.array([[1.0, 1.0, 1.0, 1.0,   3.0, -1.0, -1.0, -1.0],     # block 0: 2*1 > 1 yes; block 1: 2*0 > 3 no
+                  [0.5, 0.6, 0.7, 0.4,  -1.0, -1.0, -1.0, -1.0]])    # block 0: 1.1 > 0.7 yes; block 1: -2 > -1 no
+    assert O.rms_detect(w, 4).tolist() == [[True, False], [True, False]]
+    # the criterion compares the first row of the rotated weight with the original maximum (Sec. 3.2)
+    rng = np.random.default_rng(3)
+    w = rng.standard_normal((6, 64)) + rng.standard_normal((6, 1)) * 0.5
+    first_row = O.rotate_dense(w, 32)[:, ::32]
+    assert np.array_equal(O.rms_detect(w, 32), first_row > w.reshape(6, 2, 32).max(axis=2))
+
+
+def test_rms_split_is_exact_without_quantization_and_costs_one_row_per_block():
+    rng = np.random.default_rng(5)
+    n, K, N, T = 32, 128, 10, 7
+    w_rot = O.rotate_dense(rng.standard_normal((N, K)) + 0.8, n)
+    x_rot = rng.standard_normal((T, K))
+    w_main, w_side = O.rms_split(w_rot, n)
+    assert np.all(w_main[:, ::n] == 0) and np.array_equal(w_side, w_rot[:, ::n])
+    # step 3: the GEMV term added back restores the unsplit product exactly (up to float64 rounding)
+    assert np.allclose(x_rot @ w_main.T + x_rot[:, ::n] @ w_side.T, x_rot @ w_rot.T, rtol=0, atol=1e-12)
+    # the split takes the large first-row entries out of the main matrix ...
+    assert np.abs(w_main).max() < np.abs(w_rot).max()
+    # ... at a cost of one input row per rotation block: 1/n of the GEMM (1/K when one block spans K)
+    assert w_side.size * n == w_rot.size
+    assert O.rms_split(w_rot, K)[1].shape == (N, 1)
+
+
+def test_rms_linear_reduces_to_the_plain_linear_when_the_split_rows_are_zero():
+    rng = np.random.default_rng(9)
+    T, K, N, n = 9, 64, 6, 32
+    x = O.bf16_rne(rng.standard_normal((T, K)).astype(np.float32))
+    w = rng.standard_normal((N, K)).astype(np.float32) * 0.02
+    w[:, ::n] = 0                                            # nothing to split off
+    seg_end, seg_mod = np.array([5, 9]), np.array([1, 0])
+    qw, s_w = O.quantize_weight_int4(w)
+    plain = O.linear_w4a8_msq(x, seg_end, seg_mod, 0.05, 0.03, n, qw, s_w)
+    rms = O.linear_w4a8_msq_rms(x, seg_end, seg_mod, 0.05, 0.03, n, qw, s_w, np.zeros((N, K // n), np.int8),
+                                np.ones(N, np.float32))
+    assert np.array_equal(rms["acc_main"], plain["acc"]) and not rms["acc_side"].any()
+    assert np.array_equal(rms["y32"], plain["y32"])
+    # and with a real split the quantized result stays within the quantization error bound of the exact product
+    w2 = (rng.standard_normal((N, K)) * 0.02 + 0.05).astype(np.float32)
+    w2_rot = O.rotate_dense(w2, n).astype(np.float32)
+    w_main, w_side = O.rms_split(w2_rot, n)
+    qm, sm = O.quantize_weight_int4(w_main)
+    qs, ss = O.quantize_weight_int4(w_side)
+    out = O.linear_w4a8_msq_rms(x, seg_end, seg_mod, 0.05, 0.03, n, qm, sm, qs, ss)
+    exact = O.rotate_dense(x, n) @ w2_rot.astype(np.float64).T
+    plain2 = O.linear_w4a8_msq(x, seg_end, seg_mod, 0.05, 0.03, n, *O.quantize_weight_int4(w2_rot))
+    assert np.abs(out["y64"] - exact).mean() < np.abs(plain2["y64"] - exact).mean()   # the point of RMS
+
+
 def test_dynamic_quantizer_uses_row_absmax():
     r = np.array([[1.0, -2.0], [0.5, 0.25]], np.float32)
     q, s = O.quantize_act_int8_dynamic(r)
