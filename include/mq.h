@@ -235,6 +235,68 @@ int mq_w4a8_msq_linear_noalloc(const mq_linear_desc* d, const void* X, int64_t l
                                const void* W_layout, const float* s_w, const float* bias, void* Y,
                                int64_t ldy, int32_t* acc_out, int32_t* status_out, void* stream);
 
+/* ---- Rotation Magnitude Suppression (Sec. 3.2, Eq. 9) ------------------------------------
+ *
+ * Applies to a linear whose input is rotated online by I (x) H_n (the down-projection).  The
+ * rotation concentrates a non-zero mean of each n-wide block of a weight row into the
+ * block's FIRST rotated input channel (value sqrt(n) * mean, the relation stated between
+ * Eq. 7 and Eq. 9).  Eq. 9 marks an (output channel, block) pair when that value exceeds the
+ * block's largest original weight.  The remedy: split the first input channel of every
+ * block off the rotated weight, zero it in the main matrix, run it as a separate small
+ * product on the same activation codes, and add that product back.
+ */
+
+/* Row length (in codes = bytes) of the split part q_side: K / rot_block rounded up to a
+ * multiple of 4.  Returns 0 for an invalid (K, rot_block). */
+size_t mq_rms_side_ld(int32_t K, int32_t rot_block);
+
+/*
+ * Eq. 9 on the UNROTATED weight W (device fp32 [N, K], row = output channel, leading
+ * dimension ldw): flag[n, b] = sqrt(n_rot) * mean(W[n, b*n_rot .. +n_rot-1]) >
+ * max(W[n, b*n_rot .. +n_rot-1]), evaluated in double precision.
+ *   flags      device uint8 [N, K / rot_block], may be NULL
+ *   count_out  device int32[1], number of flagged pairs, may be NULL (not both NULL)
+ * rot_block: a power of two in [32, 1024] that divides K.  Offline, asynchronous on `stream`.
+ */
+int mq_rms_detect(const float* W, int32_t N, int32_t K, int64_t ldw, int32_t rot_block, uint8_t* flags,
+                  int32_t* count_out, void* stream);
+
+/*
+ * mq_pack_w4 for a weight that gets the remedy.  W_rot is the ROTATED weight (device fp32
+ * [N, K]).  Input channels k with k % rot_block == 0 form the split part:
+ *   main part  all other channels; per-channel scale s_w[n] = max|.| / 7 over them; codes
+ *              written to `packed` (canonical, may be NULL) and `gemm_layout` (may be NULL)
+ *              exactly as mq_pack_w4 does, with code 0 at the split channels;
+ *   split part q_side: device int8 [N, mq_rms_side_ld(K, rot_block)], 16-byte aligned, one
+ *              int4 code per byte (value in [-8, 7]), code b of row n = channel b*rot_block,
+ *              padding codes 0; s_w_side[n] = max|.| / 7 over the split channels (1 if all 0).
+ * All outputs are caller-owned device memory.  Offline, asynchronous on `stream`.
+ */
+int mq_pack_w4_rms(const float* W_rot, int32_t N, int32_t K, int64_t ldw, int32_t rot_block, uint8_t* packed,
+                   float* s_w, void* gemm_layout, int8_t* q_side, float* s_w_side, void* stream);
+
+/* Workspace of mq_w4a8_msq_linear_rms: that of mq_w4a8_msq_linear plus an fp32 [T, N]
+ * buffer for the main part's output.  0 for a descriptor the call would reject. */
+size_t mq_rms_workspace_bytes(const mq_linear_desc* d);
+
+/*
+ * The W4A8 MSQ linear with the remedy (step 3: add the split part's product back):
+ *   qx       = Q_int8(FWHT(X))                      as in mq_w4a8_msq_linear
+ *   acc_main = qx . q_main^T                         (split channels are 0 in q_main)
+ *   acc_side = qx[:, 0::rot_block] . q_side^T
+ *   y32      = fl(acc_main * fl(s_a * s_w[n])) + fl(acc_side * fl(s_a * s_w_side[n])) (+ bias[n])
+ *   Y        = bf16(y32), or y32 with MQ_FLAG_Y_IS_F32
+ * d->rot_block must be non-zero and MQ_FLAG_X_IS_INT8 is not accepted (MQ_ERR_INVALID_ARG).
+ * W_layout / s_w / q_side / s_w_side come from mq_pack_w4_rms.  acc_out and acc_side_out
+ * (device int32 [T, N], either may be NULL) receive the two integer accumulators.  ws:
+ * device, 256-byte aligned, at least mq_rms_workspace_bytes(d) (else MQ_ERR_WORKSPACE).
+ * Everything else as mq_w4a8_msq_linear.  Asynchronous on `stream`.
+ */
+int mq_w4a8_msq_linear_rms(const mq_linear_desc* d, const void* X, int64_t ldx, const mq_segments* seg, float s_vis,
+                           float s_txt, const void* W_layout, const float* s_w, const int8_t* q_side,
+                           const float* s_w_side, const float* bias, void* Y, int64_t ldy, int32_t* acc_out,
+                           int32_t* acc_side_out, void* ws, size_t ws_bytes, void* stream);
+
 /* Waits for `stream`, then returns the status word kernels left in the workspace
  * (MQ_OK or MQ_ERR_TIMEOUT) and, if site_out != NULL (host), where the wait gave up. */
 int mq_last_device_status(void* ws, void* stream, int32_t* site_out);

@@ -77,6 +77,12 @@ def load(build_if_missing: bool = False):
         "mq_fwht_quant_i8": (C.c_int, [vp, i32, i32, i64, segp, f32, f32, i32, vp, i64, vp, vp]),
         "mq_w4a8_msq_linear": (C.c_int, [descp, vp, i64, segp, f32, f32, vp, vp, vp, vp, i64, vp, vp, sz, vp]),
         "mq_w4a8_msq_linear_noalloc": (C.c_int, [descp, vp, i64, segp, f32, f32, vp, vp, vp, vp, i64, vp, vp, vp]),
+        "mq_rms_side_ld": (sz, [i32, i32]),
+        "mq_rms_detect": (C.c_int, [vp, i32, i32, i64, i32, vp, vp, vp]),
+        "mq_pack_w4_rms": (C.c_int, [vp, i32, i32, i64, i32, vp, vp, vp, vp, vp, vp]),
+        "mq_rms_workspace_bytes": (sz, [descp]),
+        "mq_w4a8_msq_linear_rms": (C.c_int, [descp, vp, i64, segp, f32, f32, vp, vp, vp, vp, vp, vp, i64, vp, vp,
+                                             vp, sz, vp]),
         "mq_last_device_status": (C.c_int, [vp, vp, C.POINTER(C.c_int32)]),
         "mq_reset_device_status": (C.c_int, [vp, vp]),
     }
@@ -91,7 +97,8 @@ def load(build_if_missing: bool = False):
 EXPORTED = ["mq_version", "mq_status_string", "mq_workspace_bytes", "mq_w4_layout_bytes",
             "mq_calibrate_static_scales", "mq_pack_w4", "mq_repack_w4", "mq_unpack_w4", "mq_aifs_reorder",
             "mq_attn_mask_remap", "mq_fwht_quant_i8", "mq_w4a8_msq_linear", "mq_w4a8_msq_linear_noalloc", "mq_last_device_status",
-            "mq_reset_device_status"]
+            "mq_reset_device_status", "mq_rms_side_ld", "mq_rms_detect", "mq_pack_w4_rms", "mq_rms_workspace_bytes",
+            "mq_w4a8_msq_linear_rms"]
 
 
 def status_string(status: int) -> str:
@@ -250,6 +257,57 @@ def mq_w4a8_msq_linear_noalloc(x, seg: Segments, s_vis, s_txt, w_layout, s_w, y,
                                              _ptr(w_layout), _ptr(s_w), _ptr(bias), _ptr(y), _ld(y),
                                              _ptr(acc_out), _ptr(status_out), _stream()),
            "mq_w4a8_msq_linear_noalloc")
+
+
+def mq_rms_side_ld(K, rot_block) -> int:
+    return int(load().mq_rms_side_ld(K, rot_block))
+
+
+def mq_rms_detect(w, rot_block, flags=None, count_out=None):
+    """Eq. 9 on the unrotated weight [N, K]: flags uint8 [N, K / rot_block], count int32[1]."""
+    assert w.dtype == torch.float32
+    N, K = w.shape
+    _check(load().mq_rms_detect(_ptr(w), N, K, _ld(w), rot_block, _ptr(flags), _ptr(count_out), _stream()),
+           "mq_rms_detect")
+
+
+def mq_pack_w4_rms(w_rot, rot_block, s_w, q_side, s_w_side, packed=None, gemm_layout=None):
+    assert w_rot.dtype == torch.float32 and q_side.dtype == torch.int8
+    N, K = w_rot.shape
+    _check(load().mq_pack_w4_rms(_ptr(w_rot), N, K, _ld(w_rot), rot_block, _ptr(packed), _ptr(s_w),
+                                 _ptr(gemm_layout), _ptr(q_side), _ptr(s_w_side), _stream()), "mq_pack_w4_rms")
+
+
+def mq_rms_workspace_bytes(T, K, N, rot_block, flags=0) -> int:
+    d = mq_linear_desc(T, K, N, rot_block, 0, flags)
+    return int(load().mq_rms_workspace_bytes(C.byref(d)))
+
+
+def new_rms_workspace(T, K, N, rot_block, flags=0, device="cuda") -> torch.Tensor:
+    n = mq_rms_workspace_bytes(T, K, N, rot_block, flags)
+    if n == 0:
+        raise MqError(MQ_ERR_INVALID_ARG, "mq_rms_workspace_bytes")
+    ws = torch.empty(n, dtype=torch.uint8, device=device)
+    _check(load().mq_reset_device_status(_ptr(ws), _stream()), "mq_reset_device_status")
+    return ws
+
+
+def mq_w4a8_msq_linear_rms(x, seg: Segments, s_vis, s_txt, w_layout, s_w, q_side, s_w_side, y, N, rot_block, ws,
+                           bias=None, acc_out=None, acc_side_out=None):
+    """The rotated linear with rotation magnitude suppression (Sec. 3.2): main GEMM plus the
+    split first-channel-of-each-block product, added before the bias."""
+    assert x.dtype == torch.bfloat16
+    T, K = x.shape
+    flags = 0
+    if y.dtype == torch.float32:
+        flags |= MQ_FLAG_Y_IS_F32
+    else:
+        assert y.dtype == torch.bfloat16
+    d = mq_linear_desc(T, K, N, rot_block, 0, flags)
+    _check(load().mq_w4a8_msq_linear_rms(C.byref(d), _ptr(x), _ld(x), seg.ref(), float(s_vis), float(s_txt),
+                                         _ptr(w_layout), _ptr(s_w), _ptr(q_side), _ptr(s_w_side), _ptr(bias),
+                                         _ptr(y), _ld(y), _ptr(acc_out), _ptr(acc_side_out), _ptr(ws), ws.numel(),
+                                         _stream()), "mq_w4a8_msq_linear_rms")
 
 
 def mq_last_device_status(ws):

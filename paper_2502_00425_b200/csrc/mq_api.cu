@@ -220,6 +220,75 @@ int mq_w4a8_msq_linear(const mq_linear_desc* d, const void* X, int64_t ldx, cons
   return launch_gemm(a, cs);
 }
 
+// ---- rotation magnitude suppression (Sec. 3.2) -------------------------------------------
+namespace {
+int check_rms_shape(int32_t N, int32_t K, int32_t rot_block) {
+  if (N <= 0 || K <= 0 || K % 32 || N % 16) return MQ_ERR_INVALID_ARG;
+  if (rot_block == 0) return MQ_ERR_INVALID_ARG;  // the split columns are defined by the rotation block
+  return check_rot(rot_block, K);
+}
+size_t rms_side_ld(int32_t K, int32_t rot_block) { return align_up((size_t)(K / rot_block), 4); }
+}  // namespace
+
+size_t mq_rms_side_ld(int32_t K, int32_t rot_block) {
+  if (K <= 0 || check_rot(rot_block, K) != MQ_OK || rot_block == 0) return 0;
+  return rms_side_ld(K, rot_block);
+}
+
+int mq_rms_detect(const float* W, int32_t N, int32_t K, int64_t ldw, int32_t rot_block, uint8_t* flags,
+                  int32_t* count_out, void* stream) {
+  int rc = check_rms_shape(N, K, rot_block);
+  if (rc != MQ_OK) return rc;
+  if (!W || ldw < K || (!flags && !count_out)) return MQ_ERR_INVALID_ARG;
+  return launch_rms_detect(W, N, K, ldw, rot_block, flags, count_out, static_cast<cudaStream_t>(stream));
+}
+
+int mq_pack_w4_rms(const float* W_rot, int32_t N, int32_t K, int64_t ldw, int32_t rot_block, uint8_t* packed,
+                   float* s_w, void* gemm_layout, int8_t* q_side, float* s_w_side, void* stream) {
+  int rc = check_rms_shape(N, K, rot_block);
+  if (rc != MQ_OK) return rc;
+  if (!W_rot || !s_w || !q_side || !s_w_side || ldw < K) return MQ_ERR_INVALID_ARG;
+  if (gemm_layout && !aligned(gemm_layout, 128)) return MQ_ERR_ALIGNMENT;
+  if (!aligned16(q_side)) return MQ_ERR_ALIGNMENT;
+  return launch_rms_pack(W_rot, N, K, ldw, rot_block, packed, s_w, gemm_layout, q_side,
+                         (int)rms_side_ld(K, rot_block), s_w_side, static_cast<cudaStream_t>(stream));
+}
+
+size_t mq_rms_workspace_bytes(const mq_linear_desc* d) {
+  if (check_desc(d) != MQ_OK || d->rot_block == 0 || (d->flags & MQ_FLAG_X_IS_INT8)) return 0;
+  return ws_layout(d).total + align_up((size_t)d->T * d->N * sizeof(float), 256);
+}
+
+int mq_w4a8_msq_linear_rms(const mq_linear_desc* d, const void* X, int64_t ldx, const mq_segments* seg, float s_vis,
+                           float s_txt, const void* W_layout, const float* s_w, const int8_t* q_side,
+                           const float* s_w_side, const float* bias, void* Y, int64_t ldy, int32_t* acc_out,
+                           int32_t* acc_side_out, void* ws, size_t ws_bytes, void* stream) {
+  int rc = check_desc(d);
+  if (rc != MQ_OK) return rc;
+  if (d->rot_block == 0 || (d->flags & MQ_FLAG_X_IS_INT8)) return MQ_ERR_INVALID_ARG;
+  if (!q_side || !s_w_side || !Y || ldy < d->N) return MQ_ERR_INVALID_ARG;
+  if (!aligned16(q_side)) return MQ_ERR_ALIGNMENT;
+  SegTable st;
+  if ((rc = check_seg(seg, &st)) != MQ_OK) return rc;
+  if (!ws) return MQ_ERR_WORKSPACE;
+  if (!aligned(ws, 256)) return MQ_ERR_ALIGNMENT;
+  const WsLayout wl = ws_layout(d);
+  const size_t y_bytes = align_up((size_t)d->T * d->N * sizeof(float), 256);
+  if (ws_bytes < wl.total + y_bytes) return MQ_ERR_WORKSPACE;
+  uint8_t* wsb = static_cast<uint8_t*>(ws);
+  float* y_main = reinterpret_cast<float*>(wsb + wl.total);
+  // main part: the ordinary linear, fp32 output, no bias (the bias is added once, after the sum)
+  mq_linear_desc dm = *d;
+  dm.flags |= MQ_FLAG_Y_IS_F32;
+  rc = mq_w4a8_msq_linear(&dm, X, ldx, seg, s_vis, s_txt, W_layout, s_w, nullptr, y_main, d->N, acc_out, ws,
+                          wl.total, stream);
+  if (rc != MQ_OK) return rc;
+  const int8_t* qx = reinterpret_cast<const int8_t*>(wsb + wl.qx_off);
+  return launch_rms_combine(y_main, qx, d->K, d->T, d->K, d->N, d->rot_block, st, s_vis, s_txt, q_side,
+                            (int)rms_side_ld(d->K, d->rot_block), s_w_side, bias, Y, ldy,
+                            (d->flags & MQ_FLAG_Y_IS_F32) ? 1 : 0, acc_side_out, static_cast<cudaStream_t>(stream));
+}
+
 int mq_last_device_status(void* ws, void* stream, int32_t* site_out) {
   if (!ws) return MQ_ERR_INVALID_ARG;
   int32_t host[2] = {0, 0};

@@ -89,6 +89,8 @@ int launch_calibrate(const void* X, int T, int K, int64_t ldx, SegTable seg, int
                      cudaStream_t st);
 int launch_pack_w4(const float* W, int N, int K, int64_t ldw, uint8_t* packed, float* s_w,
                    void* layout, cudaStream_t st);
+int launch_pack_codes(const float* W, int N, int K, int64_t ldw, const float* s_w, uint8_t* packed,
+                      void* layout, int skip, cudaStream_t st);
 int launch_repack_w4(const uint8_t* packed, int N, int K, void* layout, cudaStream_t st);
 int launch_unpack_w4(const uint8_t* packed, const void* layout, int N, int K, int8_t* q,
                      int64_t ldq, cudaStream_t st);
@@ -98,6 +100,15 @@ int launch_aifs_reorder(const void* X, void* X_out, int L, int D, int64_t ldx, i
 int launch_mask_remap(const int32_t* perm, const int32_t* pos_ids, const uint8_t* is_pad,
                       const int32_t* n_first, int L, int32_t* pos_out, int32_t* seg_end_out,
                       uint8_t* seg_mod_out, uint8_t* dense, cudaStream_t st);
+
+// rotation magnitude suppression (mq_rms.cu)
+int launch_rms_detect(const float* W, int N, int K, int64_t ldw, int nb, uint8_t* flags, int32_t* count,
+                      cudaStream_t st);
+int launch_rms_pack(const float* W, int N, int K, int64_t ldw, int nb, uint8_t* packed, float* s_w, void* layout,
+                    int8_t* q_side, int side_ld, float* s_w_side, cudaStream_t st);
+int launch_rms_combine(const float* y_main, const int8_t* qx, int64_t ldq, int T, int K, int N, int nb, SegTable seg,
+                       float s_vis, float s_txt, const int8_t* q_side, int side_ld, const float* s_w_side,
+                       const float* bias, void* Y, int64_t ldy, int y_is_f32, int32_t* acc_side_out, cudaStream_t st);
 
 struct GemmArgs {
   int T, K, N;

@@ -41,15 +41,21 @@ __global__ void row_scale_kernel(const float* __restrict__ W, int N, int K, int6
   }
 }
 
+// skip != 0: input channels k with k % skip == 0 are written as code 0 (they were split off the
+// main matrix, see mq_rms.cu).
+__device__ __forceinline__ int rtn_int4_masked(const float* W, int64_t idx, int k, float s, int skip) {
+  return (skip && k % skip == 0) ? 0 : rtn_int4(W[idx], s);
+}
+
 __global__ void pack_canonical_kernel(const float* __restrict__ W, int N, int K, int64_t ldw,
-                                      const float* __restrict__ s_w, uint8_t* __restrict__ packed) {
+                                      const float* __restrict__ s_w, uint8_t* __restrict__ packed, int skip) {
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   const int half = K / 2;
   if (idx >= (int64_t)N * half) return;
   const int n = (int)(idx / half), j = (int)(idx % half);
   const float s = s_w[n];
-  const int q0 = rtn_int4(W[(int64_t)n * ldw + 2 * j], s);
-  const int q1 = rtn_int4(W[(int64_t)n * ldw + 2 * j + 1], s);
+  const int q0 = rtn_int4_masked(W, (int64_t)n * ldw + 2 * j, 2 * j, s, skip);
+  const int q1 = rtn_int4_masked(W, (int64_t)n * ldw + 2 * j + 1, 2 * j + 1, s, skip);
   packed[idx] = (uint8_t)((q0 & 15) | ((q1 & 15) << 4));
 }
 
@@ -71,7 +77,7 @@ __device__ __forceinline__ WordCoord layout_word_coord(int64_t word, int KB) {
 
 __global__ void pack_layout_kernel(const float* __restrict__ W, int N, int K, int64_t ldw,
                                    const float* __restrict__ s_w, uint32_t* __restrict__ layout,
-                                   int KB, int64_t n_words) {
+                                   int KB, int64_t n_words, int skip) {
   const int64_t word = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (word >= n_words) return;
   const WordCoord c = layout_word_coord(word, KB);
@@ -81,8 +87,8 @@ __global__ void pack_layout_kernel(const float* __restrict__ W, int N, int K, in
 #pragma unroll
     for (int b = 0; b < 4; ++b) {
       const int klo = c.k0 + b, khi = c.k0 + 4 + b;
-      const int qlo = klo < K ? rtn_int4(W[(int64_t)c.n * ldw + klo], s) : 0;
-      const int qhi = khi < K ? rtn_int4(W[(int64_t)c.n * ldw + khi], s) : 0;
+      const int qlo = klo < K ? rtn_int4_masked(W, (int64_t)c.n * ldw + klo, klo, s, skip) : 0;
+      const int qhi = khi < K ? rtn_int4_masked(W, (int64_t)c.n * ldw + khi, khi, s, skip) : 0;
       out |= (uint32_t)((qlo & 15) | ((qhi & 15) << 4)) << (8 * b);
     }
   }
@@ -135,20 +141,27 @@ inline int64_t layout_words(int N, int K) {
 
 }  // namespace
 
-int launch_pack_w4(const float* W, int N, int K, int64_t ldw, uint8_t* packed, float* s_w,
-                   void* layout, cudaStream_t st) {
+// Codes and layouts from scales that are already in s_w (skip: see pack_canonical_kernel).
+int launch_pack_codes(const float* W, int N, int K, int64_t ldw, const float* s_w, uint8_t* packed,
+                      void* layout, int skip, cudaStream_t st) {
   if (N == 0 || K == 0) return MQ_OK;
-  row_scale_kernel<<<N, 256, 0, st>>>(W, N, K, ldw, s_w);
   if (packed) {
     const int64_t n = (int64_t)N * (K / 2);
-    pack_canonical_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(W, N, K, ldw, s_w, packed);
+    pack_canonical_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(W, N, K, ldw, s_w, packed, skip);
   }
   if (layout) {
     const int64_t nw = layout_words(N, K);
     pack_layout_kernel<<<(unsigned)((nw + 255) / 256), 256, 0, st>>>(
-        W, N, K, ldw, s_w, static_cast<uint32_t*>(layout), (K + MQ_W_TILE_K - 1) / MQ_W_TILE_K, nw);
+        W, N, K, ldw, s_w, static_cast<uint32_t*>(layout), (K + MQ_W_TILE_K - 1) / MQ_W_TILE_K, nw, skip);
   }
   return cuda_status(cudaGetLastError());
+}
+
+int launch_pack_w4(const float* W, int N, int K, int64_t ldw, uint8_t* packed, float* s_w,
+                   void* layout, cudaStream_t st) {
+  if (N == 0 || K == 0) return MQ_OK;
+  row_scale_kernel<<<N, 256, 0, st>>>(W, N, K, ldw, s_w);
+  return launch_pack_codes(W, N, K, ldw, s_w, packed, layout, 0, st);
 }
 
 int launch_repack_w4(const uint8_t* packed, int N, int K, void* layout, cudaStream_t st) {

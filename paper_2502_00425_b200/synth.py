@@ -260,3 +260,17 @@ def embedding_rows(seed: int, L: int, D: int, is_visual: np.ndarray) -> np.ndarr
     x = rng.standard_normal((L, D)).astype(np.float32)
     x[np.asarray(is_visual) == VISUAL] *= np.float32(4.0)
     return round_to_bf16(x)
+
+
+def mean_shifted_weight(seed: int, N: int, K: int, block: int, shifted_fraction: float = 0.3,
+                        sigma: float = 0.02, shift: float = 0.01) -> np.ndarray:
+    """float32 [N, K] weight in which a fraction of the (output channel, block) pairs has a
+    non-zero mean over the block's input channels -- the structure that an online block
+    rotation turns into one large entry per block (the case a down-projection shows)."""
+    rng = np.random.default_rng(seed)
+    w = (rng.standard_normal((N, K)) * sigma).astype(np.float32)
+    nb = K // block
+    shifted = rng.random((N, nb)) < shifted_fraction
+    sign = np.where(rng.random((N, nb)) < 0.5, -1.0, 1.0)
+    offs = (shifted * sign * shift * (0.5 + rng.random((N, nb)))).astype(np.float32)
+    return (w.reshape(N, nb, block) + offs[:, :, None]).reshape(N, K).astype(np.float32)
