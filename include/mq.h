@@ -246,8 +246,8 @@ int mq_w4a8_msq_linear_noalloc(const mq_linear_desc* d, const void* X, int64_t l
  * product on the same activation codes, and add that product back.
  */
 
-/* Row length (in codes = bytes) of the split part q_side: K / rot_block rounded up to a
- * multiple of 4.  Returns 0 for an invalid (K, rot_block). */
+/* Row length (in codes) of the split part: K / rot_block rounded up to a multiple of 32, the
+ * K granularity of the GEMM that multiplies it.  Returns 0 for an invalid (K, rot_block). */
 size_t mq_rms_side_ld(int32_t K, int32_t rot_block);
 
 /*
@@ -267,16 +267,21 @@ int mq_rms_detect(const float* W, int32_t N, int32_t K, int64_t ldw, int32_t rot
  *   main part  all other channels; per-channel scale s_w[n] = max|.| / 7 over them; codes
  *              written to `packed` (canonical, may be NULL) and `gemm_layout` (may be NULL)
  *              exactly as mq_pack_w4 does, with code 0 at the split channels;
- *   split part q_side: device int8 [N, mq_rms_side_ld(K, rot_block)], 16-byte aligned, one
- *              int4 code per byte (value in [-8, 7]), code b of row n = channel b*rot_block,
- *              padding codes 0; s_w_side[n] = max|.| / 7 over the split channels (1 if all 0).
+ *   split part q_side: device int8 [N, mq_rms_side_ld(K, rot_block)], one int4 code per byte
+ *              (value in [-8, 7]), code b of row n = channel b*rot_block, padding codes 0;
+ *              s_w_side[n] = max|.| / 7 over the split channels (1 if all 0);
+ *              side_layout (may be NULL): the same codes in the GEMM weight layout, 128-byte
+ *              aligned, mq_w4_layout_bytes(N, mq_rms_side_ld(K, rot_block)) bytes -- this is
+ *              what mq_w4a8_msq_linear_rms reads; q_side is the inspectable form.
  * All outputs are caller-owned device memory.  Offline, asynchronous on `stream`.
  */
 int mq_pack_w4_rms(const float* W_rot, int32_t N, int32_t K, int64_t ldw, int32_t rot_block, uint8_t* packed,
-                   float* s_w, void* gemm_layout, int8_t* q_side, float* s_w_side, void* stream);
+                   float* s_w, void* gemm_layout, int8_t* q_side, float* s_w_side, void* side_layout,
+                   void* stream);
 
-/* Workspace of mq_w4a8_msq_linear_rms: that of mq_w4a8_msq_linear plus an fp32 [T, N]
- * buffer for the main part's output.  0 for a descriptor the call would reject. */
+/* Workspace of mq_w4a8_msq_linear_rms: that of mq_w4a8_msq_linear plus the gathered split
+ * activation codes [T, mq_rms_side_ld] (and, for small T, one more [T, N] int32 slice).
+ * 0 for a descriptor the call would reject. */
 size_t mq_rms_workspace_bytes(const mq_linear_desc* d);
 
 /*
@@ -287,13 +292,16 @@ size_t mq_rms_workspace_bytes(const mq_linear_desc* d);
  *   y32      = fl(acc_main * fl(s_a * s_w[n])) + fl(acc_side * fl(s_a * s_w_side[n])) (+ bias[n])
  *   Y        = bf16(y32), or y32 with MQ_FLAG_Y_IS_F32
  * d->rot_block must be non-zero and MQ_FLAG_X_IS_INT8 is not accepted (MQ_ERR_INVALID_ARG).
- * W_layout / s_w / q_side / s_w_side come from mq_pack_w4_rms.  acc_out and acc_side_out
+ * One GEMM launch computes both products: every output tile first accumulates the split
+ * product (K = mq_rms_side_ld codes) into a second tensor-memory accumulator, then the main
+ * product, and the epilogue combines them; there is no separate pass over Y.
+ * W_layout / s_w / side_layout / s_w_side come from mq_pack_w4_rms.  acc_out and acc_side_out
  * (device int32 [T, N], either may be NULL) receive the two integer accumulators.  ws:
  * device, 256-byte aligned, at least mq_rms_workspace_bytes(d) (else MQ_ERR_WORKSPACE).
  * Everything else as mq_w4a8_msq_linear.  Asynchronous on `stream`.
  */
 int mq_w4a8_msq_linear_rms(const mq_linear_desc* d, const void* X, int64_t ldx, const mq_segments* seg, float s_vis,
-                           float s_txt, const void* W_layout, const float* s_w, const int8_t* q_side,
+                           float s_txt, const void* W_layout, const float* s_w, const void* side_layout,
                            const float* s_w_side, const float* bias, void* Y, int64_t ldy, int32_t* acc_out,
                            int32_t* acc_side_out, void* ws, size_t ws_bytes, void* stream);
 

@@ -79,7 +79,7 @@ def load(build_if_missing: bool = False):
         "mq_w4a8_msq_linear_noalloc": (C.c_int, [descp, vp, i64, segp, f32, f32, vp, vp, vp, vp, i64, vp, vp, vp]),
         "mq_rms_side_ld": (sz, [i32, i32]),
         "mq_rms_detect": (C.c_int, [vp, i32, i32, i64, i32, vp, vp, vp]),
-        "mq_pack_w4_rms": (C.c_int, [vp, i32, i32, i64, i32, vp, vp, vp, vp, vp, vp]),
+        "mq_pack_w4_rms": (C.c_int, [vp, i32, i32, i64, i32, vp, vp, vp, vp, vp, vp, vp]),
         "mq_rms_workspace_bytes": (sz, [descp]),
         "mq_w4a8_msq_linear_rms": (C.c_int, [descp, vp, i64, segp, f32, f32, vp, vp, vp, vp, vp, vp, i64, vp, vp,
                                              vp, sz, vp]),
@@ -271,11 +271,12 @@ def mq_rms_detect(w, rot_block, flags=None, count_out=None):
            "mq_rms_detect")
 
 
-def mq_pack_w4_rms(w_rot, rot_block, s_w, q_side, s_w_side, packed=None, gemm_layout=None):
+def mq_pack_w4_rms(w_rot, rot_block, s_w, q_side, s_w_side, packed=None, gemm_layout=None, side_layout=None):
     assert w_rot.dtype == torch.float32 and q_side.dtype == torch.int8
     N, K = w_rot.shape
     _check(load().mq_pack_w4_rms(_ptr(w_rot), N, K, _ld(w_rot), rot_block, _ptr(packed), _ptr(s_w),
-                                 _ptr(gemm_layout), _ptr(q_side), _ptr(s_w_side), _stream()), "mq_pack_w4_rms")
+                                 _ptr(gemm_layout), _ptr(q_side), _ptr(s_w_side), _ptr(side_layout), _stream()),
+           "mq_pack_w4_rms")
 
 
 def mq_rms_workspace_bytes(T, K, N, rot_block, flags=0) -> int:
@@ -292,7 +293,7 @@ def new_rms_workspace(T, K, N, rot_block, flags=0, device="cuda") -> torch.Tenso
     return ws
 
 
-def mq_w4a8_msq_linear_rms(x, seg: Segments, s_vis, s_txt, w_layout, s_w, q_side, s_w_side, y, N, rot_block, ws,
+def mq_w4a8_msq_linear_rms(x, seg: Segments, s_vis, s_txt, w_layout, s_w, side_layout, s_w_side, y, N, rot_block, ws,
                            bias=None, acc_out=None, acc_side_out=None):
     """The rotated linear with rotation magnitude suppression (Sec. 3.2): main GEMM plus the
     split first-channel-of-each-block product, added before the bias."""
@@ -305,7 +306,7 @@ def mq_w4a8_msq_linear_rms(x, seg: Segments, s_vis, s_txt, w_layout, s_w, q_side
         assert y.dtype == torch.bfloat16
     d = mq_linear_desc(T, K, N, rot_block, 0, flags)
     _check(load().mq_w4a8_msq_linear_rms(C.byref(d), _ptr(x), _ld(x), seg.ref(), float(s_vis), float(s_txt),
-                                         _ptr(w_layout), _ptr(s_w), _ptr(q_side), _ptr(s_w_side), _ptr(bias),
+                                         _ptr(w_layout), _ptr(s_w), _ptr(side_layout), _ptr(s_w_side), _ptr(bias),
                                          _ptr(y), _ld(y), _ptr(acc_out), _ptr(acc_side_out), _ptr(ws), ws.numel(),
                                          _stream()), "mq_w4a8_msq_linear_rms")
 

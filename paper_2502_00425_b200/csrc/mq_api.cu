@@ -227,12 +227,27 @@ int check_rms_shape(int32_t N, int32_t K, int32_t rot_block) {
   if (rot_block == 0) return MQ_ERR_INVALID_ARG;  // the split columns are defined by the rotation block
   return check_rot(rot_block, K);
 }
-size_t rms_side_ld(int32_t K, int32_t rot_block) { return align_up((size_t)(K / rot_block), 4); }
+// K of the split product: one code per rotation block, padded to the GEMM's granularity.
+int rms_side_k(int32_t K, int32_t rot_block) { return (int)align_up((size_t)(K / rot_block), 32); }
+
+struct RmsWsLayout {
+  size_t qx_off, xs_off, splitk_off, splitk_bytes, total;
+};
+RmsWsLayout rms_ws_layout(const mq_linear_desc* d) {
+  RmsWsLayout w{};
+  const int sk = rms_side_k(d->K, d->rot_block);
+  w.qx_off = kStatusBytes;
+  w.xs_off = w.qx_off + align_up((size_t)d->T * d->K, 256);
+  w.splitk_off = w.xs_off + align_up((size_t)d->T * sk, 256);
+  w.splitk_bytes = align_up(gemm_splitk_bytes(d->T, d->K, d->N, true), 256);
+  w.total = w.splitk_off + w.splitk_bytes;
+  return w;
+}
 }  // namespace
 
 size_t mq_rms_side_ld(int32_t K, int32_t rot_block) {
-  if (K <= 0 || check_rot(rot_block, K) != MQ_OK || rot_block == 0) return 0;
-  return rms_side_ld(K, rot_block);
+  if (K <= 0 || K % 32 || rot_block == 0 || check_rot(rot_block, K) != MQ_OK) return 0;
+  return (size_t)rms_side_k(K, rot_block);
 }
 
 int mq_rms_detect(const float* W, int32_t N, int32_t K, int64_t ldw, int32_t rot_block, uint8_t* flags,
@@ -244,49 +259,65 @@ int mq_rms_detect(const float* W, int32_t N, int32_t K, int64_t ldw, int32_t rot
 }
 
 int mq_pack_w4_rms(const float* W_rot, int32_t N, int32_t K, int64_t ldw, int32_t rot_block, uint8_t* packed,
-                   float* s_w, void* gemm_layout, int8_t* q_side, float* s_w_side, void* stream) {
+                   float* s_w, void* gemm_layout, int8_t* q_side, float* s_w_side, void* side_layout,
+                   void* stream) {
   int rc = check_rms_shape(N, K, rot_block);
   if (rc != MQ_OK) return rc;
   if (!W_rot || !s_w || !q_side || !s_w_side || ldw < K) return MQ_ERR_INVALID_ARG;
   if (gemm_layout && !aligned(gemm_layout, 128)) return MQ_ERR_ALIGNMENT;
-  if (!aligned16(q_side)) return MQ_ERR_ALIGNMENT;
-  return launch_rms_pack(W_rot, N, K, ldw, rot_block, packed, s_w, gemm_layout, q_side,
-                         (int)rms_side_ld(K, rot_block), s_w_side, static_cast<cudaStream_t>(stream));
+  if (side_layout && !aligned(side_layout, 128)) return MQ_ERR_ALIGNMENT;
+  return launch_rms_pack(W_rot, N, K, ldw, rot_block, packed, s_w, gemm_layout, q_side, rms_side_k(K, rot_block),
+                         s_w_side, side_layout, static_cast<cudaStream_t>(stream));
 }
 
 size_t mq_rms_workspace_bytes(const mq_linear_desc* d) {
   if (check_desc(d) != MQ_OK || d->rot_block == 0 || (d->flags & MQ_FLAG_X_IS_INT8)) return 0;
-  return ws_layout(d).total + align_up((size_t)d->T * d->N * sizeof(float), 256);
+  return rms_ws_layout(d).total;
 }
 
 int mq_w4a8_msq_linear_rms(const mq_linear_desc* d, const void* X, int64_t ldx, const mq_segments* seg, float s_vis,
-                           float s_txt, const void* W_layout, const float* s_w, const int8_t* q_side,
+                           float s_txt, const void* W_layout, const float* s_w, const void* side_layout,
                            const float* s_w_side, const float* bias, void* Y, int64_t ldy, int32_t* acc_out,
                            int32_t* acc_side_out, void* ws, size_t ws_bytes, void* stream) {
   int rc = check_desc(d);
   if (rc != MQ_OK) return rc;
   if (d->rot_block == 0 || (d->flags & MQ_FLAG_X_IS_INT8)) return MQ_ERR_INVALID_ARG;
-  if (!q_side || !s_w_side || !Y || ldy < d->N) return MQ_ERR_INVALID_ARG;
-  if (!aligned16(q_side)) return MQ_ERR_ALIGNMENT;
+  if (!good_scale(s_vis) || !good_scale(s_txt)) return MQ_ERR_INVALID_ARG;
   SegTable st;
   if ((rc = check_seg(seg, &st)) != MQ_OK) return rc;
+  if (d->T == 0) return MQ_OK;
+  if (!X || !W_layout || !s_w || !side_layout || !s_w_side || !Y) return MQ_ERR_INVALID_ARG;
+  if (ldx < d->K || ldy < d->N) return MQ_ERR_INVALID_ARG;
+  if (!aligned16(X) || (ldx * 2) % 16) return MQ_ERR_ALIGNMENT;
+  if (!aligned(W_layout, 128) || !aligned(side_layout, 128) || !aligned16(Y) || !aligned16(s_w) ||
+      !aligned16(s_w_side))
+    return MQ_ERR_ALIGNMENT;
   if (!ws) return MQ_ERR_WORKSPACE;
   if (!aligned(ws, 256)) return MQ_ERR_ALIGNMENT;
-  const WsLayout wl = ws_layout(d);
-  const size_t y_bytes = align_up((size_t)d->T * d->N * sizeof(float), 256);
-  if (ws_bytes < wl.total + y_bytes) return MQ_ERR_WORKSPACE;
+  const RmsWsLayout wl = rms_ws_layout(d);
+  if (ws_bytes < wl.total) return MQ_ERR_WORKSPACE;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
   uint8_t* wsb = static_cast<uint8_t*>(ws);
-  float* y_main = reinterpret_cast<float*>(wsb + wl.total);
-  // main part: the ordinary linear, fp32 output, no bias (the bias is added once, after the sum)
-  mq_linear_desc dm = *d;
-  dm.flags |= MQ_FLAG_Y_IS_F32;
-  rc = mq_w4a8_msq_linear(&dm, X, ldx, seg, s_vis, s_txt, W_layout, s_w, nullptr, y_main, d->N, acc_out, ws,
-                          wl.total, stream);
+  const int sk = rms_side_k(d->K, d->rot_block);
+  int8_t* qx = reinterpret_cast<int8_t*>(wsb + wl.qx_off);
+  int8_t* xs = reinterpret_cast<int8_t*>(wsb + wl.xs_off);
+
+  // activation codes, then the codes of the first channel of every rotation block side by side
+  rc = launch_fwht_quant(X, d->T, d->K, ldx, st, s_vis, s_txt, d->rot_block, qx, d->K, nullptr, cs);
   if (rc != MQ_OK) return rc;
-  const int8_t* qx = reinterpret_cast<const int8_t*>(wsb + wl.qx_off);
-  return launch_rms_combine(y_main, qx, d->K, d->T, d->K, d->N, d->rot_block, st, s_vis, s_txt, q_side,
-                            (int)rms_side_ld(d->K, d->rot_block), s_w_side, bias, Y, ldy,
-                            (d->flags & MQ_FLAG_Y_IS_F32) ? 1 : 0, acc_side_out, static_cast<cudaStream_t>(stream));
+  rc = launch_rms_gather(qx, d->K, d->T, d->K / d->rot_block, d->rot_block, xs, sk, cs);
+  if (rc != MQ_OK) return rc;
+  // one GEMM launch: every tile runs the split product into a second accumulator, then the main one
+  GemmArgs a{};
+  a.T = d->T; a.K = d->K; a.N = d->N;
+  a.Qx = qx; a.ldq = d->K; a.seg = st; a.s_vis = s_vis; a.s_txt = s_txt;
+  a.W_layout = W_layout; a.s_w = s_w; a.bias = bias; a.Y = Y; a.ldy = ldy;
+  a.y_is_f32 = (d->flags & MQ_FLAG_Y_IS_F32) ? 1 : 0;
+  a.acc_out = acc_out;
+  a.status = reinterpret_cast<int32_t*>(wsb);
+  a.splitk_acc = wl.splitk_bytes ? reinterpret_cast<int32_t*>(wsb + wl.splitk_off) : nullptr;
+  a.Qs = xs; a.side_k = sk; a.side_layout = side_layout; a.s_w_side = s_w_side; a.acc_side_out = acc_side_out;
+  return launch_gemm(a, cs);
 }
 
 int mq_last_device_status(void* ws, void* stream, int32_t* site_out) {

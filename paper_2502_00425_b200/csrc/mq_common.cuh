@@ -105,10 +105,9 @@ int launch_mask_remap(const int32_t* perm, const int32_t* pos_ids, const uint8_t
 int launch_rms_detect(const float* W, int N, int K, int64_t ldw, int nb, uint8_t* flags, int32_t* count,
                       cudaStream_t st);
 int launch_rms_pack(const float* W, int N, int K, int64_t ldw, int nb, uint8_t* packed, float* s_w, void* layout,
-                    int8_t* q_side, int side_ld, float* s_w_side, cudaStream_t st);
-int launch_rms_combine(const float* y_main, const int8_t* qx, int64_t ldq, int T, int K, int N, int nb, SegTable seg,
-                       float s_vis, float s_txt, const int8_t* q_side, int side_ld, const float* s_w_side,
-                       const float* bias, void* Y, int64_t ldy, int y_is_f32, int32_t* acc_side_out, cudaStream_t st);
+                    int8_t* q_side, int side_k, float* s_w_side, void* side_layout, cudaStream_t st);
+int launch_rms_gather(const int8_t* qx, int64_t ldq, int T, int KBn, int nb, int8_t* xs, int side_k, cudaStream_t st);
+int launch_layout_from_codes(const int8_t* q, int64_t ldq, int N, int K, void* layout, cudaStream_t st);
 
 struct GemmArgs {
   int T, K, N;
@@ -124,9 +123,17 @@ struct GemmArgs {
   int y_is_f32;
   int32_t* acc_out;
   int32_t* status;     // device int32[2]: status, site
-  int32_t* splitk_acc; // device int32 [T,N] scratch (small-T path) or nullptr
+  int32_t* splitk_acc; // device int32 scratch of gemm_splitk_bytes (small-T path) or nullptr
+  // Split part of the rotation-magnitude-suppression linear (side_layout != nullptr selects it):
+  // a second product on K = side_k with its own weights and scale, accumulated beside the main one
+  // and added in the epilogue:  y = fl(acc * fl(s_a s_w)) + fl(acc_side * fl(s_a s_w_side)) (+ bias).
+  const int8_t* Qs;    // activation codes of the split product [T, side_k], pitch side_k
+  int side_k;          // multiple of 32
+  const void* side_layout;
+  const float* s_w_side;
+  int32_t* acc_side_out;
 };
 int launch_gemm(const GemmArgs& a, cudaStream_t st);
-size_t gemm_splitk_bytes(int T, int K, int N);
+size_t gemm_splitk_bytes(int T, int K, int N, bool rms = false);
 
 }  // namespace mq

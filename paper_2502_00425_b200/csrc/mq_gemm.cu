@@ -79,6 +79,13 @@ struct KernelParams {
   int32_t* acc_out;
   int32_t* splitk_acc;
   int32_t* status;
+  // split part of the rotation-magnitude-suppression linear (only read by the RMS instantiation)
+  int side_kb;                 // K blocks of the split product per tile (0: none)
+  int side_col;                // tensor-memory columns from an accumulator to its split accumulator
+  const uint8_t* side_layout;  // split weights, GEMM layout, side_kb tiles per channel tile
+  const float* s_w_side;
+  int32_t* acc_side_out;       // optional dump of the split accumulator [T, N]
+  int32_t* splitk_side;        // split-K launches: the split accumulator's own [T, N] slice
 };
 
 struct __align__(16) Barriers {
@@ -290,6 +297,27 @@ struct TileIter {
 // output) share one generic variant that tests its flags at run time.
 enum : int { kEpiSplitK = 1, kEpiAcc = 2, kEpiF32 = 4, kEpiBias = 8, kEpiGeneric = 16, kEpiStaged = 32 };
 
+// bf16 output of a 16 x 32 (token x channel) block held one channel per lane: transpose it
+// through this warp's staging buffer so that every lane stores 16 bytes (8 channels of one
+// token) instead of 2.
+__device__ __forceinline__ void staged_store(const KernelParams& p, const float (&y)[16], int t_first, int nvalid,
+                                             int n, __nv_bfloat16* stage) {
+  const int lane = threadIdx.x & 31;
+#pragma unroll
+  for (int j = 0; j < 16; ++j) stage[j * 32 + lane] = __float2bfloat16_rn(y[j]);
+  __syncwarp();
+  const int n8 = n - lane + (lane & 3) * 8;  // first of this lane's 8 channels
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    const int row = (lane >> 2) + 8 * h;
+    if (row < nvalid && n8 < p.N) {
+      const uint4 val = *reinterpret_cast<const uint4*>(stage + row * 32 + (lane & 3) * 8);
+      *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.Y) + (size_t)(t_first + row) * p.ldy + n8) = val;
+    }
+  }
+  __syncwarp();
+}
+
 // 16 token columns of one channel (this lane's n): dequantize and store, or add into the
 // split-K sums.  `nvalid` (1..16) masks the ragged end of the token range.
 template <int MODE>
@@ -329,22 +357,7 @@ __device__ __forceinline__ void epilogue_chunk(const KernelParams& p, const uint
     if (MODE & kEpiBias) y[j] = __fadd_rn(y[j], bs);
   }
   if (MODE & kEpiStaged) {
-    // bf16 output: transpose the 16 x 32 (token x channel) block through this warp's staging
-    // buffer so that every lane stores 16 bytes (8 channels of one token) instead of 2.
-    const int lane = threadIdx.x & 31;
-#pragma unroll
-    for (int j = 0; j < 16; ++j) stage[j * 32 + lane] = __float2bfloat16_rn(y[j]);
-    __syncwarp();
-    const int n8 = n - lane + (lane & 3) * 8;  // first of this lane's 8 channels
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-      const int row = (lane >> 2) + 8 * h;
-      if (row < nvalid && n8 < p.N) {
-        const uint4 val = *reinterpret_cast<const uint4*>(stage + row * 32 + (lane & 3) * 8);
-        *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(p.Y) + (size_t)(t_first + row) * p.ldy + n8) = val;
-      }
-    }
-    __syncwarp();
+    staged_store(p, y, t_first, nvalid, n, stage);
     return;
   }
 #pragma unroll
@@ -380,9 +393,80 @@ __device__ __forceinline__ void epilogue_tile(const KernelParams& p, uint32_t d_
   }
 }
 
+// Epilogue of a tile that carries a split accumulator (rotation magnitude suppression): the
+// main accumulator at d_tmem and the split one p.side_col columns further on, each with its
+// own per-channel weight scale:
+//   y = fl(acc_main * fl(s_a * s_w)) + fl(acc_side * fl(s_a * s_w_side)), then + bias.
+// STAGED: bf16 output through the staging buffer; otherwise every output the call asked for
+// (accumulator dumps, fp32 or bf16 Y) with predicated per-element stores.
+template <bool STAGED>
+__device__ __forceinline__ void epilogue_tile_side(const KernelParams& p, uint32_t d_tmem, int t0, int n, bool n_ok,
+                                                   float sw, float sws, float bs, const float* stok,
+                                                   __nv_bfloat16* stage) {
+  const int ncols = min(p.TN, p.T - t0);
+  const bool has_bias = p.bias != nullptr;
+  for (int cc = 0; cc < ncols; cc += 16) {
+    uint32_t vm[16], vs[16];
+    __syncwarp();
+    tmem_ld_x16(d_tmem + cc, vm);
+    tmem_ld_x16(d_tmem + p.side_col + cc, vs);
+    tmem_wait_ld();
+    const int nvalid = min(16, ncols - cc);
+    const int t_first = t0 + cc;
+    float y[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      const float st = stok[cc + j];
+      y[j] = __fadd_rn(__fmul_rn((float)(((int)vm[j]) >> 4), __fmul_rn(st, sw)),
+                       __fmul_rn((float)(((int)vs[j]) >> 4), __fmul_rn(st, sws)));
+      if (has_bias) y[j] = __fadd_rn(y[j], bs);
+    }
+    if (STAGED) {
+      staged_store(p, y, t_first, nvalid, n, stage);
+    } else if (n_ok) {
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        if (j < nvalid) {
+          const size_t t = (size_t)(t_first + j);
+          if (p.acc_out) p.acc_out[t * p.N + n] = ((int)vm[j]) >> 4;
+          if (p.acc_side_out) p.acc_side_out[t * p.N + n] = ((int)vs[j]) >> 4;
+          if (p.y_is_f32) static_cast<float*>(p.Y)[t * p.ldy + n] = y[j];
+          else static_cast<__nv_bfloat16*>(p.Y)[t * p.ldy + n] = __float2bfloat16_rn(y[j]);
+        }
+      }
+    }
+  }
+}
+
+// Split-K launch: the tile of K split 0 also owns the split accumulator; it goes to its own slice.
+__device__ __forceinline__ void epilogue_tile_side_slice(const KernelParams& p, uint32_t d_tmem, int t0, int n,
+                                                         bool n_ok) {
+  const int ncols = min(p.TN, p.T - t0);
+  for (int cc = 0; cc < ncols; cc += 16) {
+    uint32_t vs[16];
+    __syncwarp();
+    tmem_ld_x16(d_tmem + p.side_col + cc, vs);
+    tmem_wait_ld();
+    if (n_ok) {
+      int32_t* dst = p.splitk_side + (size_t)(t0 + cc) * p.N + n;
+#pragma unroll
+      for (int j = 0; j < 16; ++j)
+        if (cc + j < ncols) dst[(size_t)j * p.N] = ((int)vs[j]) >> 4;
+    }
+  }
+}
+
 // ------------------------------------------------------------------------------ the kernel
+// RMS = true is the instantiation behind the rotation-magnitude-suppression linear: every tile
+// (of K split 0) first runs the split product -- p.side_kb K blocks whose activations come
+// through tmap_side and whose weights come from p.side_layout -- into a second accumulator,
+// then the main product, and the epilogue combines the two.  The K blocks of both products
+// go through the same rings; only the sources and the MMA's destination differ.  A separate
+// instantiation keeps the ordinary kernel's code and register allocation as they were.
+template <bool RMS>
 __global__ void __launch_bounds__(kMaxThreads, 1)
-w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const KernelParams p) {
+w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const __grid_constant__ CUtensorMap tmap_side,
+                 const KernelParams p) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   // carve: activation stages (1024-aligned), weight stages, barriers, token scales
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -431,6 +515,15 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const KernelParam
       bool wrapped = false, ok = true;
       for (TileIter c = first; c.valid(p) && ok; c.next(p)) {
         const int row0 = c.tt * p.TN;
+        if (RMS && c.ks == 0) {
+          for (int sb = 0; sb < p.side_kb; ++sb, ++it) {
+            if (wrapped && !(ok = mbar_wait(&sh->done[s], ph ^ 1u, sh, p.status, 1))) break;
+            mbar_arrive_expect_tx(&sh->full[s], act_stage_bytes);
+            tma_load_2d(act_smem + (size_t)s * act_stage_bytes, &tmap_side, sb * kBlockK, row0, &sh->full[s]);
+            if (++s == p.stages) { s = 0; ph ^= 1u; wrapped = true; }
+          }
+          if (!ok) break;
+        }
         for (int kb = c.kb0(p), kb_end = c.kb1(p); kb < kb_end; ++kb, ++it) {
           if (wrapped && !(ok = mbar_wait(&sh->done[s], ph ^ 1u, sh, p.status, 1))) break;
           mbar_arrive_expect_tx(&sh->full[s], act_stage_bytes);
@@ -455,6 +548,16 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const KernelParam
       uint32_t ph = 0;
       bool wrapped = false, ok = true;
       for (TileIter c = first; c.valid(p) && ok; c.next(p)) {
+        if (RMS && c.ks == 0) {
+          const uint8_t* ssrc = p.side_layout + (size_t)c.tn * p.side_kb * kWTileBytes;
+          for (int sb = 0; sb < p.side_kb; ++sb, ++it, ssrc += kWTileBytes) {
+            if (wrapped && !(ok = mbar_wait(&sh->w_empty[s], ph ^ 1u, sh, p.status, 2))) break;
+            mbar_arrive_expect_tx(&sh->w_full[s], kWTileBytes);
+            bulk_load_1d(w_smem + (size_t)s * kWTileBytes, ssrc, kWTileBytes, &sh->w_full[s]);
+            if (++s == p.w_stages) { s = 0; ph ^= 1u; wrapped = true; }
+          }
+          if (!ok) break;
+        }
         const uint8_t* wsrc = p.W_layout + ((size_t)c.tn * p.kb_total + c.kb0(p)) * kWTileBytes;
         for (int kb = c.kb0(p), kb_end = c.kb1(p); kb < kb_end; ++kb, ++it, wsrc += kWTileBytes) {
           if (wrapped && !(ok = mbar_wait(&sh->w_empty[s], ph ^ 1u, sh, p.status, 2))) break;
@@ -483,6 +586,27 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const KernelParam
       tc_fence_after();
       const uint32_t d_tmem = tmem_base + (uint32_t)(d * p.d_stride);
       uint32_t accumulate = 0;
+      if (RMS && c.ks == 0) {
+        // the split product first, into its own accumulator
+        const uint32_t ds_tmem = d_tmem + (uint32_t)p.side_col;
+        for (int sb = 0; sb < p.side_kb; ++sb) {
+          if (!(ok = warp_all(mbar_wait(&sh->full[s], ph, sh, p.status, 4)))) break;
+          tc_fence_after();
+          const uint64_t bdesc = bdesc0 + (uint64_t)((uint32_t)s * bdesc_step);
+          const uint32_t a_tmem = tmem_base + (uint32_t)(p.a_base + a * 32);
+          if (elect_one()) {
+#pragma unroll
+            for (int k4 = 0; k4 < 4; ++k4)
+              mma_i8_ts(ds_tmem, a_tmem + k4 * 8, bdesc + (uint64_t)(k4 * 2), idesc, (accumulate | (uint32_t)k4));
+            tc_commit(&sh->done[s]);
+          }
+          accumulate = 1;
+          if (++s == p.stages) { s = 0; ph ^= 1u; }
+          if (++a == p.num_a) a = 0;
+        }
+        if (!ok) break;
+        accumulate = 0;
+      }
       for (int kb = c.kb0(p), kb_end = c.kb1(p); kb < kb_end; ++kb) {
         if (!(ok = warp_all(mbar_wait(&sh->full[s], ph, sh, p.status, 4)))) break;
         tc_fence_after();
@@ -517,7 +641,8 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const KernelParam
     const int grp = (warp - 4) >> 2;
     const int r = q * 32 + lane;  // channel row inside the tile == tensor-memory lane
     int total_it = 0;
-    for (TileIter c = first; c.valid(p); c.next(p)) total_it += c.kb1(p) - c.kb0(p);
+    for (TileIter c = first; c.valid(p); c.next(p))
+      total_it += c.kb1(p) - c.kb0(p) + ((RMS && c.ks == 0) ? p.side_kb : 0);
     int sw = grp, a = grp, s = grp;
     uint32_t ph_w = 0, ph = 0;
     bool ok = true;
@@ -583,11 +708,22 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const KernelParam
       const float sw = n_ok ? p.s_w[n] : 0.0f;
       const float bs = (n_ok && p.bias) ? p.bias[n] : 0.0f;
       const uint32_t d_tmem = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(d * p.d_stride);
-      switch (epi_mode) {
+      if (RMS) {
+        if (p.ksplit > 1) {
+          epilogue_tile<kEpiSplitK>(p, d_tmem, t0, n, n_ok, sw, bs, stok, stage, c.ks);
+          if (c.ks == 0) epilogue_tile_side_slice(p, d_tmem, t0, n, n_ok);
+        } else {
+          const float sws = n_ok ? p.s_w_side[n] : 0.0f;
+          if (plain && !p.acc_side_out) epilogue_tile_side<true>(p, d_tmem, t0, n, n_ok, sw, sws, bs, stok, stage);
+          else epilogue_tile_side<false>(p, d_tmem, t0, n, n_ok, sw, sws, bs, stok, stage);
+        }
+      } else {
+        switch (epi_mode) {
 #define MQ_EPI_CASE(M) case M: epilogue_tile<M>(p, d_tmem, t0, n, n_ok, sw, bs, stok, stage, c.ks); break;
-        MQ_EPI_CASE(kEpiStaged) MQ_EPI_CASE(kEpiStaged | kEpiBias) MQ_EPI_CASE(kEpiSplitK)
+          MQ_EPI_CASE(kEpiStaged) MQ_EPI_CASE(kEpiStaged | kEpiBias) MQ_EPI_CASE(kEpiSplitK)
 #undef MQ_EPI_CASE
-        default: epilogue_tile<kEpiGeneric>(p, d_tmem, t0, n, n_ok, sw, bs, stok, stage, c.ks); break;
+          default: epilogue_tile<kEpiGeneric>(p, d_tmem, t0, n, n_ok, sw, bs, stok, stage, c.ks); break;
+        }
       }
       tc_fence_before();
       __syncwarp();
@@ -606,9 +742,13 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const KernelParam
 
 
 // Split-K finalize: exact int32 partial sums -> dequantized output.
+// side_acc (optional): the split accumulator of the rotation-magnitude-suppression linear with
+// its own weight scale s_w_side; its term is added before the bias.
 __global__ void splitk_finalize_kernel(const int32_t* __restrict__ acc, int ksplit, int T, int N, SegTable seg, float s_vis,
                                        float s_txt, const float* __restrict__ s_w, const float* __restrict__ bias,
-                                       void* Y, int64_t ldy, int y_is_f32, int32_t* __restrict__ acc_out) {
+                                       void* Y, int64_t ldy, int y_is_f32, int32_t* __restrict__ acc_out,
+                                       const int32_t* __restrict__ side_acc, const float* __restrict__ s_w_side,
+                                       int32_t* __restrict__ acc_side_out) {
   pdl_launch_dependents();
   pdl_wait();
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -619,6 +759,11 @@ __global__ void splitk_finalize_kernel(const int32_t* __restrict__ acc, int kspl
   if (acc_out) acc_out[idx] = a;
   const float st = thread_row_modality(seg, t) == MQ_VISUAL ? s_vis : s_txt;
   float y = __fmul_rn((float)a, __fmul_rn(st, s_w[n]));
+  if (side_acc) {
+    const int sa = side_acc[idx];
+    if (acc_side_out) acc_side_out[idx] = sa;
+    y = __fadd_rn(y, __fmul_rn((float)sa, __fmul_rn(st, s_w_side[n])));
+  }
   if (bias) y = __fadd_rn(y, bias[n]);
   const size_t oy = (size_t)t * ldy + n;
   if (y_is_f32) static_cast<float*>(Y)[oy] = y;
@@ -658,16 +803,20 @@ int sm_count() {
   return n;
 }
 
-Plan make_plan(int T, int K, int N) {
+// rms: the launch carries a split accumulator next to every accumulator (rotation magnitude
+// suppression), so a token tile may use at most 224 of the 512 tensor-memory columns twice over,
+// there is a single accumulator pair, and what is left (>= 64 columns) holds the weight slots.
+Plan make_plan(int T, int K, int N, bool rms = false) {
   Plan pl{};
   const int sms = sm_count();
   pl.n_tn = (N + kTileN - 1) / kTileN;
   const int kb_total = (K + kBlockK - 1) / kBlockK;
   // token tile: as few tiles as possible, each as even as possible, multiple of 16
-  int n_tt = (T + 255) / 256;
+  const int tn_cap = rms ? 224 : 256;
+  int n_tt = (T + tn_cap - 1) / tn_cap;
   int TN = (((T + n_tt - 1) / n_tt) + 15) / 16 * 16;
   // several tiles per CTA: prefer <= 192 tokens so two accumulators fit and the epilogue overlaps
-  if ((long long)pl.n_tn * n_tt > sms && TN > 192) {
+  if (!rms && (long long)pl.n_tn * n_tt > sms && TN > 192) {
     n_tt = (T + 191) / 192;
     TN = (((T + n_tt - 1) / n_tt) + 15) / 16 * 16;
   }
@@ -676,6 +825,11 @@ Plan make_plan(int T, int K, int N) {
   pl.d_stride = TN <= 128 ? 128 : (TN <= 192 ? 192 : 256);
   pl.num_d = pl.d_stride <= 192 ? 2 : 1;
   pl.a_base = pl.num_d * pl.d_stride;
+  if (rms) {
+    pl.d_stride = (TN + 31) / 32 * 32;  // here: columns from the accumulator to its split accumulator
+    pl.num_d = 1;
+    pl.a_base = 2 * pl.d_stride;
+  }
   pl.num_a = (512 - pl.a_base) / 32;
   if (pl.num_a > kMaxStages) pl.num_a = kMaxStages;
   // split K when the tiles alone cannot fill the machine (small T: weight streaming)
@@ -713,15 +867,17 @@ Plan make_plan(int T, int K, int N) {
 
 }  // namespace
 
-size_t gemm_splitk_bytes(int T, int K, int N) {
+size_t gemm_splitk_bytes(int T, int K, int N, bool rms) {
   if (T <= 0 || K <= 0 || N <= 0) return 0;
-  const Plan pl = make_plan(T, K, N);
-  return pl.ksplit > 1 ? (size_t)pl.ksplit * T * N * sizeof(int32_t) : 0;  // one [T,N] slice per K split
+  const Plan pl = make_plan(T, K, N, rms);
+  // one [T,N] slice per K split, and one more for the split accumulator
+  return pl.ksplit > 1 ? (size_t)(pl.ksplit + (rms ? 1 : 0)) * T * N * sizeof(int32_t) : 0;
 }
 
 int launch_gemm(const GemmArgs& a, cudaStream_t st) {
   if (a.T == 0 || a.N == 0) return MQ_OK;
-  const Plan pl = make_plan(a.T, a.K, a.N);
+  const bool rms = a.side_layout != nullptr;
+  const Plan pl = make_plan(a.T, a.K, a.N, rms);
   EncodeTiledFn encode = get_encode_fn();
   if (!encode) return MQ_ERR_CUDA;
 
@@ -735,12 +891,23 @@ int launch_gemm(const GemmArgs& a, cudaStream_t st) {
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return MQ_ERR_CUDA;
 
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(w4a8_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget) !=
-        cudaSuccess)
+  // the split product's activation codes [T, side_k] (the ordinary launch passes the main map twice)
+  CUtensorMap tmap_side = tmap;
+  if (rms) {
+    const cuuint64_t sdims[2] = {(cuuint64_t)a.side_k, (cuuint64_t)a.T};
+    const cuuint64_t sstrides[1] = {(cuuint64_t)a.side_k};
+    if (encode(&tmap_side, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t*>(a.Qs), sdims, sstrides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return MQ_ERR_CUDA;
-    attr_set = true;
+  }
+
+  auto kernel = rms ? w4a8_gemm_kernel<true> : w4a8_gemm_kernel<false>;
+  static bool attr_set[2] = {false, false};
+  if (!attr_set[rms ? 1 : 0]) {
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget) != cudaSuccess)
+      return MQ_ERR_CUDA;
+    attr_set[rms ? 1 : 0] = true;
   }
 
   KernelParams p{};
@@ -757,15 +924,26 @@ int launch_gemm(const GemmArgs& a, cudaStream_t st) {
   p.W_layout = static_cast<const uint8_t*>(a.W_layout);
   p.s_w = a.s_w; p.bias = a.bias; p.Y = a.Y; p.ldy = a.ldy; p.y_is_f32 = a.y_is_f32;
   p.acc_out = a.acc_out; p.splitk_acc = a.splitk_acc; p.status = a.status;
+  int32_t* side_slice = nullptr;
+  if (rms) {
+    p.side_kb = (a.side_k + kBlockK - 1) / kBlockK;
+    p.side_col = pl.d_stride;
+    p.side_layout = static_cast<const uint8_t*>(a.side_layout);
+    p.s_w_side = a.s_w_side;
+    p.acc_side_out = a.acc_side_out;
+    if (pl.ksplit > 1 && a.splitk_acc) side_slice = a.splitk_acc + (size_t)pl.ksplit * a.T * a.N;
+    p.splitk_side = side_slice;
+  }
 
   if (pl.ksplit > 1 && !a.splitk_acc) return MQ_ERR_WORKSPACE;
-  if (launch_pdl(w4a8_gemm_kernel, dim3(pl.grid), dim3((8 + 4 * pl.groups) * 32), pl.smem, st, tmap, p) != cudaSuccess)
+  if (launch_pdl(kernel, dim3(pl.grid), dim3((8 + 4 * pl.groups) * 32), pl.smem, st, tmap, tmap_side, p) != cudaSuccess)
     return MQ_ERR_CUDA;
   if (pl.ksplit > 1) {
     const int64_t n = (int64_t)a.T * a.N;
     if (launch_pdl(splitk_finalize_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), 0, st,
                    static_cast<const int32_t*>(a.splitk_acc), pl.ksplit, a.T, a.N, a.seg, a.s_vis, a.s_txt, a.s_w, a.bias, a.Y,
-                   a.ldy, a.y_is_f32, a.acc_out) != cudaSuccess)
+                   a.ldy, a.y_is_f32, a.acc_out, static_cast<const int32_t*>(side_slice), a.s_w_side,
+                   a.acc_side_out) != cudaSuccess)
       return MQ_ERR_CUDA;
   }
   return MQ_OK;

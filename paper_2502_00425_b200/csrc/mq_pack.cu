@@ -117,6 +117,25 @@ __global__ void repack_kernel(const uint8_t* __restrict__ packed, int N, int K,
   layout[word] = out;
 }
 
+// GEMM layout from int4 codes stored one per byte (q [N, K], pitch ldq).
+__global__ void layout_from_codes_kernel(const int8_t* __restrict__ q, int64_t ldq, int N, int K,
+                                         uint32_t* __restrict__ layout, int KB, int64_t n_words) {
+  const int64_t word = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (word >= n_words) return;
+  const WordCoord c = layout_word_coord(word, KB);
+  uint32_t out = 0;
+  if (c.n < N) {
+#pragma unroll
+    for (int b = 0; b < 4; ++b) {
+      const int klo = c.k0 + b, khi = c.k0 + 4 + b;
+      const int qlo = klo < K ? q[(int64_t)c.n * ldq + klo] & 15 : 0;
+      const int qhi = khi < K ? q[(int64_t)c.n * ldq + khi] & 15 : 0;
+      out |= (uint32_t)(qlo | (qhi << 4)) << (8 * b);
+    }
+  }
+  layout[word] = out;
+}
+
 __global__ void unpack_kernel(const uint8_t* __restrict__ packed, const uint8_t* __restrict__ layout,
                               int N, int K, int KB, int8_t* __restrict__ q, int64_t ldq) {
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -154,6 +173,14 @@ int launch_pack_codes(const float* W, int N, int K, int64_t ldw, const float* s_
     pack_layout_kernel<<<(unsigned)((nw + 255) / 256), 256, 0, st>>>(
         W, N, K, ldw, s_w, static_cast<uint32_t*>(layout), (K + MQ_W_TILE_K - 1) / MQ_W_TILE_K, nw, skip);
   }
+  return cuda_status(cudaGetLastError());
+}
+
+int launch_layout_from_codes(const int8_t* q, int64_t ldq, int N, int K, void* layout, cudaStream_t st) {
+  if (N == 0 || K == 0) return MQ_OK;
+  const int64_t nw = layout_words(N, K);
+  layout_from_codes_kernel<<<(unsigned)((nw + 255) / 256), 256, 0, st>>>(
+      q, ldq, N, K, static_cast<uint32_t*>(layout), (K + MQ_W_TILE_K - 1) / MQ_W_TILE_K, nw);
   return cuda_status(cudaGetLastError());
 }
 

@@ -12,12 +12,14 @@
 //   rms_detect_kernel   Eq. 9 on the UNROTATED weight (offline; flags + count).
 //   rms_scale_kernel    per-output-channel int4 scales of the main part (split columns
 //                       excluded) and of the split part (only the split columns).
-//   rms_side_quant      int4 codes of the split part, one int8 per code, rows padded to a
-//                       multiple of four codes so the combine kernel reads 32-bit words.
-//   rms_combine_kernel  acc_side[t, n] = sum_b qx[t, b*n_rot] * q_side[n, b] and
-//                       y = main + float(acc_side) * (s_a * s_w_side[n]) + bias.
-// The main matrix goes through the ordinary W4A8 GEMM with the split columns packed as
-// code 0, so that kernel is unchanged.
+//   rms_side_quant      int4 codes of the split part, one int8 per code, rows padded with
+//                       zeros to a multiple of 32 codes (the GEMM's K granularity).
+//   rms_gather_kernel   the activation codes at the split channels, side by side.
+// The forward pass is ONE launch of the W4A8 GEMM (its RMS instantiation, see mq_gemm.cu):
+// every output tile first accumulates the split product -- activations from the gathered
+// codes, weights from the split part's layout -- into a second tensor-memory accumulator,
+// then the main product (split columns packed as code 0), and the epilogue computes
+//   y = fl(acc_main * fl(s_a * s_w[n])) + fl(acc_side * fl(s_a * s_w_side[n])) (+ bias[n]).
 #include <cuda_bf16.h>
 
 #include "mq_common.cuh"
@@ -101,59 +103,17 @@ __global__ void rms_side_quant_kernel(const float* __restrict__ W, int N, int KB
   q_side[idx] = b < KBn ? (int8_t)rtn_int4(W[(int64_t)n * ldw + (int64_t)b * nb], s_side[n]) : (int8_t)0;
 }
 
-// ------------------------------------------------------------------------------ combine
-// Step 3 of the remedy: the split part's product is added back.  A CTA owns kTok tokens and
-// kCombineThreads output channels.  The tokens' codes at the first channel of every block are
-// gathered into shared memory once (stride n_rot in the code matrix); a thread then walks
-// its channel's row of q_side four codes at a time with dp4a.  Arithmetic of the fp32 result:
-//   y = fadd(y_main, fmul(float(acc_side), fmul(s_a, s_w_side[n]))), then fadd(bias[n]).
-constexpr int kTok = 8;
-constexpr int kCombineThreads = 256;
-
-__global__ void __launch_bounds__(kCombineThreads)
-rms_combine_kernel(const float* __restrict__ y_main, const int8_t* __restrict__ qx, int64_t ldq, int T, int N, int nb,
-                   int KBn, SegTable seg, float s_vis, float s_txt, const int8_t* __restrict__ q_side, int side_ld,
-                   const float* __restrict__ s_w_side, const float* __restrict__ bias, void* __restrict__ Y,
-                   int64_t ldy, int y_is_f32, int32_t* __restrict__ acc_side_out) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  int32_t* xs = reinterpret_cast<int32_t*>(smem_raw);  // [kTok][side_ld / 4] words
-  __shared__ float s_tok[kTok];
-  const int t0 = blockIdx.y * kTok;
-  const int words = side_ld >> 2;
-  int8_t* xb = reinterpret_cast<int8_t*>(xs);
-  for (int i = threadIdx.x; i < kTok * side_ld; i += blockDim.x) {
-    const int tt = i / side_ld, b = i % side_ld;
-    const int t = t0 + tt;
-    xb[i] = (t < T && b < KBn) ? qx[(int64_t)t * ldq + (int64_t)b * nb] : (int8_t)0;
-  }
-  if (threadIdx.x < kTok) {
-    const int t = t0 + threadIdx.x;
-    s_tok[threadIdx.x] = (t < T && thread_row_modality(seg, t) == MQ_VISUAL) ? s_vis : s_txt;
-  }
-  __syncthreads();
-  const int n = blockIdx.x * kCombineThreads + threadIdx.x;
-  if (n >= N) return;
-  int acc[kTok];
-#pragma unroll
-  for (int j = 0; j < kTok; ++j) acc[j] = 0;
-  const int32_t* qrow = reinterpret_cast<const int32_t*>(q_side + (int64_t)n * side_ld);
-  for (int w = 0; w < words; ++w) {
-    const int q = __ldg(qrow + w);
-#pragma unroll
-    for (int j = 0; j < kTok; ++j) acc[j] = __dp4a(xs[j * words + w], q, acc[j]);
-  }
-  const float sw = s_w_side[n];
-  const float bs = bias ? bias[n] : 0.0f;
-#pragma unroll
-  for (int j = 0; j < kTok; ++j) {
-    const int t = t0 + j;
-    if (t >= T) break;
-    float y = __fadd_rn(y_main[(int64_t)t * N + n], __fmul_rn((float)acc[j], __fmul_rn(s_tok[j], sw)));
-    if (bias) y = __fadd_rn(y, bs);
-    if (y_is_f32) static_cast<float*>(Y)[(int64_t)t * ldy + n] = y;
-    else static_cast<__nv_bfloat16*>(Y)[(int64_t)t * ldy + n] = __float2bfloat16_rn(y);
-    if (acc_side_out) acc_side_out[(int64_t)t * N + n] = acc[j];
-  }
+// Codes of the first channel of every rotation block, side by side: xs[t, b] = qx[t, b * nb]
+// (b < KBn; the padding up to side_k is 0).  This is the activation operand of the split
+// product, K-contiguous so that the GEMM's tensor map can fetch it.
+__global__ void rms_gather_kernel(const int8_t* __restrict__ qx, int64_t ldq, int T, int KBn, int nb,
+                                  int8_t* __restrict__ xs, int side_k) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= (int64_t)T * side_k) return;
+  const int t = (int)(idx / side_k), b = (int)(idx % side_k);
+  xs[idx] = b < KBn ? qx[(int64_t)t * ldq + (int64_t)b * nb] : (int8_t)0;
 }
 
 }  // namespace
@@ -169,28 +129,26 @@ int launch_rms_detect(const float* W, int N, int K, int64_t ldw, int nb, uint8_t
 }
 
 int launch_rms_pack(const float* W, int N, int K, int64_t ldw, int nb, uint8_t* packed, float* s_w, void* layout,
-                    int8_t* q_side, int side_ld, float* s_w_side, cudaStream_t st) {
+                    int8_t* q_side, int side_k, float* s_w_side, void* side_layout, cudaStream_t st) {
   if (N == 0 || K == 0) return MQ_OK;
   rms_scale_kernel<<<N, 256, 0, st>>>(W, N, K, ldw, nb, s_w, s_w_side);
-  const int64_t n = (int64_t)N * side_ld;
+  const int64_t n = (int64_t)N * side_k;
   rms_side_quant_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(W, N, K / nb, ldw, nb, s_w_side, q_side,
-                                                                       side_ld);
+                                                                       side_k);
   if (cudaGetLastError() != cudaSuccess) return MQ_ERR_CUDA;
+  if (side_layout) {
+    const int rc = launch_layout_from_codes(q_side, side_k, N, side_k, side_layout, st);
+    if (rc != MQ_OK) return rc;
+  }
   return launch_pack_codes(W, N, K, ldw, s_w, packed, layout, nb, st);
 }
 
-int launch_rms_combine(const float* y_main, const int8_t* qx, int64_t ldq, int T, int K, int N, int nb, SegTable seg,
-                       float s_vis, float s_txt, const int8_t* q_side, int side_ld, const float* s_w_side,
-                       const float* bias, void* Y, int64_t ldy, int y_is_f32, int32_t* acc_side_out,
-                       cudaStream_t st) {
-  if (T == 0 || N == 0) return MQ_OK;
-  const size_t smem = (size_t)kTok * side_ld;
-  if (smem > 48 * 1024) return MQ_ERR_UNSUPPORTED;
-  dim3 grid((N + kCombineThreads - 1) / kCombineThreads, (T + kTok - 1) / kTok);
-  rms_combine_kernel<<<grid, kCombineThreads, smem, st>>>(y_main, qx, ldq, T, N, nb, K / nb, seg, s_vis, s_txt,
-                                                          q_side, side_ld, s_w_side, bias, Y, ldy, y_is_f32,
-                                                          acc_side_out);
-  return cuda_status(cudaGetLastError());
+int launch_rms_gather(const int8_t* qx, int64_t ldq, int T, int KBn, int nb, int8_t* xs, int side_k,
+                      cudaStream_t st) {
+  if (T == 0) return MQ_OK;
+  const int64_t n = (int64_t)T * side_k;
+  return cuda_status(launch_pdl(rms_gather_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), 0, st, qx, ldq, T,
+                                KBn, nb, xs, side_k));
 }
 
 }  // namespace mq

@@ -128,11 +128,13 @@ def test_other_entry_points_validate(lib):
 def test_rms_entry_points_validate(lib):
     A = 0x10000
     seg = B.mq_segments(0, None, None)
-    assert B.mq_rms_side_ld(18944, 128) == 148
-    assert B.mq_rms_side_ld(1152, 128) == 12                       # 9 blocks, padded to a multiple of 4
+    assert B.mq_rms_side_ld(18944, 128) == 160                     # 148 blocks, padded to a multiple of 32
+    assert B.mq_rms_side_ld(1152, 128) == 32
     assert B.mq_rms_side_ld(1152, 0) == 0 and B.mq_rms_side_ld(1152, 48) == 0
     base = B.mq_workspace_bytes(1088, 18944, 3584, 128)
-    assert B.mq_rms_workspace_bytes(1088, 18944, 3584, 128) == base + 1088 * 3584 * 4
+    assert B.mq_rms_workspace_bytes(1088, 18944, 3584, 128) == base + 1088 * 160    # + the gathered split codes
+    small_t = B.mq_workspace_bytes(8, 4096, 256, 128)
+    assert B.mq_rms_workspace_bytes(8, 4096, 256, 128) == small_t + 256 + 8 * 256 * 4   # + codes, + one more slice
     assert B.mq_rms_workspace_bytes(1088, 18944, 3584, 0) == 0      # no rotation, no split columns
     assert B.mq_rms_workspace_bytes(8, 128, 128, 0, B.MQ_FLAG_X_IS_INT8) == 0
     det = lib.mq_rms_detect
@@ -141,9 +143,9 @@ def test_rms_entry_points_validate(lib):
     assert det(A, 128, 256, 256, 16, A, A, None) == B.MQ_ERR_UNSUPPORTED
     assert det(A, 128, 256, 200, 128, A, A, None) == B.MQ_ERR_INVALID_ARG      # ldw < K
     pk = lib.mq_pack_w4_rms
-    assert pk(A, 128, 256, 256, 128, None, A, None, None, A, None) == B.MQ_ERR_INVALID_ARG   # q_side missing
-    assert pk(A, 128, 256, 256, 128, None, A, None, A + 4, A, None) == B.MQ_ERR_ALIGNMENT
-    assert pk(A, 128, 256, 256, 96, None, A, None, A, A, None) == B.MQ_ERR_INVALID_ARG
+    assert pk(A, 128, 256, 256, 128, None, A, None, None, A, None, None) == B.MQ_ERR_INVALID_ARG   # q_side missing
+    assert pk(A, 128, 256, 256, 128, None, A, None, A, A, A + 16, None) == B.MQ_ERR_ALIGNMENT
+    assert pk(A, 128, 256, 256, 96, None, A, None, A, A, None, None) == B.MQ_ERR_INVALID_ARG
     f = lib.mq_w4a8_msq_linear_rms
     d = _desc(8, 256, 128, rot=0)
     assert f(C.byref(d), A, 256, C.byref(seg), 1.0, 1.0, A, A, A, A, None, A, 128, None, None, A, 1 << 30,

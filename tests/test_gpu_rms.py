@@ -27,8 +27,9 @@ def _gpu_pack_rms(w_rot, rot):
     layout = torch.empty(B.mq_w4_layout_bytes(N, K), dtype=torch.uint8, device=DEV)
     q_side = torch.full((N, side_ld), 99, dtype=torch.int8, device=DEV)
     s_side = torch.empty(N, dtype=torch.float32, device=DEV)
-    B.mq_pack_w4_rms(wd, rot, s_w, q_side, s_side, packed, layout)
-    return packed, s_w, layout, q_side, s_side
+    side_layout = torch.empty(B.mq_w4_layout_bytes(N, side_ld), dtype=torch.uint8, device=DEV)
+    B.mq_pack_w4_rms(wd, rot, s_w, q_side, s_side, packed, layout, side_layout)
+    return packed, s_w, layout, q_side, s_side, side_layout
 
 
 @pytest.mark.parametrize("N,K,rot", [(64, 512, 128), (272, 1152, 128), (48, 160, 32), (16, 2048, 1024)])
@@ -54,13 +55,16 @@ def test_rms_pack_matches_oracle(N, K, rot):
     w_main, w_side = O.rms_split(w_rot, rot)
     q_main, s_main = O.quantize_weight_int4(w_main)
     q_sd, s_sd = O.quantize_weight_int4(w_side)
-    packed, s_w, layout, q_side, s_side = _gpu_pack_rms(w_rot, rot)
+    packed, s_w, layout, q_side, s_side, side_layout = _gpu_pack_rms(w_rot, rot)
     assert np.array_equal(s_w.cpu().numpy(), s_main)
     assert np.array_equal(s_side.cpu().numpy(), s_sd)
     nb = K // rot
     qs = q_side.cpu().numpy()
     assert np.array_equal(qs[:, :nb], q_sd)
     assert not qs[:, nb:].any()               # padding codes
+    side = torch.empty((N, qs.shape[1]), dtype=torch.int8, device=DEV)
+    B.mq_unpack_w4(N, qs.shape[1], side, gemm_layout=side_layout)
+    assert np.array_equal(side.cpu().numpy(), qs)
     for src in ("packed", "layout"):
         out = torch.empty((N, K), dtype=torch.int8, device=DEV)
         B.mq_unpack_w4(N, K, out, packed=packed if src == "packed" else None,
@@ -71,11 +75,11 @@ def test_rms_pack_matches_oracle(N, K, rot):
 
 
 @pytest.mark.parametrize("T_vis,T_txt,K,N,rot,with_bias", [
-    (40, 27, 1152, 272, 128, False),   # ragged token group, ragged channel tile, 9 blocks (side row padded to 12)
+    (40, 27, 1152, 272, 128, False),   # ragged token group, ragged channel tile, 9 blocks (side row padded to 32)
     (3, 5, 4096, 256, 128, True),      # T = 8: the small-T GEMM path underneath, 32 blocks
     (150, 60, 160, 144, 32, True),     # five blocks of 32, two token tiles of the main GEMM
     (0, 9, 2048, 64, 1024, False),     # two blocks of 1024
-    (300, 33, 2304, 528, 128, True),   # several CTAs in both grid dimensions of the combine kernel
+    (300, 33, 2304, 528, 128, True),   # 18 blocks, five channel tiles, two token tiles
 ])
 def test_rms_linear_matches_oracle(T_vis, T_txt, K, N, rot, with_bias):
     c, w, w_rot = _rms_case(300 + K + N, T_vis, T_txt, K, N, rot)
@@ -88,7 +92,7 @@ def test_rms_linear_matches_oracle(T_vis, T_txt, K, N, rot, with_bias):
         bias = (np.random.default_rng(5).standard_normal(N) * 0.5).astype(np.float32)
     ref = O.linear_w4a8_msq_rms(c.x, c.seg.seg_end, c.seg.seg_mod, s_v, s_t, rot, q_main, s_main, q_sd, s_sd, bias)
     assert np.abs(ref["acc_side"]).max() > 0
-    packed, s_w, layout, q_side, s_side = _gpu_pack_rms(w_rot, rot)
+    packed, s_w, layout, q_side, s_side, side_layout = _gpu_pack_rms(w_rot, rot)
     T = c.T
     x = bf16_to_dev(c.x)
     seg = dev_segments(c.seg)
@@ -98,7 +102,7 @@ def test_rms_linear_matches_oracle(T_vis, T_txt, K, N, rot, with_bias):
         y = torch.full((T, N), float("nan"), dtype=dt, device=DEV)
         acc = torch.full((T, N), -(2 ** 31), dtype=torch.int32, device=DEV)
         acc_s = torch.full((T, N), -(2 ** 31), dtype=torch.int32, device=DEV)
-        B.mq_w4a8_msq_linear_rms(x, seg, s_v, s_t, layout, s_w, q_side, s_side, y, N, rot, ws, bias=bias_d,
+        B.mq_w4a8_msq_linear_rms(x, seg, s_v, s_t, layout, s_w, side_layout, s_side, y, N, rot, ws, bias=bias_d,
                                  acc_out=acc, acc_side_out=acc_s)
         assert B.mq_last_device_status(ws) == (B.MQ_OK, 0)
         assert np.array_equal(acc.cpu().numpy(), ref["acc_main"])
@@ -116,7 +120,7 @@ def test_rms_linear_matches_oracle(T_vis, T_txt, K, N, rot, with_bias):
     # without the optional accumulator outputs
     ws = B.new_rms_workspace(T, K, N, rot)
     y2 = torch.empty((T, N), dtype=torch.bfloat16, device=DEV)
-    B.mq_w4a8_msq_linear_rms(x, seg, s_v, s_t, layout, s_w, q_side, s_side, y2, N, rot, ws, bias=bias_d)
+    B.mq_w4a8_msq_linear_rms(x, seg, s_v, s_t, layout, s_w, side_layout, s_side, y2, N, rot, ws, bias=bias_d)
     assert np.array_equal(bf16_from_dev(y2), ref["y_bf16"])
 
 
@@ -127,11 +131,11 @@ def test_rms_recovers_what_plain_w4_loses():
     c, w, w_rot = _rms_case(900, 64, 32, K, N, rot)
     s_v, s_t = gpu_calibrate(c.x_calib, c.seg_calib, rot)
     exact = c.x.astype(np.float64) @ w.astype(np.float64).T
-    packed, s_w, layout, q_side, s_side = _gpu_pack_rms(w_rot, rot)
+    packed, s_w, layout, q_side, s_side, side_layout = _gpu_pack_rms(w_rot, rot)
     x, seg = bf16_to_dev(c.x), dev_segments(c.seg)
     ws = B.new_rms_workspace(c.T, K, N, rot)
     y_rms = torch.empty((c.T, N), dtype=torch.float32, device=DEV)
-    B.mq_w4a8_msq_linear_rms(x, seg, s_v, s_t, layout, s_w, q_side, s_side, y_rms, N, rot, ws)
+    B.mq_w4a8_msq_linear_rms(x, seg, s_v, s_t, layout, s_w, side_layout, s_side, y_rms, N, rot, ws)
     # plain: same rotated weight, one scale per channel over all input channels
     wd = torch.from_numpy(w_rot).to(DEV)
     s_plain = torch.empty(N, dtype=torch.float32, device=DEV)
