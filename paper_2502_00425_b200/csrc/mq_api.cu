@@ -302,10 +302,9 @@ int mq_w4a8_msq_linear_rms(const mq_linear_desc* d, const void* X, int64_t ldx, 
   int8_t* qx = reinterpret_cast<int8_t*>(wsb + wl.qx_off);
   int8_t* xs = reinterpret_cast<int8_t*>(wsb + wl.xs_off);
 
-  // activation codes, then the codes of the first channel of every rotation block side by side
-  rc = launch_fwht_quant(X, d->T, d->K, ldx, st, s_vis, s_txt, d->rot_block, qx, d->K, nullptr, cs);
-  if (rc != MQ_OK) return rc;
-  rc = launch_rms_gather(qx, d->K, d->T, d->K / d->rot_block, d->rot_block, xs, sk, cs);
+  // activation codes; the quantizer also writes the codes of the first channel of every
+  // rotation block side by side (the split product's operand)
+  rc = launch_fwht_quant(X, d->T, d->K, ldx, st, s_vis, s_txt, d->rot_block, qx, d->K, nullptr, cs, xs, sk);
   if (rc != MQ_OK) return rc;
   // one GEMM launch: every tile runs the split product into a second accumulator, then the main one
   GemmArgs a{};
@@ -316,7 +315,7 @@ int mq_w4a8_msq_linear_rms(const mq_linear_desc* d, const void* X, int64_t ldx, 
   a.acc_out = acc_out;
   a.status = reinterpret_cast<int32_t*>(wsb);
   a.splitk_acc = wl.splitk_bytes ? reinterpret_cast<int32_t*>(wsb + wl.splitk_off) : nullptr;
-  a.Qs = xs; a.side_k = sk; a.side_layout = side_layout; a.s_w_side = s_w_side; a.acc_side_out = acc_side_out;
+  a.Qs = xs; a.side_k = sk; a.side_cols = d->K / d->rot_block; a.side_layout = side_layout; a.s_w_side = s_w_side; a.acc_side_out = acc_side_out;
   return launch_gemm(a, cs);
 }
 

@@ -83,7 +83,7 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
 // host launchers implemented in the .cu files -----------------------------------------
 int launch_fwht_quant(const void* X, int T, int K, int64_t ldx, SegTable seg, float s_vis,
                       float s_txt, int rot_block, int8_t* Q, int64_t ldq, float* rotated_out,
-                      cudaStream_t st);
+                      cudaStream_t st, int8_t* side_out = nullptr, int side_ld = 0);
 int launch_calibrate(const void* X, int T, int K, int64_t ldx, SegTable seg, int rot_block,
                      int accumulate, uint32_t* amax_state, float* s_vis_out, float* s_txt_out,
                      cudaStream_t st);
@@ -106,7 +106,6 @@ int launch_rms_detect(const float* W, int N, int K, int64_t ldw, int nb, uint8_t
                       cudaStream_t st);
 int launch_rms_pack(const float* W, int N, int K, int64_t ldw, int nb, uint8_t* packed, float* s_w, void* layout,
                     int8_t* q_side, int side_k, float* s_w_side, void* side_layout, cudaStream_t st);
-int launch_rms_gather(const int8_t* qx, int64_t ldq, int T, int KBn, int nb, int8_t* xs, int side_k, cudaStream_t st);
 int launch_layout_from_codes(const int8_t* q, int64_t ldq, int N, int K, void* layout, cudaStream_t st);
 
 struct GemmArgs {
@@ -127,8 +126,9 @@ struct GemmArgs {
   // Split part of the rotation-magnitude-suppression linear (side_layout != nullptr selects it):
   // a second product on K = side_k with its own weights and scale, accumulated beside the main one
   // and added in the epilogue:  y = fl(acc * fl(s_a s_w)) + fl(acc_side * fl(s_a s_w_side)) (+ bias).
-  const int8_t* Qs;    // activation codes of the split product [T, side_k], pitch side_k
+  const int8_t* Qs;    // activation codes of the split product [T, side_cols], pitch side_k
   int side_k;          // multiple of 32
+  int side_cols;       // columns of Qs that hold codes (<= side_k); the rest is never read
   const void* side_layout;
   const float* s_w_side;
   int32_t* acc_side_out;

@@ -23,7 +23,10 @@ namespace {
 constexpr int kWarpsPerCta = 8;
 constexpr int kWarpTile = 1024;  // channels per warp pass
 
-enum Mode { kQuant = 0, kQuantDump = 1, kAbsMax = 2 };
+// kQuantSide: also writes the code of the first channel of every rotation block to
+// side_out[row, block] -- the activation operand of the split product of rotation
+// magnitude suppression (Sec. 3.2), K-contiguous for the GEMM's tensor map.
+enum Mode { kQuant = 0, kQuantDump = 1, kAbsMax = 2, kQuantSide = 3 };
 
 __device__ __forceinline__ uint32_t pack_sat_s8x4(int q0, int q1, int q2, int q3) {
   // cvt.pack.sat.s8.s32.b32 d, a, b, c : d = { c[15:0], sat8(a), sat8(b) } (b in the low byte)
@@ -38,7 +41,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32)
 fwht_quant_kernel(const uint16_t* __restrict__ X, int T, int K, int64_t ldx, SegTable seg,
                   float inv_vis, float inv_txt, float c_n, int8_t* __restrict__ Q, int64_t ldq,
                   float* __restrict__ rotated_out, uint32_t* __restrict__ amax_state,
-                  int tiles_per_row, unsigned n_warp_tiles) {
+                  int tiles_per_row, unsigned n_warp_tiles, int8_t* __restrict__ side_out, int side_ld) {
   constexpr int TPB = 1 << LOG_TPB;
   pdl_launch_dependents();
   pdl_wait();
@@ -142,6 +145,8 @@ fwht_quant_kernel(const uint16_t* __restrict__ X, int T, int K, int64_t ldx, Seg
     o.x = pack_sat_s8x4(q[0], q[1], q[2], q[3]);
     o.y = pack_sat_s8x4(q[4], q[5], q[6], q[7]);
     *reinterpret_cast<uint2*>(qrow + off) = o;
+    if (MODE == kQuantSide && i == 0 && j == 0)  // element 0 of the block is in chunk 0 of lane-in-block 0
+      side_out[(int64_t)row * side_ld + (blk_start >> (5 + LOG_TPB))] = (int8_t)(o.x & 0xffu);
   }
 }
 
@@ -161,7 +166,7 @@ __global__ void calib_finalize_kernel(const uint32_t* amax_state, float* s_vis_o
 template <int MODE>
 int dispatch(const void* X, int T, int K, int64_t ldx, SegTable seg, float inv_vis, float inv_txt,
              int rot_block, int8_t* Q, int64_t ldq, float* rotated_out, uint32_t* amax_state,
-             cudaStream_t st) {
+             cudaStream_t st, int8_t* side_out = nullptr, int side_ld = 0) {
   if (T == 0 || K == 0) return MQ_OK;
   const int tiles_per_row = (K + kWarpTile - 1) / kWarpTile;
   const long long n_warp_tiles = (long long)T * tiles_per_row;
@@ -172,7 +177,7 @@ int dispatch(const void* X, int T, int K, int64_t ldx, SegTable seg, float inv_v
   const uint16_t* x = static_cast<const uint16_t*>(X);
 #define MQ_LAUNCH(LOG_TPB, ROT)                                                              \
   launch_pdl(fwht_quant_kernel<LOG_TPB, ROT, MODE>, grid, block, 0, st, x, T, K, ldx, seg, inv_vis, inv_txt, c_n, \
-             Q, ldq, rotated_out, amax_state, tiles_per_row, (unsigned)n_warp_tiles)
+             Q, ldq, rotated_out, amax_state, tiles_per_row, (unsigned)n_warp_tiles, side_out, side_ld)
   switch (rot_block) {
     case 0: MQ_LAUNCH(2, false); break;
     case 32: MQ_LAUNCH(0, true); break;
@@ -191,8 +196,13 @@ int dispatch(const void* X, int T, int K, int64_t ldx, SegTable seg, float inv_v
 
 int launch_fwht_quant(const void* X, int T, int K, int64_t ldx, SegTable seg, float s_vis,
                       float s_txt, int rot_block, int8_t* Q, int64_t ldq, float* rotated_out,
-                      cudaStream_t st) {
+                      cudaStream_t st, int8_t* side_out, int side_ld) {
   const float inv_vis = 1.0f / s_vis, inv_txt = 1.0f / s_txt;
+  if (side_out) {
+    if (!rot_block || rotated_out) return MQ_ERR_INVALID_ARG;
+    return dispatch<kQuantSide>(X, T, K, ldx, seg, inv_vis, inv_txt, rot_block, Q, ldq, nullptr, nullptr, st,
+                                side_out, side_ld);
+  }
   if (rotated_out)
     return dispatch<kQuantDump>(X, T, K, ldx, seg, inv_vis, inv_txt, rot_block, Q, ldq, rotated_out,
                                 nullptr, st);

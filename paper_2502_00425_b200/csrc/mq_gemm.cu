@@ -894,7 +894,8 @@ int launch_gemm(const GemmArgs& a, cudaStream_t st) {
   // the split product's activation codes [T, side_k] (the ordinary launch passes the main map twice)
   CUtensorMap tmap_side = tmap;
   if (rms) {
-    const cuuint64_t sdims[2] = {(cuuint64_t)a.side_k, (cuuint64_t)a.T};
+    // columns past side_cols are out of bounds for the map and arrive as zeros
+    const cuuint64_t sdims[2] = {(cuuint64_t)a.side_cols, (cuuint64_t)a.T};
     const cuuint64_t sstrides[1] = {(cuuint64_t)a.side_k};
     if (encode(&tmap_side, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t*>(a.Qs), sdims, sstrides, box, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,

@@ -14,7 +14,7 @@
 //                       excluded) and of the split part (only the split columns).
 //   rms_side_quant      int4 codes of the split part, one int8 per code, rows padded with
 //                       zeros to a multiple of 32 codes (the GEMM's K granularity).
-//   rms_gather_kernel   the activation codes at the split channels, side by side.
+// (The activation codes at the split channels are written side by side by the quantizer.)
 // The forward pass is ONE launch of the W4A8 GEMM (its RMS instantiation, see mq_gemm.cu):
 // every output tile first accumulates the split product -- activations from the gathered
 // codes, weights from the split part's layout -- into a second tensor-memory accumulator,
@@ -103,19 +103,6 @@ __global__ void rms_side_quant_kernel(const float* __restrict__ W, int N, int KB
   q_side[idx] = b < KBn ? (int8_t)rtn_int4(W[(int64_t)n * ldw + (int64_t)b * nb], s_side[n]) : (int8_t)0;
 }
 
-// Codes of the first channel of every rotation block, side by side: xs[t, b] = qx[t, b * nb]
-// (b < KBn; the padding up to side_k is 0).  This is the activation operand of the split
-// product, K-contiguous so that the GEMM's tensor map can fetch it.
-__global__ void rms_gather_kernel(const int8_t* __restrict__ qx, int64_t ldq, int T, int KBn, int nb,
-                                  int8_t* __restrict__ xs, int side_k) {
-  pdl_launch_dependents();
-  pdl_wait();
-  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx >= (int64_t)T * side_k) return;
-  const int t = (int)(idx / side_k), b = (int)(idx % side_k);
-  xs[idx] = b < KBn ? qx[(int64_t)t * ldq + (int64_t)b * nb] : (int8_t)0;
-}
-
 }  // namespace
 
 int launch_rms_detect(const float* W, int N, int K, int64_t ldw, int nb, uint8_t* flags, int32_t* count,
@@ -141,14 +128,6 @@ int launch_rms_pack(const float* W, int N, int K, int64_t ldw, int nb, uint8_t* 
     if (rc != MQ_OK) return rc;
   }
   return launch_pack_codes(W, N, K, ldw, s_w, packed, layout, nb, st);
-}
-
-int launch_rms_gather(const int8_t* qx, int64_t ldq, int T, int KBn, int nb, int8_t* xs, int side_k,
-                      cudaStream_t st) {
-  if (T == 0) return MQ_OK;
-  const int64_t n = (int64_t)T * side_k;
-  return cuda_status(launch_pdl(rms_gather_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), 0, st, qx, ldq, T,
-                                KBn, nb, xs, side_k));
 }
 
 }  // namespace mq
