@@ -811,14 +811,33 @@ Plan make_plan(int T, int K, int N, bool rms = false) {
   const int sms = sm_count();
   pl.n_tn = (N + kTileN - 1) / kTileN;
   const int kb_total = (K + kBlockK - 1) / kBlockK;
-  // token tile: as few tiles as possible, each as even as possible, multiple of 16
+  // Token tile.  Candidates: T cut into n_tt even tiles (multiple of 16, at most tn_cap tokens).
+  // Each is rated with a small model of the kernel: a CTA runs `rounds` tiles one after the
+  // other; a K block costs four MMAs whose duration is flat up to 192 tokens and grows beyond
+  // (measured: 112 cycles up to N = 192, 120 at 224, 136 at 256); the epilogue (~25 cycles per
+  // token column) hides behind the next tile's main loop only when two accumulators fit
+  // (tiles of <= 192 tokens).  The cheapest candidate wins; ties go to the larger tile.
   const int tn_cap = rms ? 224 : 256;
   int n_tt = (T + tn_cap - 1) / tn_cap;
   int TN = (((T + n_tt - 1) / n_tt) + 15) / 16 * 16;
-  // several tiles per CTA: prefer <= 192 tokens so two accumulators fit and the epilogue overlaps
-  if (!rms && (long long)pl.n_tn * n_tt > sms && TN > 192) {
-    n_tt = (T + 191) / 192;
-    TN = (((T + n_tt - 1) / n_tt) + 15) / 16 * 16;
+  if ((long long)pl.n_tn * n_tt > sms) {  // several tiles per CTA; otherwise the fewest tiles are right
+    double best = 0.0;
+    const int n_min = n_tt;
+    for (int cand = n_min; cand <= n_min * 4 && cand <= (T + 15) / 16; ++cand) {
+      const int tn = (((T + cand - 1) / cand) + 15) / 16 * 16;
+      const long long tiles_c = (long long)pl.n_tn * cand;
+      const long long rounds = (tiles_c + sms - 1) / sms;
+      const double mma = tn <= 192 ? 112.0 : (tn <= 224 ? 112.0 + (tn - 192) * 0.25 : 120.0 + (tn - 224) * 0.5);
+      const double epi = 25.0 * tn;
+      const bool two_acc = !rms && tn <= 192;
+      const double main_loop = 4.0 * mma * kb_total;
+      const double est = two_acc ? rounds * main_loop + epi : rounds * (main_loop + epi);
+      if (cand == n_min || est < best * 0.995) {
+        best = est;
+        n_tt = cand;
+        TN = tn;
+      }
+    }
   }
   pl.TN = TN;
   pl.n_tt = n_tt;
