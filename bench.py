@@ -223,6 +223,60 @@ def decode_sweep(torch, B, dev, peaks, n_sets=6, reps=20):
     return out
 
 
+# ------------------------------------------------------------------------------------------ RMS linear
+def rms_linear_timing(torch, B, dev, T, K, N, rot, n_sets=4, reps=10):
+    """Rotation magnitude suppression (Sec. 3.2) on the config-2 down-projection: the linear with
+    the split product (one launch, second accumulator) against the plain linear of the same
+    shape, both as rotation + quantizer + GEMM, CUDA-graph replays over n_sets rotating copies of
+    activations and weights (larger than L2 in total).  Random valid weight bytes: timing only,
+    parity is covered by the tests."""
+    g = torch.Generator(device="cpu").manual_seed(12)
+    seg = B.Segments.from_host([T - 64, T], [1, 0], dev)
+    side_k = B.mq_rms_side_ld(K, rot)
+    sets = []
+    for _ in range(n_sets):
+        x = (torch.randn((T, K), generator=g, dtype=torch.float32) * 2).to(torch.bfloat16).to(dev)
+        lay = torch.randint(0, 256, (B.mq_w4_layout_bytes(N, K),), dtype=torch.uint8, generator=g).to(dev)
+        slay = torch.randint(0, 256, (B.mq_w4_layout_bytes(N, side_k),), dtype=torch.uint8, generator=g).to(dev)
+        s_w = (torch.rand(N, generator=g) * 0.01 + 0.001).to(dev)
+        s_ws = (torch.rand(N, generator=g) * 0.05 + 0.001).to(dev)
+        y = torch.empty((T, N), dtype=torch.bfloat16, device=dev)
+        sets.append((x, lay, slay, s_w, s_ws, y, B.new_workspace(T, K, N, rot), B.new_rms_workspace(T, K, N, rot)))
+
+    def plain(i):
+        x, lay, slay, s_w, s_ws, y, ws, wsr = sets[i % n_sets]
+        B.mq_w4a8_msq_linear(x, seg, 0.5, 0.05, lay, s_w, y, ws, N, rot_block=rot)
+
+    def rms(i):
+        x, lay, slay, s_w, s_ws, y, ws, wsr = sets[i % n_sets]
+        B.mq_w4a8_msq_linear_rms(x, seg, 0.5, 0.05, lay, s_w, slay, s_ws, y, N, rot, wsr)
+
+    out = {}
+    for name, fn in (("plain_us", plain), ("rms_us", rms)):
+        for i in range(n_sets):
+            fn(i)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            for i in range(n_sets):
+                fn(i)
+        graph.replay()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            graph.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        out[name] = e0.elapsed_time(e1) * 1e3 / (reps * n_sets)
+        del graph
+    ok = all(B.mq_last_device_status(s_[6])[0] == 0 and B.mq_last_device_status(s_[7])[0] == 0 for s_ in sets)
+    out.update({"workload": "config2 down_proj T=%d K=%d N=%d rot=%d: quantizer + GEMM" % (T, K, N, rot),
+                "overhead_frac": out["rms_us"] / out["plain_us"] - 1.0,
+                "split_k_codes": side_k, "split_macs_frac": (K // rot) / K, "status_ok": ok})
+    return out
+
+
 # ------------------------------------------------------------------------------------------ layer linear suites
 def linear_suite(torch, B, dev, name, T, n_vis_per_seq, n_txt_per_seq, batch, shape, reps=5):
     """The seven W4A8 MSQ linears of one decoder block (configs 3 and 4, linear-suite mode): every
@@ -310,7 +364,7 @@ class BufferSet:
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one w4a8_gemm_kernel launch on this workload
 # (ncu capture summarised in profiles/); None once the kernel has changed since the capture.
-GEMM_TRAFFIC_BYTES = 56.64e6
+GEMM_TRAFFIC_BYTES = 57.44e6
 LAUNCHES_PER_STEP = 5  # index scan, row gather, remap, rotation+quantizer, GEMM
 
 
@@ -523,7 +577,7 @@ def run_ours(args, info):
     e2e_ops, _ = D.aggregate_throughput(ops_per_step() * e2e_steps, e0.elapsed_time(e1) * 1e-3, dev)
 
     # ---- decode-shaped sweep (rank 0, N = 1 only): the HBM-bound regime of the same path
-    decode, suites = None, None
+    decode, suites, rms_timing = None, None, None
     if info.is_main and info.world == 1 and not args.no_decode:
         del graphs, ev_graphs
         decode = decode_sweep(torch, B, dev, peaks)
@@ -533,6 +587,7 @@ def run_ours(args, info):
                                3360, 3072, 288, 1, synth.QWEN2_7B),
                   linear_suite(torch, B, dev, "config4: 8B-shaped block, 4 sequences x (2304 visual + 128 text)",
                                9728, 2304, 128, 4, synth.LLAMA_8B)]
+        rms_timing = rms_linear_timing(torch, B, dev, case.T, case.K, case.N, ROT)
 
     # ---- CPU baseline: the oracle on this host (rank 0, N = 1 only)
     cpu = None
@@ -582,6 +637,7 @@ def run_ours(args, info):
                                "frac": quant_bytes / kern["fwht_quant"] / 1e9 / peaks["hbm_gbs"]},
             "decode": decode,
             "layer_linear_suites": suites,
+            "rms_linear": rms_timing,
             "device_status": list(status),
             "cpu_baseline": cpu,
         }
