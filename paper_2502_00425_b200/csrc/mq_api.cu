@@ -200,6 +200,15 @@ int mq_w4a8_msq_linear(const mq_linear_desc* d, const void* X, int64_t ldx, cons
 
   const int8_t* qx;
   int64_t ldq;
+  if (!x_i8 && gemv_applies(d->T, d->K, d->N)) {
+    // one to four tokens: a single kernel rotates, quantizes and multiplies (mq_gemv.cu)
+    GemmArgs g{};
+    g.T = d->T; g.K = d->K; g.N = d->N;
+    g.Xb = X; g.ldx = ldx; g.rot_block = d->rot_block; g.seg = st; g.s_vis = s_vis; g.s_txt = s_txt;
+    g.W_layout = W_layout; g.s_w = s_w; g.bias = bias; g.Y = Y; g.ldy = ldy; g.y_is_f32 = y_f32 ? 1 : 0;
+    g.acc_out = acc_out;
+    return launch_gemv(g, cs);
+  }
   if (x_i8) {
     qx = static_cast<const int8_t*>(X);
     ldq = ldx;

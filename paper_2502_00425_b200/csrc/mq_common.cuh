@@ -112,6 +112,10 @@ struct GemmArgs {
   int T, K, N;
   const int8_t* Qx;
   int64_t ldq;
+  // launch_gemv only, when Qx == nullptr: bf16 activations that the kernel rotates and quantizes itself
+  const void* Xb;
+  int64_t ldx;
+  int rot_block;
   SegTable seg;
   float s_vis, s_txt;
   const void* W_layout;
@@ -134,6 +138,9 @@ struct GemmArgs {
   int32_t* acc_side_out;
 };
 int launch_gemm(const GemmArgs& a, cudaStream_t st);
+// one to four tokens: CUDA-core GEMV (mq_gemv.cu); launch_gemm routes there when it applies
+bool gemv_applies(int T, int K, int N);
+int launch_gemv(const GemmArgs& a, cudaStream_t st);
 size_t gemm_splitk_bytes(int T, int K, int N, bool rms = false);
 
 }  // namespace mq

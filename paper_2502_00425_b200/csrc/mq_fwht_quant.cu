@@ -16,25 +16,18 @@
 // sector touched is used completely; the kernel is bounded by HBM traffic of 3 bytes per
 // element (2 read + 1 written).
 #include "mq_common.cuh"
+#include "mq_fwht_warp.cuh"
 
 namespace mq {
 namespace {
 
 constexpr int kWarpsPerCta = 8;
-constexpr int kWarpTile = 1024;  // channels per warp pass
+constexpr int kWarpTile = kFwhtWarpTile;  // channels per warp pass
 
 // kQuantSide: also writes the code of the first channel of every rotation block to
 // side_out[row, block] -- the activation operand of the split product of rotation
 // magnitude suppression (Sec. 3.2), K-contiguous for the GEMM's tensor map.
 enum Mode { kQuant = 0, kQuantDump = 1, kAbsMax = 2, kQuantSide = 3 };
-
-__device__ __forceinline__ uint32_t pack_sat_s8x4(int q0, int q1, int q2, int q3) {
-  // cvt.pack.sat.s8.s32.b32 d, a, b, c : d = { c[15:0], sat8(a), sat8(b) } (b in the low byte)
-  uint32_t hi, out;
-  asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(hi) : "r"(q3), "r"(q2), "r"(0));
-  asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(out) : "r"(q1), "r"(q0), "r"(hi));
-  return out;
-}
 
 template <int LOG_TPB, bool ROT, int MODE>
 __global__ void __launch_bounds__(kWarpsPerCta * 32)
@@ -56,62 +49,7 @@ fwht_quant_kernel(const uint16_t* __restrict__ X, int T, int K, int64_t ldx, Seg
   const int blk_start = tile * kWarpTile + blk * (32 * TPB);
 
   float v[4][8];
-  const uint16_t* xrow = X + (int64_t)row * ldx;
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const int off = blk_start + (i * TPB + j) * 8;
-    uint4 w = make_uint4(0u, 0u, 0u, 0u);
-    if (off < K) w = __ldg(reinterpret_cast<const uint4*>(xrow + off));
-    const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
-#pragma unroll
-    for (int p = 0; p < 4; ++p) {
-      v[i][2 * p] = __uint_as_float(ww[p] << 16);
-      v[i][2 * p + 1] = __uint_as_float(ww[p] & 0xffff0000u);
-    }
-  }
-
-  if (ROT) {
-    // strides 1, 2, 4: inside each 8-element chunk
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-#pragma unroll
-      for (int h = 1; h < 8; h <<= 1) {
-#pragma unroll
-        for (int r = 0; r < 8; ++r) {
-          if ((r & h) == 0) {
-            const float a = v[i][r], b = v[i][r + h];
-            v[i][r] = __fadd_rn(a, b);
-            v[i][r + h] = __fsub_rn(a, b);
-          }
-        }
-      }
-    }
-    // strides 8 * 2^b for b < log2(TPB): partner lane j ^ 2^b
-#pragma unroll
-    for (int b = 0; b < LOG_TPB; ++b) {
-      const float sgn = ((j >> b) & 1) ? -1.0f : 1.0f;
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-#pragma unroll
-        for (int r = 0; r < 8; ++r) {
-          const float p = __shfl_xor_sync(0xffffffffu, v[i][r], 1 << b);
-          // lower element: own + partner; upper element: partner - own (one rounding)
-          v[i][r] = __fmaf_rn(v[i][r], sgn, p);
-        }
-      }
-    }
-    // strides 8 * TPB and 16 * TPB: across the four chunks of this lane
-#pragma unroll
-    for (int r = 0; r < 8; ++r) {
-      float a0 = v[0][r], a1 = v[1][r], a2 = v[2][r], a3 = v[3][r];
-      float b0 = __fadd_rn(a0, a1), b1 = __fsub_rn(a0, a1);
-      float b2 = __fadd_rn(a2, a3), b3 = __fsub_rn(a2, a3);
-      v[0][r] = __fmul_rn(__fadd_rn(b0, b2), c_n);
-      v[1][r] = __fmul_rn(__fadd_rn(b1, b3), c_n);
-      v[2][r] = __fmul_rn(__fsub_rn(b0, b2), c_n);
-      v[3][r] = __fmul_rn(__fsub_rn(b1, b3), c_n);
-    }
-  }
+  fwht_warp_tile<LOG_TPB, ROT>(X + (int64_t)row * ldx, K, blk_start, j, c_n, v);
 
   const int mod = warp_row_modality(seg, row);
 
@@ -138,12 +76,7 @@ fwht_quant_kernel(const uint16_t* __restrict__ X, int T, int K, int64_t ldx, Seg
       dst[0] = make_float4(v[i][0], v[i][1], v[i][2], v[i][3]);
       dst[1] = make_float4(v[i][4], v[i][5], v[i][6], v[i][7]);
     }
-    int q[8];
-#pragma unroll
-    for (int r = 0; r < 8; ++r) q[r] = __float2int_rn(__fmul_rn(v[i][r], inv));  // NaN -> 0, saturating
-    uint2 o;
-    o.x = pack_sat_s8x4(q[0], q[1], q[2], q[3]);
-    o.y = pack_sat_s8x4(q[4], q[5], q[6], q[7]);
+    const uint2 o = quant_chunk_s8(v[i], inv);
     *reinterpret_cast<uint2*>(qrow + off) = o;
     if (MODE == kQuantSide && i == 0 && j == 0)  // element 0 of the block is in chunk 0 of lane-in-block 0
       side_out[(int64_t)row * side_ld + (blk_start >> (5 + LOG_TPB))] = (int8_t)(o.x & 0xffu);

@@ -888,6 +888,7 @@ Plan make_plan(int T, int K, int N, bool rms = false) {
 
 size_t gemm_splitk_bytes(int T, int K, int N, bool rms) {
   if (T <= 0 || K <= 0 || N <= 0) return 0;
+  if (!rms && gemv_applies(T, K, N)) return 0;  // the GEMV path reduces inside its CTAs
   const Plan pl = make_plan(T, K, N, rms);
   // one [T,N] slice per K split, and one more for the split accumulator
   return pl.ksplit > 1 ? (size_t)(pl.ksplit + (rms ? 1 : 0)) * T * N * sizeof(int32_t) : 0;
@@ -896,6 +897,7 @@ size_t gemm_splitk_bytes(int T, int K, int N, bool rms) {
 int launch_gemm(const GemmArgs& a, cudaStream_t st) {
   if (a.T == 0 || a.N == 0) return MQ_OK;
   const bool rms = a.side_layout != nullptr;
+  if (!rms && gemv_applies(a.T, a.K, a.N)) return launch_gemv(a, st);  // one to four tokens: see mq_gemv.cu
   const Plan pl = make_plan(a.T, a.K, a.N, rms);
   EncodeTiledFn encode = get_encode_fn();
   if (!encode) return MQ_ERR_CUDA;

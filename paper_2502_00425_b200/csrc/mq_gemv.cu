@@ -1,0 +1,273 @@
+// K2v: the W4A8 linear for one to four tokens (single-sequence decode) as a GEMV on the
+// CUDA cores, with rotation and quantizer in the same kernel.
+//
+// Method: the same arithmetic as the quantizer + GEMM pair (Fig. 4(a), App. A.3, Eq. 2, Eq. 3):
+// codes Qx = Q_int8(FWHT(x)), acc[t,n] = sum_k Qx[t,k] q_w[n,k] in int32,
+// Y = float(acc) * (s_mod(t) * s_w[n]) (+ bias).  The paper measures its decode speed with a
+// dedicated W4A8 GEMV kernel (Sec. 4.3, decode table); this is that case.
+//
+// Why not the tensor-core kernel.  With a handful of tokens the product is one pass over the
+// int4 weights, i.e. bounded by HBM.  A tcgen05 MMA with the 128 weight channels as its rows
+// keeps the tensor pipe busy for ~112 cycles per K = 32 step however few token columns it
+// has, which caps a CTA at 8 KB of packed weights per ~450 cycles -- below the HBM rate per
+// SM.  For very few tokens the integer dot-product instruction (dp4a) needs a fraction of the
+// issue slots at the HBM rate, so the CUDA cores are enough and nothing has to be staged.
+//
+// Mapping.  A CTA owns 32 consecutive output channels (one quarter of a 128-channel layout
+// tile) and ALL of K; warp w takes the K blocks w, w + W, w + 2W, ...  A lane owns one channel:
+// its 32 codes of a K = 32 piece are one 16-byte load, and the 32 lanes of a warp read 512
+// contiguous bytes of the layout tile.  The weights of the next K block are in flight while
+// the current one is multiplied.  The int8 activation codes of the (up to four) tokens sit
+// in shared memory; every lane reads the same address (broadcast).  With bf16 input every
+// CTA rotates and quantizes the few rows for itself (the quantizer kernel's own warp routine),
+// which removes one kernel boundary -- about 2 us, as much as the weights of a 4096 x 13696
+// linear take to stream -- from every linear.  The warps' partial sums are added through
+// shared memory and the first warp runs the dequant epilogue.
+//
+// Overlap between consecutive launches.  The kernel is launched with programmatic stream
+// serialization.  Before it waits for its predecessor it asks L2 for its slice of the weights
+// (a prefetch hint only, see below), so HBM streams the next linear's weights while the current
+// one computes; it releases its own dependents only after its wait, so exactly one later
+// launch runs ahead like this, not a chain of them.  W (warps per CTA) is chosen for about 24
+// warps per SM over the launch, which leaves room for the CTAs of that next launch.
+#include <cmath>
+#include <cuda_bf16.h>
+
+#include "mq_common.cuh"
+#include "mq_fwht_warp.cuh"
+
+namespace mq {
+namespace {
+
+constexpr int kGemvMaxT = 4;
+constexpr int kGemvMaxWarps = 32;
+constexpr int kGemvWarpsPerSm = 24;
+constexpr int kGemvSmemLimit = 200 * 1024;
+
+struct GemvParams {
+  int T, K, N;
+  int kb_total;   // K blocks of 128
+  int kpad;       // kb_total * 128: row pitch of the activation codes in shared memory
+  const int8_t* Qx;   // int8 activation codes [T, K] (pitch ldq), or nullptr: quantize Xb here
+  int64_t ldq;
+  const uint16_t* Xb; // bf16 activations [T, K] (pitch ldx), used when Qx == nullptr
+  int64_t ldx;
+  int rot_block;      // 0 or the Hadamard block (power of two, 32..1024) applied to Xb
+  float inv_vis, inv_txt, c_n;  // reciprocal activation scales, 1 / sqrt(rot_block)
+  SegTable seg;
+  float s_vis, s_txt;
+  const uint8_t* W_layout;
+  const float* s_w;
+  const float* bias;
+  void* Y;
+  int64_t ldy;
+  int y_is_f32;
+  int32_t* acc_out;
+};
+
+__device__ __forceinline__ uint4 ldg_stream(const uint4* p) {
+  uint4 v;
+  // the weights are read exactly once: keep them out of L1
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(p));
+  return v;
+}
+
+// Rotates and quantizes the rows of Xb into the shared-memory code array (row pitch kpad).
+template <int LOG_TPB, bool ROT>
+__device__ __forceinline__ void stage_rows(const GemvParams& p, uint8_t* xs, int warp, int lane, int warps) {
+  constexpr int TPB = 1 << LOG_TPB;
+  const int tiles_per_row = (p.K + kFwhtWarpTile - 1) / kFwhtWarpTile;
+  const int j = lane & (TPB - 1);
+  const int blk = lane >> LOG_TPB;
+  for (int wt = warp; wt < p.T * tiles_per_row; wt += warps) {  // warp-uniform trip count
+    const int row = wt / tiles_per_row, tile = wt - row * tiles_per_row;
+    const int blk_start = tile * kFwhtWarpTile + blk * (32 * TPB);
+    float v[4][8];
+    fwht_warp_tile<LOG_TPB, ROT>(p.Xb + (int64_t)row * p.ldx, p.K, blk_start, j, p.c_n, v);
+    const float inv = thread_row_modality(p.seg, row) == MQ_VISUAL ? p.inv_vis : p.inv_txt;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int off = blk_start + (i * TPB + j) * 8;
+      if (off < p.K) *reinterpret_cast<uint2*>(xs + (size_t)row * p.kpad + off) = quant_chunk_s8(v[i], inv);
+    }
+  }
+}
+
+template <int TT>
+__global__ void __launch_bounds__(kGemvMaxWarps * 32)
+w4a8_gemv_kernel(const GemvParams p) {
+  extern __shared__ __align__(16) uint8_t smem_raw[];
+  uint4* xs = reinterpret_cast<uint4*>(smem_raw);                                  // [TT][kpad] int8
+  int32_t* red = reinterpret_cast<int32_t*>(smem_raw + (size_t)TT * p.kpad);       // [warps][TT][32]
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int warps = blockDim.x >> 5;
+  const int tn = blockIdx.x >> 2, quarter = blockIdx.x & 3;
+  const int r = quarter * 32 + lane;
+  const int n = tn * MQ_W_TILE_N + r;
+  const bool live = tn * MQ_W_TILE_N + quarter * 32 < p.N;  // false: a quarter past the last channel (whole CTA)
+  if (live) {
+    // The weights do not depend on the kernel running in front of this one: ask L2 for this CTA's
+    // whole slice now, 512 contiguous bytes per (K block, piece), so that HBM streams while that
+    // kernel finishes.  Only a hint: the loads below run after pdl_wait and go through L2, the
+    // point of coherence.  (Issuing the requests from a few CTAs for everybody was measured and
+    // is far slower: the bulk-prefetch rate of one SM is the limit then.)
+    const uint8_t* slice = p.W_layout + (size_t)tn * p.kb_total * 8192 + quarter * 512;
+    for (int c = threadIdx.x; c < p.kb_total * 4; c += blockDim.x)
+      asm volatile("cp.async.bulk.prefetch.L2.global [%0], 512;" ::"l"(slice + (size_t)c * 2048) : "memory");
+  }
+  pdl_wait();  // the activations come from the kernel launched just before
+  // Dependents may start only now: exactly one later launch is then resident ahead of its turn
+  // (prefetching its weights while this one computes), not an unbounded chain of them.
+  pdl_launch_dependents();
+  if (!live) return;
+
+  // activation codes -> shared memory, zero-padded to whole K blocks
+  const int chunks = p.kpad >> 4;
+  if (p.Qx) {
+    for (int i = threadIdx.x; i < TT * chunks; i += blockDim.x) {
+      const int t = i / chunks, c = i - t * chunks;
+      uint4 v = make_uint4(0u, 0u, 0u, 0u);
+      if (t < p.T && c * 16 < p.K) v = __ldg(reinterpret_cast<const uint4*>(p.Qx + (int64_t)t * p.ldq + c * 16));
+      xs[i] = v;
+    }
+  } else {
+    uint32_t* xs32 = reinterpret_cast<uint32_t*>(xs);
+    const int words = p.kpad >> 2;
+    // zero what the passes below do not write: channels K .. kpad of every row, and rows >= T
+    for (int t = 0; t < TT; ++t) {
+      const int first = t < p.T ? (p.K >> 2) : 0;
+      for (int c = first + threadIdx.x; c < words; c += blockDim.x) xs32[t * words + c] = 0u;
+    }
+    switch (p.rot_block) {
+#define MQ_STAGE(LOG_TPB, ROT) stage_rows<LOG_TPB, ROT>(p, reinterpret_cast<uint8_t*>(xs), warp, lane, warps); break;
+      case 0: MQ_STAGE(2, false)
+      case 32: MQ_STAGE(0, true)
+      case 64: MQ_STAGE(1, true)
+      case 128: MQ_STAGE(2, true)
+      case 256: MQ_STAGE(3, true)
+      case 512: MQ_STAGE(4, true)
+      default: MQ_STAGE(5, true)
+#undef MQ_STAGE
+    }
+  }
+  // the activations' own loads went out first: they are few and everything waits for them
+  const uint4* wsrc = reinterpret_cast<const uint4*>(p.W_layout + (size_t)tn * p.kb_total * 8192) + r;
+  uint4 wv[4], wn[4];
+  int kb = warp;
+  if (kb < p.kb_total) {
+#pragma unroll
+    for (int jj = 0; jj < 4; ++jj) wv[jj] = ldg_stream(wsrc + ((size_t)kb * 4 + jj) * 128);
+  }
+  __syncthreads();
+
+  int acc[TT];
+#pragma unroll
+  for (int t = 0; t < TT; ++t) acc[t] = 0;
+  for (; kb < p.kb_total; kb += warps) {
+    const int kb_next = kb + warps;
+    if (kb_next < p.kb_total) {
+#pragma unroll
+      for (int jj = 0; jj < 4; ++jj) wn[jj] = ldg_stream(wsrc + ((size_t)kb_next * 4 + jj) * 128);
+    }
+#pragma unroll
+    for (int jj = 0; jj < 4; ++jj) {
+      const uint32_t ww[4] = {wv[jj].x, wv[jj].y, wv[jj].z, wv[jj].w};
+#pragma unroll
+      for (int t = 0; t < TT; ++t) {
+        // the 32 codes of token t that meet this piece: two 16-byte broadcast reads
+        const uint4* xp = xs + (size_t)t * chunks + kb * 8 + jj * 2;
+        const uint4 xa = xp[0], xb = xp[1];
+        const uint32_t xw[8] = {xa.x, xa.y, xa.z, xa.w, xb.x, xb.y, xb.z, xb.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int lo = (int)((ww[i] << 4) & 0xF0F0F0F0u);  // codes k0 .. k0+3, each x16
+          const int hi = (int)(ww[i] & 0xF0F0F0F0u);         // codes k0+4 .. k0+7, each x16
+          acc[t] = __dp4a(lo, (int)xw[2 * i], acc[t]);
+          acc[t] = __dp4a(hi, (int)xw[2 * i + 1], acc[t]);
+        }
+      }
+    }
+#pragma unroll
+    for (int jj = 0; jj < 4; ++jj) wv[jj] = wn[jj];
+  }
+
+#pragma unroll
+  for (int t = 0; t < TT; ++t) red[(warp * TT + t) * 32 + lane] = acc[t];
+  __syncthreads();
+  if (warp != 0 || n >= p.N) return;
+  const float sw = p.s_w[n];
+  const float bs = p.bias ? p.bias[n] : 0.0f;
+#pragma unroll
+  for (int t = 0; t < TT; ++t) {
+    if (t >= p.T) break;
+    int a = 0;
+    for (int w = 0; w < warps; ++w) a += red[(w * TT + t) * 32 + lane];
+    a >>= 4;  // every product carried the factor 16 of the nibble placement: exact
+    if (p.acc_out) p.acc_out[(size_t)t * p.N + n] = a;
+    const float st = thread_row_modality(p.seg, t) == MQ_VISUAL ? p.s_vis : p.s_txt;
+    float y = __fmul_rn((float)a, __fmul_rn(st, sw));
+    if (p.bias) y = __fadd_rn(y, bs);
+    if (p.y_is_f32) static_cast<float*>(p.Y)[(size_t)t * p.ldy + n] = y;
+    else static_cast<__nv_bfloat16*>(p.Y)[(size_t)t * p.ldy + n] = __float2bfloat16_rn(y);
+  }
+}
+
+int gemv_sm_count() {
+  static int n = 0;
+  if (!n) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+      n = 148;
+  }
+  return n;
+}
+
+size_t gemv_smem(int T, int K, int warps) {
+  const int tt = T <= 1 ? 1 : (T <= 2 ? 2 : 4);
+  const size_t kpad = (size_t)((K + MQ_W_TILE_K - 1) / MQ_W_TILE_K) * MQ_W_TILE_K;
+  return (size_t)tt * kpad + (size_t)warps * tt * 32 * sizeof(int32_t);
+}
+
+}  // namespace
+
+bool gemv_applies(int T, int K, int N) {
+  if (T < 1 || T > kGemvMaxT || K <= 0 || N <= 0) return false;
+  return gemv_smem(T, K, kGemvMaxWarps) <= (size_t)kGemvSmemLimit;
+}
+
+int launch_gemv(const GemmArgs& a, cudaStream_t st) {
+  GemvParams p{};
+  p.T = a.T; p.K = a.K; p.N = a.N;
+  p.kb_total = (a.K + MQ_W_TILE_K - 1) / MQ_W_TILE_K;
+  p.kpad = p.kb_total * MQ_W_TILE_K;
+  p.Qx = a.Qx; p.ldq = a.ldq; p.seg = a.seg; p.s_vis = a.s_vis; p.s_txt = a.s_txt;
+  if (!a.Qx) {
+    if (!a.Xb) return MQ_ERR_INVALID_ARG;
+    p.Xb = static_cast<const uint16_t*>(a.Xb); p.ldx = a.ldx; p.rot_block = a.rot_block;
+    p.inv_vis = 1.0f / a.s_vis; p.inv_txt = 1.0f / a.s_txt;
+    p.c_n = a.rot_block ? (float)(1.0 / sqrt((double)a.rot_block)) : 1.0f;
+  }
+  p.W_layout = static_cast<const uint8_t*>(a.W_layout);
+  p.s_w = a.s_w; p.bias = a.bias; p.Y = a.Y; p.ldy = a.ldy; p.y_is_f32 = a.y_is_f32; p.acc_out = a.acc_out;
+  const int n_tn = (a.N + MQ_W_TILE_N - 1) / MQ_W_TILE_N;
+  const int ctas = n_tn * 4;
+  int warps = (gemv_sm_count() * kGemvWarpsPerSm + ctas - 1) / ctas;
+  if (warps > kGemvMaxWarps) warps = kGemvMaxWarps;
+  if (warps > p.kb_total) warps = p.kb_total;
+  if (warps < 1) warps = 1;
+  const size_t smem = gemv_smem(a.T, a.K, warps);
+  auto kernel = a.T <= 1 ? w4a8_gemv_kernel<1> : (a.T <= 2 ? w4a8_gemv_kernel<2> : w4a8_gemv_kernel<4>);
+  static bool attr_set[3] = {false, false, false};
+  const int ki = a.T <= 1 ? 0 : (a.T <= 2 ? 1 : 2);
+  if (!attr_set[ki]) {
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemvSmemLimit) != cudaSuccess)
+      return MQ_ERR_CUDA;
+    attr_set[ki] = true;
+  }
+  return cuda_status(launch_pdl(kernel, dim3(ctas), dim3(warps * 32), smem, st, p));
+}
+
+}  // namespace mq

@@ -264,6 +264,24 @@ def test_linear_edge_shapes(T_vis, T_txt, K, N, rot):
     _check_linear(c, bias=bias)
 
 
+@pytest.mark.parametrize("T_vis,T_txt,K,N,rot", [
+    (0, 1, 4096, 272, 128),    # one token, ragged last channel quarter (N % 32 = 16), 32 K blocks
+    (1, 1, 160, 144, 32),      # two tokens of different modality, K not a multiple of the K block
+    (1, 2, 1152, 528, 128),    # three tokens in the four-token variant, nine K blocks
+    (2, 2, 13696, 64, 128),    # four tokens, 107 K blocks over 32 warps, 14 warp passes per row
+    (0, 1, 32, 16, 0),         # one K piece, half a channel quarter
+    (1, 1, 2048, 96, 1024),    # the largest rotation block (a whole warp pass)
+    (0, 2, 512, 48, 64),       # rotation 64
+])
+def test_linear_gemv_shapes(T_vis, T_txt, K, N, rot):
+    # T <= 4 runs the CUDA-core GEMV (mq_gemv.cu): with bf16 input it rotates and quantizes in the
+    # same kernel, with int8 input it only multiplies; _check_linear exercises both
+    c = synth.small_linear(500 + K + N + T_vis, T_vis, T_txt, K, N, rot, calib_vis=24, calib_txt=8)
+    bias = (np.random.default_rng(2).standard_normal(N)).astype(np.float32)
+    _check_linear(c, bias=bias)
+    _check_linear(c)
+
+
 def test_linear_many_segments_without_aifs():
     # MSQ without AIFS: interleaved spans, one segment per span, boundary inside a token tile
     row_mod = synth.interleaved_modality([(0, 5), (1, 130), (0, 17), (1, 64), (0, 40), (1, 33), (0, 11)])
@@ -284,7 +302,7 @@ def test_linear_clipping_variant():
     _check_linear(c, clipping_expected=True)
 
 
-@pytest.mark.parametrize("T,K,N", [(128, 13696, 512), (8, 4096, 1024), (600, 2048, 640)])
+@pytest.mark.parametrize("T,K,N", [(128, 13696, 512), (8, 4096, 1024), (600, 2048, 640), (3, 13696, 4096)])
 def test_repeated_launches_give_identical_accumulators(T, K, N):
     """A race in the producer / expander / MMA pipeline shows as a result that changes from launch
     to launch.  Exact integer reference (int8 x int4 codes, float64 matmul is exact here), the
