@@ -162,8 +162,8 @@ def run_reference(args, info):
 # ------------------------------------------------------------------------------------------ decode sweep
 def decode_sweep(torch, B, dev, peaks, n_sets=6, reps=20):
     """Config-5-shaped decode steps: the linears of a 4096 / 13696 SwiGLU MLP (gate, up: 4096 -> 13696;
-    down: 13696 -> 4096 behind the 128-block rotation) at T = 1, 8, 32, 128 text tokens.  Each step
-    runs rotation + quantizer + W4A8 product per linear; n_sets independent copies of the int4
+    down: 13696 -> 4096 behind the 128-block rotation) at T = 1, 2, 4, 8, 32, 128 text tokens.  Each step
+    runs rotation + quantizer + W4A8 product per linear (one fused GEMV kernel up to T = 4); n_sets independent copies of the int4
     weights (84 MB each, more than four L2 sizes in all) are cycled so that the weights come from
     HBM.  Two arrangements are timed: the three linears as three calls, and gate and up stored as
     one [27392, 4096] weight (they share their input), i.e. two calls.  Reported per T:
@@ -184,7 +184,7 @@ def decode_sweep(torch, B, dev, peaks, n_sets=6, reps=20):
                 per_set.append((lay, (torch.rand(N, generator=g) * 0.01 + 0.001).to(dev)))
             weights.append(per_set)
         res = {}
-        for T in (1, 8, 32, 128):
+        for T in (1, 2, 4, 8, 32, 128):
             xs = [(torch.randn((T, K), generator=g) * 2).to(torch.bfloat16).to(dev) for K, _, _ in shapes]
             ys = [torch.empty((T, N), dtype=torch.bfloat16, device=dev) for _, N, _ in shapes]
             wss = [B.new_workspace(T, K, N, rot) for K, N, rot in shapes]

@@ -196,6 +196,13 @@ int mq_fwht_quant_i8(const void* X, int32_t T, int32_t K, int64_t ldx, const mq_
  *   acc_out  optional int32 [T,N] (leading dimension N) dump of the accumulators
  *   ws       workspace of at least mq_workspace_bytes(d) bytes, 256-byte aligned
  * T = 0 is a successful no-op.
+ * Which kernel runs is an internal choice that does not change the result: one to four
+ * rows (single-sequence decode, the case the paper times with a W4A8 GEMV kernel,
+ * Sec. 4.3) run rotation, quantizer and a CUDA-core GEMV in ONE kernel; more rows run the
+ * quantizer kernel and the tensor-core GEMM (with split-K partial sums in ws for small T).
+ * The kernels of consecutive calls on a stream overlap their prologues, and the GEMV issues
+ * L2 prefetch hints for W_layout before the preceding kernel has finished; every real read
+ * of X, W_layout and the scales is ordered after all earlier work on the stream.
  */
 int mq_w4a8_msq_linear(const mq_linear_desc* d, const void* X, int64_t ldx,
                        const mq_segments* seg, float s_vis, float s_txt, const void* W_layout,
