@@ -477,3 +477,18 @@ def quantize_act_int8_dynamic(r):
     r = np.asarray(r, dtype=np.float32)
     s = np.array([static_scale(row) for row in r], dtype=np.float32)
     return quantize_act_int8(r, s), s
+
+
+def linear_w4a8_dynamic(x, rot_block, qw, s_w, bias=None):
+    """The comparison linear with per-token dynamic activation scales (Sec. 1, Sec. 4.3: the
+    scheme whose per-token scale computation MSQ + AIFS remove): rotate, take each row's own
+    Eq. 2 scale from the rotated row, quantize with it, integer GEMM, dequantize with that
+    row's scale.  Same rounding conventions as linear_w4a8_msq."""
+    x = np.asarray(x, dtype=np.float32)
+    r = fwht_blocks(x, rot_block, np.float32)
+    qx, s_rows = quantize_act_int8_dynamic(r)
+    acc = int_gemm(qx, qw)
+    y64 = dequant(acc, s_rows, s_w, bias, np.float64)
+    y32 = dequant(acc, s_rows, s_w, bias, np.float32)
+    return {"rotated": r, "s_rows": s_rows, "qx": qx, "acc": acc, "y64": y64, "y32": y32,
+            "y_bf16": bf16_rne(y32)}

@@ -452,3 +452,31 @@ def test_dynamic_quantizer_uses_row_absmax():
     q, s = O.quantize_act_int8_dynamic(r)
     assert s.tolist() == [np.float32(2 / 127), np.float32(0.5 / 127)]
     assert q.tolist() == [[64, -127], [127, 64]]
+
+
+def test_dynamic_linear_is_scale_invariant_per_row_and_matches_msq_on_equal_scales():
+    rng = np.random.default_rng(21)
+    T, K, N, n = 6, 64, 5, 32
+    x = O.bf16_rne(rng.standard_normal((T, K)).astype(np.float32))
+    qw, s_w = O.quantize_weight_int4(rng.standard_normal((N, K)).astype(np.float32) * 0.02)
+    d = O.linear_w4a8_dynamic(x, n, qw, s_w)
+    # every row uses the whole code range: its largest code is +-127
+    assert (np.abs(d["qx"].astype(np.int32)).max(axis=1) == 127).all()
+    # scaling a row by a power of two changes its scale, not its codes, and scales its output exactly
+    x2 = x.copy()
+    x2[1] *= 4.0
+    x2[3] *= 0.125
+    d2 = O.linear_w4a8_dynamic(x2, n, qw, s_w)
+    assert np.array_equal(d2["qx"], d["qx"]) and np.array_equal(d2["acc"], d["acc"])
+    assert d2["s_rows"][1] == d["s_rows"][1] * 4 and d2["s_rows"][3] == d["s_rows"][3] * 0.125
+    assert np.array_equal(d2["y32"][1], d["y32"][1] * 4) and np.array_equal(d2["y32"][0], d["y32"][0])
+    # with a static scale equal to a row's own dynamic scale, MSQ gives that row the same result
+    for t in (0, 4):
+        m = O.linear_w4a8_msq(x[t:t + 1], np.array([1]), np.array([0]), 1.0, d["s_rows"][t], n, qw, s_w)
+        assert np.array_equal(m["qx"][0], d["qx"][t]) and np.array_equal(m["y32"][0], d["y32"][t])
+    # the error bound of Eq. 2 per row: |q s - r| <= s / 2
+    assert (np.abs(d["qx"] * d["s_rows"][:, None].astype(np.float64) - d["rotated"]) <=
+            d["s_rows"][:, None] * 0.5 * (1 + 1e-6)).all()
+    # an all-zero row stays defined
+    z = O.linear_w4a8_dynamic(np.zeros((1, K), np.float32), n, qw, s_w)
+    assert z["s_rows"][0] == 1.0 and not z["qx"].any() and not z["y32"].any()
