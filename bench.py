@@ -277,6 +277,56 @@ def rms_linear_timing(torch, B, dev, T, K, N, rot, n_sets=4, reps=10):
     return out
 
 
+# ------------------------------------------------------------------------------------------ static vs dynamic A8
+def dynamic_linear_timing(torch, B, dev, T, K, N, rot, n_sets=4, reps=10):
+    """The comparison the paper's latency table makes (Sec. 4.3): the same linear with per-token
+    dynamic activation scales (row abs-max at run time) against MSQ's static per-modality scales.
+    Both as rotation + quantizer + GEMM on the config-2 shape, CUDA-graph replays over n_sets
+    rotating copies (larger than L2 in total); also the two quantizer kernels alone."""
+    g = torch.Generator(device="cpu").manual_seed(13)
+    seg = B.Segments.from_host([T - 64, T], [1, 0], dev)
+    sets = []
+    for _ in range(n_sets):
+        x = (torch.randn((T, K), generator=g, dtype=torch.float32) * 2).to(torch.bfloat16).to(dev)
+        lay = torch.randint(0, 256, (B.mq_w4_layout_bytes(N, K),), dtype=torch.uint8, generator=g).to(dev)
+        s_w = (torch.rand(N, generator=g) * 0.01 + 0.001).to(dev)
+        y = torch.empty((T, N), dtype=torch.bfloat16, device=dev)
+        q = torch.empty((T, K), dtype=torch.int8, device=dev)
+        sr = torch.empty(T, dtype=torch.float32, device=dev)
+        sets.append((x, lay, s_w, y, q, sr, B.new_workspace(T, K, N, rot), B.new_dynamic_workspace(T, K, N, rot)))
+
+    fns = {
+        "static_linear_us": lambda s_: B.mq_w4a8_msq_linear(s_[0], seg, 0.5, 0.05, s_[1], s_[2], s_[3], s_[6], N, rot_block=rot),
+        "dynamic_linear_us": lambda s_: B.mq_w4a8_dynamic_linear(s_[0], s_[1], s_[2], s_[3], s_[7], N, rot_block=rot),
+        "static_quant_us": lambda s_: B.mq_fwht_quant_i8(s_[0], seg, 0.5, 0.05, rot, s_[4], None),
+        "dynamic_quant_us": lambda s_: B.mq_dynamic_quant_i8(s_[0], rot, s_[4], s_[5]),
+    }
+    out = {}
+    for name, fn in fns.items():
+        for s_ in sets:
+            fn(s_)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            for s_ in sets:
+                fn(s_)
+        graph.replay()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            graph.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        out[name] = e0.elapsed_time(e1) * 1e3 / (reps * n_sets)
+        del graph
+    ok = all(B.mq_last_device_status(s_[6])[0] == 0 and B.mq_last_device_status(s_[7])[0] == 0 for s_ in sets)
+    out.update({"workload": "config2 down_proj T=%d K=%d N=%d rot=%d" % (T, K, N, rot),
+                "static_speedup_linear": out["dynamic_linear_us"] / out["static_linear_us"],
+                "static_speedup_quantizer": out["dynamic_quant_us"] / out["static_quant_us"], "status_ok": ok})
+    return out
+
+
 # ------------------------------------------------------------------------------------------ layer linear suites
 def linear_suite(torch, B, dev, name, T, n_vis_per_seq, n_txt_per_seq, batch, shape, reps=5):
     """The seven W4A8 MSQ linears of one decoder block (configs 3 and 4, linear-suite mode): every
@@ -577,7 +627,7 @@ def run_ours(args, info):
     e2e_ops, _ = D.aggregate_throughput(ops_per_step() * e2e_steps, e0.elapsed_time(e1) * 1e-3, dev)
 
     # ---- decode-shaped sweep (rank 0, N = 1 only): the HBM-bound regime of the same path
-    decode, suites, rms_timing = None, None, None
+    decode, suites, rms_timing, dyn_timing = None, None, None, None
     if info.is_main and info.world == 1 and not args.no_decode:
         del graphs, ev_graphs
         decode = decode_sweep(torch, B, dev, peaks)
@@ -588,6 +638,7 @@ def run_ours(args, info):
                   linear_suite(torch, B, dev, "config4: 8B-shaped block, 4 sequences x (2304 visual + 128 text)",
                                9728, 2304, 128, 4, synth.LLAMA_8B)]
         rms_timing = rms_linear_timing(torch, B, dev, case.T, case.K, case.N, ROT)
+        dyn_timing = dynamic_linear_timing(torch, B, dev, case.T, case.K, case.N, ROT)
 
     # ---- CPU baseline: the oracle on this host (rank 0, N = 1 only)
     cpu = None
@@ -638,6 +689,7 @@ def run_ours(args, info):
             "decode": decode,
             "layer_linear_suites": suites,
             "rms_linear": rms_timing,
+            "static_vs_dynamic_a8": dyn_timing,
             "device_status": list(status),
             "cpu_baseline": cpu,
         }

@@ -312,6 +312,39 @@ int mq_w4a8_msq_linear_rms(const mq_linear_desc* d, const void* X, int64_t ldx, 
                            const float* s_w_side, const float* bias, void* Y, int64_t ldy, int32_t* acc_out,
                            int32_t* acc_side_out, void* ws, size_t ws_bytes, void* stream);
 
+/* ---- Per-token dynamic A8: the comparison scheme -----------------------------------------
+ *
+ * The activation quantization that MSQ replaces (Sec. 1; the per-token dynamic column of the
+ * latency comparison in Sec. 4.3): every token row is quantized with its own Eq. 2 scale
+ * s_t = max_k |r[t,k]| / 127 taken from the rotated row at run time.  Provided so that the
+ * static-versus-dynamic gap can be measured with otherwise identical kernels; not part of
+ * the MSQ path, no segment table, no calibration.
+ */
+
+/*
+ * Rotation (as mq_fwht_quant_i8) + per-token dynamic int8 quantizer.
+ *   X bf16 [T,K] (ldx);  Q int8 [T,K] (ldq, multiple of 16);  s_rows device float32 [T] (out):
+ *   s_rows[t] = max_k |r[t,k]| / 127 (1 for an all-zero row),
+ *   Q[t,k] = sat_int8(round_half_even(r[t,k] * (1.0f / s_rows[t]))).
+ * K <= 32768 (MQ_ERR_UNSUPPORTED beyond).  Asynchronous on `stream`.
+ */
+int mq_dynamic_quant_i8(const void* X, int32_t T, int32_t K, int64_t ldx, int32_t rot_block, int8_t* Q,
+                        int64_t ldq, float* s_rows, void* stream);
+
+/* Workspace of mq_w4a8_dynamic_linear: that of mq_w4a8_msq_linear plus T floats. */
+size_t mq_dynamic_workspace_bytes(const mq_linear_desc* d);
+
+/*
+ * The W4A8 linear with per-token dynamic activation scales:
+ *   Qx, s_rows = mq_dynamic_quant_i8(X);  acc = Qx . q_w^T;
+ *   Y[t,n] = float(acc) * (s_rows[t] * s_w[n]) (+ bias[n]), rounded to bf16 (or float32).
+ * MQ_FLAG_X_IS_INT8 is not accepted.  s_rows_out: optional device float32 [T] that receives
+ * the scales (NULL: they stay in the workspace).  Everything else as mq_w4a8_msq_linear.
+ */
+int mq_w4a8_dynamic_linear(const mq_linear_desc* d, const void* X, int64_t ldx, const void* W_layout,
+                           const float* s_w, const float* bias, void* Y, int64_t ldy, int32_t* acc_out,
+                           float* s_rows_out, void* ws, size_t ws_bytes, void* stream);
+
 /* Waits for `stream`, then returns the status word kernels left in the workspace
  * (MQ_OK or MQ_ERR_TIMEOUT) and, if site_out != NULL (host), where the wait gave up. */
 int mq_last_device_status(void* ws, void* stream, int32_t* site_out);

@@ -83,6 +83,9 @@ def load(build_if_missing: bool = False):
         "mq_rms_workspace_bytes": (sz, [descp]),
         "mq_w4a8_msq_linear_rms": (C.c_int, [descp, vp, i64, segp, f32, f32, vp, vp, vp, vp, vp, vp, i64, vp, vp,
                                              vp, sz, vp]),
+        "mq_dynamic_quant_i8": (C.c_int, [vp, i32, i32, i64, i32, vp, i64, vp, vp]),
+        "mq_dynamic_workspace_bytes": (sz, [descp]),
+        "mq_w4a8_dynamic_linear": (C.c_int, [descp, vp, i64, vp, vp, vp, vp, i64, vp, vp, vp, sz, vp]),
         "mq_last_device_status": (C.c_int, [vp, vp, C.POINTER(C.c_int32)]),
         "mq_reset_device_status": (C.c_int, [vp, vp]),
     }
@@ -98,7 +101,7 @@ EXPORTED = ["mq_version", "mq_status_string", "mq_workspace_bytes", "mq_w4_layou
             "mq_calibrate_static_scales", "mq_pack_w4", "mq_repack_w4", "mq_unpack_w4", "mq_aifs_reorder",
             "mq_attn_mask_remap", "mq_fwht_quant_i8", "mq_w4a8_msq_linear", "mq_w4a8_msq_linear_noalloc", "mq_last_device_status",
             "mq_reset_device_status", "mq_rms_side_ld", "mq_rms_detect", "mq_pack_w4_rms", "mq_rms_workspace_bytes",
-            "mq_w4a8_msq_linear_rms"]
+            "mq_w4a8_msq_linear_rms", "mq_dynamic_quant_i8", "mq_dynamic_workspace_bytes", "mq_w4a8_dynamic_linear"]
 
 
 def status_string(status: int) -> str:
@@ -309,6 +312,35 @@ def mq_w4a8_msq_linear_rms(x, seg: Segments, s_vis, s_txt, w_layout, s_w, side_l
                                          _ptr(w_layout), _ptr(s_w), _ptr(side_layout), _ptr(s_w_side), _ptr(bias),
                                          _ptr(y), _ld(y), _ptr(acc_out), _ptr(acc_side_out), _ptr(ws), ws.numel(),
                                          _stream()), "mq_w4a8_msq_linear_rms")
+
+
+def mq_dynamic_quant_i8(x, rot_block, q, s_rows):
+    """Rotation + per-token dynamic int8 quantizer (the comparison scheme): codes and one scale per row."""
+    assert x.dtype == torch.bfloat16 and q.dtype == torch.int8 and s_rows.dtype == torch.float32
+    T, K = x.shape
+    _check(load().mq_dynamic_quant_i8(_ptr(x), T, K, _ld(x), rot_block, _ptr(q), _ld(q), _ptr(s_rows), _stream()),
+           "mq_dynamic_quant_i8")
+
+
+def new_dynamic_workspace(T, K, N, rot_block=0, device="cuda") -> torch.Tensor:
+    d = mq_linear_desc(T, K, N, rot_block, 0, 0)
+    n = int(load().mq_dynamic_workspace_bytes(C.byref(d)))
+    if n == 0:
+        raise MqError(MQ_ERR_INVALID_ARG, "mq_dynamic_workspace_bytes")
+    ws = torch.empty(n, dtype=torch.uint8, device=device)
+    _check(load().mq_reset_device_status(_ptr(ws), _stream()), "mq_reset_device_status")
+    return ws
+
+
+def mq_w4a8_dynamic_linear(x, w_layout, s_w, y, ws, N, rot_block=0, bias=None, acc_out=None, s_rows_out=None):
+    """The W4A8 linear with per-token dynamic activation scales (comparison scheme, Sec. 1 / Sec. 4.3)."""
+    assert x.dtype == torch.bfloat16
+    T, K = x.shape
+    flags = MQ_FLAG_Y_IS_F32 if y.dtype == torch.float32 else 0
+    d = mq_linear_desc(T, K, N, rot_block, 0, flags)
+    _check(load().mq_w4a8_dynamic_linear(C.byref(d), _ptr(x), _ld(x), _ptr(w_layout), _ptr(s_w), _ptr(bias), _ptr(y),
+                                         _ld(y), _ptr(acc_out), _ptr(s_rows_out), _ptr(ws), ws.numel(), _stream()),
+           "mq_w4a8_dynamic_linear")
 
 
 def mq_last_device_status(ws):

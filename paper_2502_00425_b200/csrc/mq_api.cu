@@ -328,6 +328,57 @@ int mq_w4a8_msq_linear_rms(const mq_linear_desc* d, const void* X, int64_t ldx, 
   return launch_gemm(a, cs);
 }
 
+// ---- per-token dynamic A8: the comparison scheme (Sec. 1, Sec. 4.3) -----------------------
+int mq_dynamic_quant_i8(const void* X, int32_t T, int32_t K, int64_t ldx, int32_t rot_block, int8_t* Q,
+                        int64_t ldq, float* s_rows, void* stream) {
+  if (T < 0 || K <= 0 || K % 32) return MQ_ERR_INVALID_ARG;
+  if (T == 0) return MQ_OK;
+  if (!X || !Q || !s_rows || ldx < K || ldq < K) return MQ_ERR_INVALID_ARG;
+  if (!aligned16(X) || !aligned16(Q) || (ldx * 2) % 16 || ldq % 16) return MQ_ERR_ALIGNMENT;
+  const int rc = check_rot(rot_block, K);
+  if (rc != MQ_OK) return rc;
+  if (K > 32 * 1024) return MQ_ERR_UNSUPPORTED;  // one warp per 1024 channels, one CTA per row
+  return launch_dyn_quant(X, T, K, ldx, rot_block, Q, ldq, s_rows, static_cast<cudaStream_t>(stream));
+}
+
+size_t mq_dynamic_workspace_bytes(const mq_linear_desc* d) {
+  if (check_desc(d) != MQ_OK || (d->flags & MQ_FLAG_X_IS_INT8) || d->K > 32 * 1024) return 0;
+  return ws_layout(d).total + align_up((size_t)d->T * sizeof(float), 256);
+}
+
+int mq_w4a8_dynamic_linear(const mq_linear_desc* d, const void* X, int64_t ldx, const void* W_layout,
+                           const float* s_w, const float* bias, void* Y, int64_t ldy, int32_t* acc_out,
+                           float* s_rows_out, void* ws, size_t ws_bytes, void* stream) {
+  int rc = check_desc(d);
+  if (rc != MQ_OK) return rc;
+  if (d->flags & MQ_FLAG_X_IS_INT8) return MQ_ERR_INVALID_ARG;
+  if (d->K > 32 * 1024) return MQ_ERR_UNSUPPORTED;
+  if (d->T == 0) return MQ_OK;
+  if (!X || !W_layout || !s_w || !Y) return MQ_ERR_INVALID_ARG;
+  if (ldx < d->K || ldy < d->N) return MQ_ERR_INVALID_ARG;
+  if (!aligned16(X) || (ldx * 2) % 16) return MQ_ERR_ALIGNMENT;
+  if (!aligned(W_layout, 128) || !aligned16(Y) || !aligned16(s_w)) return MQ_ERR_ALIGNMENT;
+  if (!ws) return MQ_ERR_WORKSPACE;
+  if (!aligned(ws, 256)) return MQ_ERR_ALIGNMENT;
+  const WsLayout wl = ws_layout(d);
+  if (ws_bytes < wl.total + align_up((size_t)d->T * sizeof(float), 256)) return MQ_ERR_WORKSPACE;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  uint8_t* wsb = static_cast<uint8_t*>(ws);
+  int8_t* qx = reinterpret_cast<int8_t*>(wsb + wl.qx_off);
+  float* s_rows = s_rows_out ? s_rows_out : reinterpret_cast<float*>(wsb + wl.total);
+  rc = launch_dyn_quant(X, d->T, d->K, ldx, d->rot_block, qx, d->K, s_rows, cs);
+  if (rc != MQ_OK) return rc;
+  GemmArgs a{};
+  a.T = d->T; a.K = d->K; a.N = d->N;
+  a.Qx = qx; a.ldq = d->K; a.s_vis = 1.0f; a.s_txt = 1.0f; a.row_scales = s_rows;
+  a.W_layout = W_layout; a.s_w = s_w; a.bias = bias; a.Y = Y; a.ldy = ldy;
+  a.y_is_f32 = (d->flags & MQ_FLAG_Y_IS_F32) ? 1 : 0;
+  a.acc_out = acc_out;
+  a.status = reinterpret_cast<int32_t*>(wsb);
+  a.splitk_acc = wl.splitk_bytes ? reinterpret_cast<int32_t*>(wsb + wl.splitk_off) : nullptr;
+  return launch_gemm(a, cs);
+}
+
 int mq_last_device_status(void* ws, void* stream, int32_t* site_out) {
   if (!ws) return MQ_ERR_INVALID_ARG;
   int32_t host[2] = {0, 0};

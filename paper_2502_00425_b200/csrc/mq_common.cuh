@@ -84,6 +84,8 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
 int launch_fwht_quant(const void* X, int T, int K, int64_t ldx, SegTable seg, float s_vis,
                       float s_txt, int rot_block, int8_t* Q, int64_t ldq, float* rotated_out,
                       cudaStream_t st, int8_t* side_out = nullptr, int side_ld = 0);
+int launch_dyn_quant(const void* X, int T, int K, int64_t ldx, int rot_block, int8_t* Q, int64_t ldq, float* s_rows,
+                     cudaStream_t st);
 int launch_calibrate(const void* X, int T, int K, int64_t ldx, SegTable seg, int rot_block,
                      int accumulate, uint32_t* amax_state, float* s_vis_out, float* s_txt_out,
                      cudaStream_t st);
@@ -127,6 +129,7 @@ struct GemmArgs {
   int32_t* acc_out;
   int32_t* status;     // device int32[2]: status, site
   int32_t* splitk_acc; // device int32 scratch of gemm_splitk_bytes (small-T path) or nullptr
+  const float* row_scales;  // optional device float [T]: per-token activation scales (dynamic comparison path)
   // Split part of the rotation-magnitude-suppression linear (side_layout != nullptr selects it):
   // a second product on K = side_k with its own weights and scale, accumulated beside the main one
   // and added in the epilogue:  y = fl(acc * fl(s_a s_w)) + fl(acc_side * fl(s_a s_w_side)) (+ bias).

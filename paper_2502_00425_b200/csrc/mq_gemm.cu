@@ -79,6 +79,7 @@ struct KernelParams {
   int32_t* acc_out;
   int32_t* splitk_acc;
   int32_t* status;
+  const float* row_scales;  // optional [T]: per-token activation scales instead of the per-modality pair
   // split part of the rotation-magnitude-suppression linear (only read by the RMS instantiation)
   int side_kb;                 // K blocks of the split product per tile (0: none)
   int side_col;                // tensor-memory columns from an accumulator to its split accumulator
@@ -698,7 +699,8 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const __grid_cons
       __syncwarp();
       for (int j = lane; j < p.TN; j += 32) {
         const int t = t0 + j;
-        stok[j] = (t < p.T && thread_row_modality(p.seg, t) == MQ_VISUAL) ? p.s_vis : p.s_txt;
+        if (p.row_scales) stok[j] = t < p.T ? p.row_scales[t] : 0.0f;
+        else stok[j] = (t < p.T && thread_row_modality(p.seg, t) == MQ_VISUAL) ? p.s_vis : p.s_txt;
       }
       __syncwarp();
       if (!(ok = warp_all(mbar_wait(&sh->d_full[d], ph_d, sh, p.status, 8)))) break;
@@ -748,7 +750,7 @@ __global__ void splitk_finalize_kernel(const int32_t* __restrict__ acc, int kspl
                                        float s_txt, const float* __restrict__ s_w, const float* __restrict__ bias,
                                        void* Y, int64_t ldy, int y_is_f32, int32_t* __restrict__ acc_out,
                                        const int32_t* __restrict__ side_acc, const float* __restrict__ s_w_side,
-                                       int32_t* __restrict__ acc_side_out) {
+                                       int32_t* __restrict__ acc_side_out, const float* __restrict__ row_scales) {
   pdl_launch_dependents();
   pdl_wait();
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -757,7 +759,7 @@ __global__ void splitk_finalize_kernel(const int32_t* __restrict__ acc, int kspl
   int a = 0;
   for (int ks = 0; ks < ksplit; ++ks) a += acc[(size_t)ks * T * N + idx];  // one slice per K split
   if (acc_out) acc_out[idx] = a;
-  const float st = thread_row_modality(seg, t) == MQ_VISUAL ? s_vis : s_txt;
+  const float st = row_scales ? row_scales[t] : (thread_row_modality(seg, t) == MQ_VISUAL ? s_vis : s_txt);
   float y = __fmul_rn((float)a, __fmul_rn(st, s_w[n]));
   if (side_acc) {
     const int sa = side_acc[idx];
@@ -945,7 +947,7 @@ int launch_gemm(const GemmArgs& a, cudaStream_t st) {
   p.seg = a.seg; p.s_vis = a.s_vis; p.s_txt = a.s_txt;
   p.W_layout = static_cast<const uint8_t*>(a.W_layout);
   p.s_w = a.s_w; p.bias = a.bias; p.Y = a.Y; p.ldy = a.ldy; p.y_is_f32 = a.y_is_f32;
-  p.acc_out = a.acc_out; p.splitk_acc = a.splitk_acc; p.status = a.status;
+  p.acc_out = a.acc_out; p.splitk_acc = a.splitk_acc; p.status = a.status; p.row_scales = a.row_scales;
   int32_t* side_slice = nullptr;
   if (rms) {
     p.side_kb = (a.side_k + kBlockK - 1) / kBlockK;
@@ -965,7 +967,7 @@ int launch_gemm(const GemmArgs& a, cudaStream_t st) {
     if (launch_pdl(splitk_finalize_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), 0, st,
                    static_cast<const int32_t*>(a.splitk_acc), pl.ksplit, a.T, a.N, a.seg, a.s_vis, a.s_txt, a.s_w, a.bias, a.Y,
                    a.ldy, a.y_is_f32, a.acc_out, static_cast<const int32_t*>(side_slice), a.s_w_side,
-                   a.acc_side_out) != cudaSuccess)
+                   a.acc_side_out, a.row_scales) != cudaSuccess)
       return MQ_ERR_CUDA;
   }
   return MQ_OK;

@@ -63,6 +63,7 @@ struct GemvParams {
   int64_t ldy;
   int y_is_f32;
   int32_t* acc_out;
+  const float* row_scales;  // optional [T]: per-token activation scales (int8 input only)
 };
 
 __device__ __forceinline__ uint4 ldg_stream(const uint4* p) {
@@ -206,7 +207,8 @@ w4a8_gemv_kernel(const GemvParams p) {
     for (int w = 0; w < warps; ++w) a += red[(w * TT + t) * 32 + lane];
     a >>= 4;  // every product carried the factor 16 of the nibble placement: exact
     if (p.acc_out) p.acc_out[(size_t)t * p.N + n] = a;
-    const float st = thread_row_modality(p.seg, t) == MQ_VISUAL ? p.s_vis : p.s_txt;
+    const float st = p.row_scales ? p.row_scales[t]
+                                  : (thread_row_modality(p.seg, t) == MQ_VISUAL ? p.s_vis : p.s_txt);
     float y = __fmul_rn((float)a, __fmul_rn(st, sw));
     if (p.bias) y = __fadd_rn(y, bs);
     if (p.y_is_f32) static_cast<float*>(p.Y)[(size_t)t * p.ldy + n] = y;
@@ -252,6 +254,7 @@ int launch_gemv(const GemmArgs& a, cudaStream_t st) {
   }
   p.W_layout = static_cast<const uint8_t*>(a.W_layout);
   p.s_w = a.s_w; p.bias = a.bias; p.Y = a.Y; p.ldy = a.ldy; p.y_is_f32 = a.y_is_f32; p.acc_out = a.acc_out;
+  p.row_scales = a.row_scales;
   const int n_tn = (a.N + MQ_W_TILE_N - 1) / MQ_W_TILE_N;
   const int ctas = n_tn * 4;
   int warps = (gemv_sm_count() * kGemvWarpsPerSm + ctas - 1) / ctas;

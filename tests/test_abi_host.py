@@ -160,6 +160,27 @@ def test_rms_entry_points_validate(lib):
              None) == B.MQ_ERR_WORKSPACE
 
 
+def test_dynamic_entry_points_validate(lib):
+    A = 0x10000
+    base = B.mq_workspace_bytes(1088, 18944, 3584, 128)
+    d = _desc(1088, 18944, 3584, rot=128)
+    assert lib.mq_dynamic_workspace_bytes(C.byref(d)) == base + 4352       # + 1088 floats
+    assert lib.mq_dynamic_workspace_bytes(C.byref(_desc(8, 65536, 128))) == 0   # rows longer than 32768
+    q = lib.mq_dynamic_quant_i8
+    assert q(A, 4, 100, 100, 0, A, 112, A, None) == B.MQ_ERR_INVALID_ARG
+    assert q(A, 4, 128, 128, 0, A, 128, None, None) == B.MQ_ERR_INVALID_ARG
+    assert q(A, 4, 128, 128, 0, A + 1, 128, A, None) == B.MQ_ERR_ALIGNMENT
+    assert q(A, 4, 65536, 65536, 0, A, 65536, A, None) == B.MQ_ERR_UNSUPPORTED
+    assert q(A, 4, 128, 128, 48, A, 128, A, None) == B.MQ_ERR_INVALID_ARG
+    f = lib.mq_w4a8_dynamic_linear
+    d = _desc(8, 256, 128, flags=B.MQ_FLAG_X_IS_INT8)
+    assert f(C.byref(d), A, 256, A, A, None, A, 128, None, None, A, 1 << 30, None) == B.MQ_ERR_INVALID_ARG
+    d = _desc(8, 256, 128)
+    assert f(C.byref(d), A, 256, A, A, None, A, 128, None, None, None, 0, None) == B.MQ_ERR_WORKSPACE
+    assert f(C.byref(d), A, 256, A, A, None, A, 128, None, None, A, B.mq_workspace_bytes(8, 256, 128), None) == B.MQ_ERR_WORKSPACE
+    assert f(C.byref(d), A, 200, A, A, None, A, 128, None, None, A, 1 << 30, None) == B.MQ_ERR_INVALID_ARG
+
+
 def test_binding_refuses_cpu_tensors():
     import torch
     with pytest.raises(ValueError):
