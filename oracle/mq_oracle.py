@@ -492,3 +492,32 @@ def linear_w4a8_dynamic(x, rot_block, qw, s_w, bias=None):
     y32 = dequant(acc, s_rows, s_w, bias, np.float32)
     return {"rotated": r, "s_rows": s_rows, "qx": qx, "acc": acc, "y64": y64, "y32": y32,
             "y_bf16": bf16_rne(y32)}
+
+
+# ----------------------------------------------------------------------------- glue of a decoder block (checker only)
+def rmsnorm(x, gain, eps: float = 1e-6) -> np.ndarray:
+    """RMSNorm (App. A.14: x / sqrt(||x||^2 / d + eps)), times the per-channel gain; float64."""
+    x = np.asarray(x, dtype=np.float64)
+    ms = np.mean(x * x, axis=-1, keepdims=True)
+    return x / np.sqrt(ms + eps) * np.asarray(gain, dtype=np.float64)
+
+
+def swiglu(gate, up) -> np.ndarray:
+    """SiLU(gate) * up, the activation in front of the down-projection; float64."""
+    gate = np.asarray(gate, dtype=np.float64)
+    return gate / (1.0 + np.exp(-gate)) * np.asarray(up, dtype=np.float64)
+
+
+def gqa_attention(q, k, v, allowed, n_q_heads: int, n_kv_heads: int) -> np.ndarray:
+    """Grouped-query attention: q [L, n_q_heads*D], k, v [L, n_kv_heads*D]; query head h reads
+    key/value head h // (n_q_heads / n_kv_heads); every head is attention() above."""
+    q = np.asarray(q, dtype=np.float64)
+    L = q.shape[0]
+    D = q.shape[1] // n_q_heads
+    group = n_q_heads // n_kv_heads
+    out = np.empty_like(q)
+    for h in range(n_q_heads):
+        g = h // group
+        out[:, h * D:(h + 1) * D] = attention(q[:, h * D:(h + 1) * D], np.asarray(k)[:, g * D:(g + 1) * D],
+                                              np.asarray(v)[:, g * D:(g + 1) * D], allowed)
+    return out

@@ -480,3 +480,29 @@ def test_dynamic_linear_is_scale_invariant_per_row_and_matches_msq_on_equal_scal
     # an all-zero row stays defined
     z = O.linear_w4a8_dynamic(np.zeros((1, K), np.float32), n, qw, s_w)
     assert z["s_rows"][0] == 1.0 and not z["qx"].any() and not z["y32"].any()
+
+
+def test_block_glue_against_hand_values():
+    # RMSNorm: unit gain gives unit mean square; a constant row maps to +-1 (up to eps)
+    x = np.array([[3.0, -3.0, 3.0, -3.0], [1.0, 2.0, 3.0, 4.0]])
+    y = O.rmsnorm(x, np.ones(4), eps=0.0)
+    assert np.allclose(y[0], [1, -1, 1, -1]) and np.allclose((y * y).mean(axis=1), 1.0)
+    assert np.allclose(O.rmsnorm(x, [2, 2, 2, 2], eps=0.0), 2 * y)
+    assert np.allclose(y[1], x[1] / np.sqrt(7.5))
+    # SwiGLU: silu(0) = 0, silu(x) -> x for large x, silu(-x) = x sigmoid(-x)
+    assert O.swiglu([0.0], [5.0])[0] == 0.0
+    assert np.isclose(O.swiglu([30.0], [2.0])[0], 60.0)
+    assert np.isclose(O.swiglu([1.0], [1.0])[0], 1.0 / (1.0 + np.exp(-1.0)))
+    # grouped-query attention: with one kv head per query head it is per-head attention;
+    # with a shared kv head, two query heads given the same q produce the same output
+    rng = np.random.default_rng(4)
+    L, D = 5, 4
+    q, k, v = rng.standard_normal((L, 2 * D)), rng.standard_normal((L, 2 * D)), rng.standard_normal((L, 2 * D))
+    allowed = O.causal_mask(L)
+    full = O.gqa_attention(q, k, v, allowed, 2, 2)
+    assert np.allclose(full[:, D:], O.attention(q[:, D:], k[:, D:], v[:, D:], allowed))
+    q2 = np.concatenate([q[:, :D], q[:, :D]], axis=1)
+    shared = O.gqa_attention(q2, k[:, :D], v[:, :D], allowed, 2, 1)
+    assert np.allclose(shared[:, :D], shared[:, D:]) and np.allclose(shared[:, :D], full[:, :D])
+    # first row attends only to itself
+    assert np.allclose(full[0, :D], v[0, :D])
