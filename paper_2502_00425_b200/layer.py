@@ -1,0 +1,167 @@
+"""Layer mode: one decoder block whose seven linears are the W4A8 MSQ linear of this library.
+
+The linears, the AIFS reorder and the mask / position remap run through the C ABI (the
+product).  Everything between them -- RMSNorm, rotary embedding, masked grouped-query
+attention, SwiGLU, the residual adds -- is plain torch on the same device: glue that lets a
+sequence flow through a whole block (Sec. 3.1: AIFS once at the input, the unified mask and the
+remapped positions in attention, MSQ in front of every linear, the online Hadamard in front of
+the down-projection, Fig. 4(a)).  The glue is not tuned and not part of the measured kernels.
+
+A block works on ONE sequence in its original token order and returns the output in that
+order; `forward` keeps every linear's input and output so that a checker can recompute each
+step from the tensor the GPU actually fed it.
+"""
+from dataclasses import dataclass, field
+from typing import Dict, List, Optional, Tuple
+
+import torch
+
+from . import binding as B
+from .synth import LayerShape
+
+
+@dataclass
+class LinearWeights:
+    layout: torch.Tensor          # GEMM weight layout (uint8)
+    s_w: torch.Tensor             # float32 [N]
+    K: int
+    N: int
+    rot_block: int = 0
+    bias: Optional[torch.Tensor] = None
+    s_vis: float = 1.0            # static activation scales of this linear's input (Eq. 3)
+    s_txt: float = 1.0
+
+
+@dataclass
+class BlockTrace:
+    """What one forward pass saw: tensors in AIFS order unless the name says otherwise."""
+    perm: torch.Tensor = None
+    pos_u: torch.Tensor = None
+    seg: B.Segments = None
+    mask: torch.Tensor = None
+    tensors: Dict[str, torch.Tensor] = field(default_factory=dict)
+
+
+def rmsnorm(x: torch.Tensor, gain: torch.Tensor, eps: float = 1e-6) -> torch.Tensor:
+    xf = x.float()
+    return (xf * torch.rsqrt(xf.pow(2).mean(-1, keepdim=True) + eps) * gain.float()).to(torch.bfloat16)
+
+
+def rope(x: torch.Tensor, pos: torch.Tensor, n_heads: int, base: float = 10000.0) -> torch.Tensor:
+    """Rotary embedding on consecutive channel pairs of every head (App. A.2), positions `pos`."""
+    L, width = x.shape
+    D = width // n_heads
+    xf = x.float().view(L, n_heads, D // 2, 2)
+    theta = base ** (-2.0 * torch.arange(D // 2, device=x.device, dtype=torch.float64) / D)
+    ang = pos.to(torch.float64)[:, None] * theta[None, :]
+    c, s = torch.cos(ang).float()[:, None, :], torch.sin(ang).float()[:, None, :]
+    out = torch.stack((xf[..., 0] * c - xf[..., 1] * s, xf[..., 0] * s + xf[..., 1] * c), dim=-1)
+    return out.view(L, width).to(torch.bfloat16)
+
+
+def gqa_attention(q, k, v, mask, n_q_heads: int, n_kv_heads: int) -> torch.Tensor:
+    L = q.shape[0]
+    D = q.shape[1] // n_q_heads
+    group = n_q_heads // n_kv_heads
+    qh = q.view(L, n_q_heads, D).transpose(0, 1)
+    kh = k.view(L, n_kv_heads, D).transpose(0, 1).repeat_interleave(group, dim=0)
+    vh = v.view(L, n_kv_heads, D).transpose(0, 1).repeat_interleave(group, dim=0)
+    o = torch.nn.functional.scaled_dot_product_attention(qh[None], kh[None], vh[None], attn_mask=mask[None, None])
+    return o[0].transpose(0, 1).reshape(L, n_q_heads * D).contiguous()
+
+
+class W4A8DecoderBlock:
+    """One decoder block over the library's linears.  `weights` maps the seven linear names of
+    LayerShape.linears() to LinearWeights; `g_attn`, `g_mlp` are the RMSNorm gains."""
+
+    def __init__(self, shape: LayerShape, weights: Dict[str, LinearWeights], g_attn: torch.Tensor,
+                 g_mlp: torch.Tensor, device="cuda"):
+        self.shape, self.w, self.g_attn, self.g_mlp, self.device = shape, weights, g_attn, g_mlp, device
+        self._ws: Dict[Tuple[str, int], torch.Tensor] = {}
+
+    # ---- pieces ------------------------------------------------------------------------
+    def aifs(self, emb: torch.Tensor, is_visual: torch.Tensor, tr: BlockTrace) -> torch.Tensor:
+        """AIFS reorder of the sequence plus the remapped positions, segment table and mask."""
+        L = emb.shape[0]
+        dev = emb.device
+        emb_u = torch.empty_like(emb)
+        perm = torch.empty(L, dtype=torch.int32, device=dev)
+        inv = torch.empty(L, dtype=torch.int32, device=dev)
+        n_first = torch.zeros(1, dtype=torch.int32, device=dev)
+        B.mq_aifs_reorder(emb, emb_u, is_visual, None, perm, inv, n_first, direction=0)
+        pos_u = torch.empty(L, dtype=torch.int32, device=dev)
+        seg_end = torch.empty(2, dtype=torch.int32, device=dev)
+        seg_mod = torch.empty(2, dtype=torch.uint8, device=dev)
+        mask = torch.empty((L, L), dtype=torch.uint8, device=dev)
+        B.mq_attn_mask_remap(perm, None, None, n_first, pos_u, seg_end, seg_mod, mask)
+        tr.perm, tr.pos_u, tr.seg, tr.mask = perm, pos_u, B.Segments(seg_end, seg_mod), mask.bool()
+        return emb_u
+
+    def linear(self, name: str, x: torch.Tensor, tr: BlockTrace, calibrate: bool) -> torch.Tensor:
+        lw = self.w[name]
+        T = x.shape[0]
+        if calibrate:
+            state = torch.zeros(2, dtype=torch.int32, device=x.device)
+            sv = torch.zeros(1, dtype=torch.float32, device=x.device)
+            st = torch.zeros(1, dtype=torch.float32, device=x.device)
+            B.mq_calibrate_static_scales(x, tr.seg, lw.rot_block, state, sv, st)
+            lw.s_vis, lw.s_txt = float(sv.item()), float(st.item())
+        key = (name, T)
+        if key not in self._ws:
+            self._ws[key] = B.new_workspace(T, lw.K, lw.N, lw.rot_block)
+        y = torch.empty((T, lw.N), dtype=torch.bfloat16, device=x.device)
+        B.mq_w4a8_msq_linear(x, tr.seg, lw.s_vis, lw.s_txt, lw.layout, lw.s_w, y, self._ws[key], lw.N,
+                             rot_block=lw.rot_block, bias=lw.bias)
+        tr.tensors[name + ".in"], tr.tensors[name + ".out"] = x, y
+        return y
+
+    # ---- the block ---------------------------------------------------------------------
+    def forward(self, emb: torch.Tensor, is_visual: torch.Tensor, calibrate: bool = False):
+        """emb: bf16 [L, hidden] in the original token order; is_visual: uint8 [L].
+        calibrate=True first sets every linear's static scales from this very sequence (single-shot
+        calibration, Algorithm 1) and then runs with them.  Returns (output in the original
+        order, BlockTrace)."""
+        sh, tr = self.shape, BlockTrace()
+        x0 = self.aifs(emb, is_visual, tr)
+        t = tr.tensors
+        t["emb_u"] = x0
+        h = rmsnorm(x0, self.g_attn)
+        t["attn_norm"] = h
+        q = self.linear("q_proj", h, tr, calibrate)
+        k = self.linear("k_proj", h, tr, calibrate)
+        v = self.linear("v_proj", h, tr, calibrate)
+        qr = rope(q, tr.pos_u, sh.n_q_heads)
+        kr = rope(k, tr.pos_u, sh.n_kv_heads)
+        t["q_rope"], t["k_rope"] = qr, kr
+        a = gqa_attention(qr, kr, v, tr.mask, sh.n_q_heads, sh.n_kv_heads)
+        t["attn"] = a
+        o = self.linear("o_proj", a, tr, calibrate)
+        x1 = (x0.float() + o.float()).to(torch.bfloat16)
+        t["resid1"] = x1
+        h2 = rmsnorm(x1, self.g_mlp)
+        t["mlp_norm"] = h2
+        gate = self.linear("gate_proj", h2, tr, calibrate)
+        up = self.linear("up_proj", h2, tr, calibrate)
+        act = (torch.nn.functional.silu(gate.float()) * up.float()).to(torch.bfloat16)
+        t["act"] = act
+        down = self.linear("down_proj", act, tr, calibrate)
+        x2 = (x1.float() + down.float()).to(torch.bfloat16)
+        t["resid2"] = x2
+        out = torch.empty_like(x2)
+        B.mq_aifs_reorder(x2, out, None, None, tr.perm, None, None, direction=1)
+        return out, tr
+
+    def device_status_ok(self) -> bool:
+        return all(B.mq_last_device_status(ws)[0] == B.MQ_OK for ws in self._ws.values())
+
+
+def random_block(shape: LayerShape, seed: int, device="cuda") -> W4A8DecoderBlock:
+    """A block with random valid weight bytes and scales: for timing only (no float weights exist)."""
+    g = torch.Generator(device="cpu").manual_seed(seed)
+    w = {}
+    for name, K, N, rot in shape.linears():
+        lay = torch.randint(0, 256, (B.mq_w4_layout_bytes(N, K),), dtype=torch.uint8, generator=g).to(device)
+        s_w = (torch.rand(N, generator=g) * 0.002 + 0.0005).to(device)
+        w[name] = LinearWeights(lay, s_w, K, N, rot)
+    ones = torch.ones(shape.hidden, device=device)
+    return W4A8DecoderBlock(shape, w, ones, ones.clone(), device)

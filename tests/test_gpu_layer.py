@@ -1,0 +1,112 @@
+"""Layer mode: a whole decoder block over the library's linears, checked step by step against the
+oracle with "teacher forcing" -- every step is recomputed on the CPU from the tensor the GPU
+actually fed it, so the integer paths stay bit-exact per linear and the float glue (plain torch)
+is compared at 2e-2 relative to the row maximum."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import mq_oracle as O
+from paper_2502_00425_b200 import binding as B
+from paper_2502_00425_b200 import layer as LY
+from paper_2502_00425_b200 import synth
+from tests.gpu_util import DEV, bf16_from_dev, bf16_to_dev, gpu_pack
+
+pytestmark = pytest.mark.gpu
+
+GLUE_TOL = 2e-2
+
+
+def _close_rowmax(got, ref, tol=GLUE_TOL):
+    ref = np.asarray(ref, dtype=np.float64)
+    scale = np.abs(ref).max(axis=-1, keepdims=True)
+    scale = np.where(scale > 0, scale, 1.0)
+    return (np.abs(np.asarray(got, dtype=np.float64) - ref) / scale).max() <= tol
+
+
+def _make_block(shape, seed):
+    rng = np.random.default_rng(seed)
+    weights, ref_w = {}, {}
+    for name, K, N, rot in shape.linears():
+        w = (rng.standard_normal((N, K)) * (1.0 / np.sqrt(K))).astype(np.float32)
+        if rot:
+            w = O.rotate_weight_input_dim(w, rot).astype(np.float32)   # offline counterpart of the online rotation
+        packed, s_w, layout = gpu_pack(w)
+        weights[name] = LY.LinearWeights(layout, s_w, K, N, rot)
+        ref_w[name] = O.quantize_weight_int4(w)
+    g1 = (1.0 + 0.1 * rng.standard_normal(shape.hidden)).astype(np.float32)
+    g2 = (1.0 + 0.1 * rng.standard_normal(shape.hidden)).astype(np.float32)
+    blk = LY.W4A8DecoderBlock(shape, weights, torch.from_numpy(g1).to(DEV), torch.from_numpy(g2).to(DEV), DEV)
+    return blk, ref_w, g1, g2
+
+
+def _check_block(shape, is_visual, seed, rows=None):
+    L = is_visual.shape[0]
+    blk, ref_w, g1, g2 = _make_block(shape, seed)
+    emb = synth.embedding_rows(seed + 1, L, shape.hidden, is_visual)
+    out, tr = blk.forward(bf16_to_dev(emb), torch.from_numpy(is_visual).to(DEV), calibrate=True)
+    assert blk.device_status_ok()
+    t = {k: bf16_from_dev(v) for k, v in tr.tensors.items()}
+    # AIFS, positions, mask
+    perm = O.aifs_perm(is_visual)
+    assert np.array_equal(tr.perm.cpu().numpy(), perm)
+    assert np.array_equal(tr.pos_u.cpu().numpy(), O.remap_positions(perm))
+    allowed = O.unified_mask(perm)
+    assert np.array_equal(tr.mask.cpu().numpy(), allowed)
+    assert np.array_equal(t["emb_u"], O.aifs_gather(emb, perm))
+    seg_end, seg_mod = O.segments_after_aifs(perm, is_visual)
+    assert np.array_equal(tr.seg.seg_end.cpu().numpy(), seg_end)
+    # every linear from the GPU's own input: scales, then the bf16 output, bit-exact
+    sel = np.arange(L) if rows is None else rows
+    for name, K, N, rot in shape.linears():
+        x_in = t[name + ".in"]
+        s_v, s_t = O.calibrate_static_scales(x_in, seg_end, seg_mod, rot)
+        lw = blk.w[name]
+        assert (np.float32(lw.s_vis), np.float32(lw.s_txt)) == (s_v, s_t), name
+        qw, s_w = ref_w[name]
+        sub_end = np.searchsorted(sel, seg_end).astype(np.int32)      # segment table of the sampled rows
+        ref = O.linear_w4a8_msq(x_in[sel], sub_end, seg_mod, s_v, s_t, rot, qw, s_w)
+        assert np.array_equal(t[name + ".out"][sel], ref["y_bf16"]), name
+    # glue, each from the GPU's inputs
+    assert _close_rowmax(t["attn_norm"], O.rmsnorm(t["emb_u"], g1))
+    pos = O.remap_positions(perm)
+    D = shape.head_dim
+    for nm, src, heads in (("q_rope", "q_proj.out", shape.n_q_heads), ("k_rope", "k_proj.out", shape.n_kv_heads)):
+        ref = np.concatenate([O.rope(t[src][:, h * D:(h + 1) * D], pos) for h in range(heads)], axis=1)
+        assert _close_rowmax(t[nm], ref), nm
+    ref_attn = O.gqa_attention(t["q_rope"], t["k_rope"], t["v_proj.out"], allowed, shape.n_q_heads, shape.n_kv_heads)
+    assert _close_rowmax(t["attn"], ref_attn)
+    assert _close_rowmax(t["resid1"], t["emb_u"].astype(np.float64) + t["o_proj.out"])
+    assert _close_rowmax(t["mlp_norm"], O.rmsnorm(t["resid1"], g2))
+    assert _close_rowmax(t["act"], O.swiglu(t["gate_proj.out"], t["up_proj.out"]))
+    assert _close_rowmax(t["resid2"], t["resid1"].astype(np.float64) + t["down_proj.out"])
+    # back to the original order, exactly
+    assert np.array_equal(bf16_from_dev(out), O.aifs_scatter(t["resid2"], perm))
+    # a second pass with the stored scales reproduces the first one bit for bit
+    out2, _ = blk.forward(bf16_to_dev(emb), torch.from_numpy(is_visual).to(DEV))
+    assert torch.equal(out2, out)
+    return blk
+
+
+def test_small_block_interleaved_modalities():
+    shape = synth.LayerShape(hidden=256, n_q_heads=4, n_kv_heads=2, head_dim=64, mlp=512)
+    is_visual = synth.interleaved_modality([(0, 7), (1, 90), (0, 20), (1, 50), (0, 33)])
+    _check_block(shape, is_visual, seed=31)
+
+
+def test_small_block_text_only_and_visual_only():
+    shape = synth.LayerShape(hidden=128, n_q_heads=2, n_kv_heads=1, head_dim=64, mlp=256)
+    _check_block(shape, np.zeros(37, np.uint8), seed=32)
+    _check_block(shape, np.ones(45, np.uint8), seed=33)
+
+
+def test_config3_block_full_size_sampled():
+    """The Qwen2-7B-shaped block of config 3 at full size (L = 3360); the linears are checked on
+    every 64th row and the rows next to the modality boundary, attention on two heads' worth of
+    the glue tolerance like everything else."""
+    shape = synth.QWEN2_7B
+    is_visual = synth.config3_sequence()
+    L = is_visual.shape[0]
+    n_vis = int(is_visual.sum())
+    rows = np.unique(np.concatenate([np.arange(0, L, 64), np.arange(n_vis - 2, n_vis + 2), [L - 1]]))
+    _check_block(shape, is_visual, seed=34, rows=rows)
