@@ -327,6 +327,35 @@ def dynamic_linear_timing(torch, B, dev, T, K, N, rot, n_sets=4, reps=10):
     return out
 
 
+# ------------------------------------------------------------------------------------------ layer mode
+def layer_mode_timing(torch, dev, name, shape, seqs, reps=5):
+    """Configs 3 and 4 as a whole decoder block (layer mode): AIFS, mask / position remap and the
+    seven W4A8 MSQ linears through the C ABI, with the glue between them (RMSNorm, rotary
+    embedding, masked grouped-query attention, SwiGLU, residuals) in plain, untuned torch.  Random
+    valid weight bytes, fixed scales: timing only (parity of the block is covered by the tests).
+    Reports tokens per second for the whole block and how much of the time the glue takes."""
+    from paper_2502_00425_b200 import layer as LY
+    blk = LY.random_block(shape, 21, dev)
+    for lw in blk.w.values():
+        lw.s_vis, lw.s_txt = 0.5, 0.05
+    g = torch.Generator(device="cpu").manual_seed(22)
+    embs = [(torch.randn((len(s_), shape.hidden), generator=g) * 2).to(torch.bfloat16).to(dev) for s_ in seqs]
+    vis = [torch.from_numpy(s_).to(dev) for s_ in seqs]
+    tokens = sum(len(s_) for s_ in seqs)
+    blk.forward_batch(embs, vis)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        blk.forward_batch(embs, vis)
+    e1.record()
+    torch.cuda.synchronize()
+    sec = e0.elapsed_time(e1) * 1e-3 / reps
+    return {"workload": name, "tokens": tokens, "us_per_block": sec * 1e6, "tokens_per_s": tokens / sec,
+            "glue": "torch (untuned): RMSNorm, RoPE, masked GQA attention, SwiGLU, residuals", "launch": "eager",
+            "status_ok": blk.device_status_ok()}
+
+
 # ------------------------------------------------------------------------------------------ layer linear suites
 def linear_suite(torch, B, dev, name, T, n_vis_per_seq, n_txt_per_seq, batch, shape, reps=5):
     """The seven W4A8 MSQ linears of one decoder block (configs 3 and 4, linear-suite mode): every
@@ -627,7 +656,7 @@ def run_ours(args, info):
     e2e_ops, _ = D.aggregate_throughput(ops_per_step() * e2e_steps, e0.elapsed_time(e1) * 1e-3, dev)
 
     # ---- decode-shaped sweep (rank 0, N = 1 only): the HBM-bound regime of the same path
-    decode, suites, rms_timing, dyn_timing = None, None, None, None
+    decode, suites, rms_timing, dyn_timing, layers = None, None, None, None, None
     if info.is_main and info.world == 1 and not args.no_decode:
         del graphs, ev_graphs
         decode = decode_sweep(torch, B, dev, peaks)
@@ -639,6 +668,11 @@ def run_ours(args, info):
                                9728, 2304, 128, 4, synth.LLAMA_8B)]
         rms_timing = rms_linear_timing(torch, B, dev, case.T, case.K, case.N, ROT)
         dyn_timing = dynamic_linear_timing(torch, B, dev, case.T, case.K, case.N, ROT)
+        torch.cuda.empty_cache()
+        layers = [layer_mode_timing(torch, dev, "config3: Qwen2-7B-shaped block, one sequence of 3360 tokens",
+                                    synth.QWEN2_7B, [synth.config3_sequence()]),
+                  layer_mode_timing(torch, dev, "config4: 8B-shaped block, 4 sequences of 2432 tokens",
+                                    synth.LLAMA_8B, [synth.config4_sequence()] * 4)]
 
     # ---- CPU baseline: the oracle on this host (rank 0, N = 1 only)
     cpu = None
@@ -690,6 +724,7 @@ def run_ours(args, info):
             "layer_linear_suites": suites,
             "rms_linear": rms_timing,
             "static_vs_dynamic_a8": dyn_timing,
+            "layer_mode": layers,
             "device_status": list(status),
             "cpu_baseline": cpu,
         }

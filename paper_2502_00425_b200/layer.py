@@ -7,9 +7,11 @@ sequence flow through a whole block (Sec. 3.1: AIFS once at the input, the unifi
 remapped positions in attention, MSQ in front of every linear, the online Hadamard in front of
 the down-projection, Fig. 4(a)).  The glue is not tuned and not part of the measured kernels.
 
-A block works on ONE sequence in its original token order and returns the output in that
-order; `forward` keeps every linear's input and output so that a checker can recompute each
-step from the tensor the GPU actually fed it.
+A block takes one sequence, or a batch of sequences, in the original token order and returns
+the outputs in that order.  Every sequence is reordered on its own; the linears then see the
+rows of all sequences stacked (two segments per sequence in the segment table), attention
+runs per sequence.  `forward` keeps every linear's input and output so that a checker can
+recompute each step from the tensor the GPU actually fed it.
 """
 from dataclasses import dataclass, field
 from typing import Dict, List, Optional, Tuple
@@ -35,10 +37,14 @@ class LinearWeights:
 @dataclass
 class BlockTrace:
     """What one forward pass saw: tensors in AIFS order unless the name says otherwise."""
-    perm: torch.Tensor = None
+    perm: torch.Tensor = None      # of the first (or only) sequence; all of them in `perms`
     pos_u: torch.Tensor = None
-    seg: B.Segments = None
+    seg: B.Segments = None         # over the stacked rows
     mask: torch.Tensor = None
+    perms: List[torch.Tensor] = field(default_factory=list)
+    pos_us: List[torch.Tensor] = field(default_factory=list)
+    masks: List[torch.Tensor] = field(default_factory=list)
+    bounds: List[int] = field(default_factory=list)   # row offsets of the sequences in the stacked tensors
     tensors: Dict[str, torch.Tensor] = field(default_factory=dict)
 
 
@@ -80,22 +86,35 @@ class W4A8DecoderBlock:
         self._ws: Dict[Tuple[str, int], torch.Tensor] = {}
 
     # ---- pieces ------------------------------------------------------------------------
-    def aifs(self, emb: torch.Tensor, is_visual: torch.Tensor, tr: BlockTrace) -> torch.Tensor:
-        """AIFS reorder of the sequence plus the remapped positions, segment table and mask."""
-        L = emb.shape[0]
-        dev = emb.device
-        emb_u = torch.empty_like(emb)
-        perm = torch.empty(L, dtype=torch.int32, device=dev)
-        inv = torch.empty(L, dtype=torch.int32, device=dev)
-        n_first = torch.zeros(1, dtype=torch.int32, device=dev)
-        B.mq_aifs_reorder(emb, emb_u, is_visual, None, perm, inv, n_first, direction=0)
-        pos_u = torch.empty(L, dtype=torch.int32, device=dev)
-        seg_end = torch.empty(2, dtype=torch.int32, device=dev)
-        seg_mod = torch.empty(2, dtype=torch.uint8, device=dev)
-        mask = torch.empty((L, L), dtype=torch.uint8, device=dev)
-        B.mq_attn_mask_remap(perm, None, None, n_first, pos_u, seg_end, seg_mod, mask)
-        tr.perm, tr.pos_u, tr.seg, tr.mask = perm, pos_u, B.Segments(seg_end, seg_mod), mask.bool()
-        return emb_u
+    def aifs(self, embs, is_visuals, tr: BlockTrace) -> torch.Tensor:
+        """AIFS reorder of every sequence plus its remapped positions and mask; returns the stacked
+        rows and leaves the segment table over them in the trace."""
+        dev = embs[0].device
+        parts, ends, mods, off = [], [], [], 0
+        tr.bounds = [0]
+        for emb, is_visual in zip(embs, is_visuals):
+            L = emb.shape[0]
+            emb_u = torch.empty_like(emb)
+            perm = torch.empty(L, dtype=torch.int32, device=dev)
+            inv = torch.empty(L, dtype=torch.int32, device=dev)
+            n_first = torch.zeros(1, dtype=torch.int32, device=dev)
+            B.mq_aifs_reorder(emb, emb_u, is_visual, None, perm, inv, n_first, direction=0)
+            pos_u = torch.empty(L, dtype=torch.int32, device=dev)
+            seg_end = torch.empty(2, dtype=torch.int32, device=dev)
+            seg_mod = torch.empty(2, dtype=torch.uint8, device=dev)
+            mask = torch.empty((L, L), dtype=torch.uint8, device=dev)
+            B.mq_attn_mask_remap(perm, None, None, n_first, pos_u, seg_end, seg_mod, mask)
+            parts.append(emb_u)
+            ends.append(seg_end + off)
+            mods.append(seg_mod)
+            tr.perms.append(perm)
+            tr.pos_us.append(pos_u)
+            tr.masks.append(mask.bool())
+            off += L
+            tr.bounds.append(off)
+        tr.perm, tr.pos_u, tr.mask = tr.perms[0], tr.pos_us[0], tr.masks[0]
+        tr.seg = B.Segments(torch.cat(ends), torch.cat(mods))
+        return parts[0] if len(parts) == 1 else torch.cat(parts, dim=0)
 
     def linear(self, name: str, x: torch.Tensor, tr: BlockTrace, calibrate: bool) -> torch.Tensor:
         lw = self.w[name]
@@ -118,22 +137,29 @@ class W4A8DecoderBlock:
     # ---- the block ---------------------------------------------------------------------
     def forward(self, emb: torch.Tensor, is_visual: torch.Tensor, calibrate: bool = False):
         """emb: bf16 [L, hidden] in the original token order; is_visual: uint8 [L].
-        calibrate=True first sets every linear's static scales from this very sequence (single-shot
+        calibrate=True first sets every linear's static scales from this very input (single-shot
         calibration, Algorithm 1) and then runs with them.  Returns (output in the original
         order, BlockTrace)."""
+        outs, tr = self.forward_batch([emb], [is_visual], calibrate)
+        return outs[0], tr
+
+    def forward_batch(self, embs, is_visuals, calibrate: bool = False):
+        """Several sequences at once: lists of bf16 [L_b, hidden] and uint8 [L_b]."""
         sh, tr = self.shape, BlockTrace()
-        x0 = self.aifs(emb, is_visual, tr)
-        t = tr.tensors
+        x0 = self.aifs(embs, is_visuals, tr)
+        t, bd = tr.tensors, tr.bounds
+        n_seq = len(embs)
         t["emb_u"] = x0
         h = rmsnorm(x0, self.g_attn)
         t["attn_norm"] = h
         q = self.linear("q_proj", h, tr, calibrate)
         k = self.linear("k_proj", h, tr, calibrate)
         v = self.linear("v_proj", h, tr, calibrate)
-        qr = rope(q, tr.pos_u, sh.n_q_heads)
-        kr = rope(k, tr.pos_u, sh.n_kv_heads)
+        qr = torch.cat([rope(q[bd[b]:bd[b + 1]], tr.pos_us[b], sh.n_q_heads) for b in range(n_seq)])
+        kr = torch.cat([rope(k[bd[b]:bd[b + 1]], tr.pos_us[b], sh.n_kv_heads) for b in range(n_seq)])
         t["q_rope"], t["k_rope"] = qr, kr
-        a = gqa_attention(qr, kr, v, tr.mask, sh.n_q_heads, sh.n_kv_heads)
+        a = torch.cat([gqa_attention(qr[bd[b]:bd[b + 1]], kr[bd[b]:bd[b + 1]], v[bd[b]:bd[b + 1]], tr.masks[b],
+                                     sh.n_q_heads, sh.n_kv_heads) for b in range(n_seq)])
         t["attn"] = a
         o = self.linear("o_proj", a, tr, calibrate)
         x1 = (x0.float() + o.float()).to(torch.bfloat16)
@@ -147,9 +173,12 @@ class W4A8DecoderBlock:
         down = self.linear("down_proj", act, tr, calibrate)
         x2 = (x1.float() + down.float()).to(torch.bfloat16)
         t["resid2"] = x2
-        out = torch.empty_like(x2)
-        B.mq_aifs_reorder(x2, out, None, None, tr.perm, None, None, direction=1)
-        return out, tr
+        outs = []
+        for b in range(n_seq):
+            out = torch.empty((bd[b + 1] - bd[b], x2.shape[1]), dtype=torch.bfloat16, device=x2.device)
+            B.mq_aifs_reorder(x2[bd[b]:bd[b + 1]], out, None, None, tr.perms[b], None, None, direction=1)
+            outs.append(out)
+        return outs, tr
 
     def device_status_ok(self) -> bool:
         return all(B.mq_last_device_status(ws)[0] == B.MQ_OK for ws in self._ws.values())
