@@ -83,7 +83,10 @@ __device__ __forceinline__ void stage_rows(const GemvParams& p, uint8_t* xs, int
   const int j = lane & (TPB - 1);
   const int blk = lane >> LOG_TPB;
   for (int wt = warp; wt < p.T * tiles_per_row; wt += warps) {  // warp-uniform trip count
-    const int row = wt / tiles_per_row, tile = wt - row * tiles_per_row;
+    // every CTA stages the same rows: start each CTA at a different tile so that the CTAs of the
+    // launch do not all ask L2 for the same lines at the same moment
+    const int row = wt / tiles_per_row;
+    const int tile = (wt - row * tiles_per_row + (int)blockIdx.x) % tiles_per_row;
     const int blk_start = tile * kFwhtWarpTile + blk * (32 * TPB);
     float v[4][8];
     fwht_warp_tile<LOG_TPB, ROT>(p.Xb + (int64_t)row * p.ldx, p.K, blk_start, j, p.c_n, v);
@@ -155,30 +158,34 @@ w4a8_gemv_kernel(const GemvParams p) {
   }
   // the activations' own loads went out first: they are few and everything waits for them
   const uint4* wsrc = reinterpret_cast<const uint4*>(p.W_layout + (size_t)tn * p.kb_total * 8192) + r;
-  uint4 wv[4], wn[4];
+  // One token: two K blocks of this warp are in flight at any time (buffers A and B are refilled
+  // as soon as they have been multiplied).  More tokens: the multiplication of a block is long
+  // enough to cover one load, and the second buffer is fetched while the first is multiplied
+  // (measured: the deeper scheme costs registers there and is slower).
+  constexpr bool kTwoInFlight = TT == 1;
+  uint4 wa[4], wb[4];
   int kb = warp;
-  if (kb < p.kb_total) {
+  auto fetch = [&](uint4 (&dst)[4], int k) {
+    if (k < p.kb_total) {
 #pragma unroll
-    for (int jj = 0; jj < 4; ++jj) wv[jj] = ldg_stream(wsrc + ((size_t)kb * 4 + jj) * 128);
-  }
+      for (int jj = 0; jj < 4; ++jj) dst[jj] = ldg_stream(wsrc + ((size_t)k * 4 + jj) * 128);
+    }
+  };
+  fetch(wa, kb);
+  if (kTwoInFlight) fetch(wb, kb + warps);
   __syncthreads();
 
   int acc[TT];
 #pragma unroll
   for (int t = 0; t < TT; ++t) acc[t] = 0;
-  for (; kb < p.kb_total; kb += warps) {
-    const int kb_next = kb + warps;
-    if (kb_next < p.kb_total) {
-#pragma unroll
-      for (int jj = 0; jj < 4; ++jj) wn[jj] = ldg_stream(wsrc + ((size_t)kb_next * 4 + jj) * 128);
-    }
+  auto multiply = [&](const uint4 (&w)[4], int k) {
 #pragma unroll
     for (int jj = 0; jj < 4; ++jj) {
-      const uint32_t ww[4] = {wv[jj].x, wv[jj].y, wv[jj].z, wv[jj].w};
+      const uint32_t ww[4] = {w[jj].x, w[jj].y, w[jj].z, w[jj].w};
 #pragma unroll
       for (int t = 0; t < TT; ++t) {
         // the 32 codes of token t that meet this piece: two 16-byte broadcast reads
-        const uint4* xp = xs + (size_t)t * chunks + kb * 8 + jj * 2;
+        const uint4* xp = xs + (size_t)t * chunks + k * 8 + jj * 2;
         const uint4 xa = xp[0], xb = xp[1];
         const uint32_t xw[8] = {xa.x, xa.y, xa.z, xa.w, xb.x, xb.y, xb.z, xb.w};
 #pragma unroll
@@ -190,8 +197,23 @@ w4a8_gemv_kernel(const GemvParams p) {
         }
       }
     }
+  };
+  if (kTwoInFlight) {
+    for (; kb < p.kb_total; kb += 2 * warps) {
+      multiply(wa, kb);
+      fetch(wa, kb + 2 * warps);
+      if (kb + warps < p.kb_total) {
+        multiply(wb, kb + warps);
+        fetch(wb, kb + 3 * warps);
+      }
+    }
+  } else {
+    for (; kb < p.kb_total; kb += warps) {
+      fetch(wb, kb + warps);
+      multiply(wa, kb);
 #pragma unroll
-    for (int jj = 0; jj < 4; ++jj) wv[jj] = wn[jj];
+      for (int jj = 0; jj < 4; ++jj) wa[jj] = wb[jj];
+    }
   }
 
 #pragma unroll
