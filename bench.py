@@ -362,7 +362,8 @@ def linear_suite(torch, B, dev, name, T, n_vis_per_seq, n_txt_per_seq, batch, sh
     linear gets its own synthetic activations in AIFS order and runs rotation (down_proj only) +
     quantizer + GEMM through mq_w4a8_msq_linear.  Weight layouts and scales are random valid bytes
     (timing only; parity of these shapes is covered by the tests).  Reports microseconds per
-    linear and TOPS over the seven."""
+    linear (the linear repeated back to back) and TOPS over the seven in sequence, both as
+    CUDA-graph replays."""
     g = torch.Generator(device="cpu").manual_seed(11)
     seg_end, seg_mod, e = [], [], 0
     for _ in range(batch):
@@ -388,25 +389,27 @@ def linear_suite(torch, B, dev, name, T, n_vis_per_seq, n_txt_per_seq, batch, sh
         lname, K, N, rot, x, lay, s_w, y, ws = it
         B.mq_w4a8_msq_linear(x, seg, 0.5, 0.05, lay, s_w, y, ws, N, rot_block=rot)
 
-    per = {}
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    for it in items:
-        run(it)
-    torch.cuda.synchronize()
-    for it in items:
+    def timed_graph(body, reps_in_graph):
+        """Microseconds per execution of body(), replayed from a CUDA graph (launch cost off the clock)."""
+        body()
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            for _ in range(reps_in_graph):
+                body()
+        graph.replay()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
-        for _ in range(reps):
-            run(it)
+        for _ in range(3):
+            graph.replay()
         e1.record()
         torch.cuda.synchronize()
-        per[it[0]] = e0.elapsed_time(e1) * 1e3 / reps
-    e0.record()
-    for _ in range(reps):
-        for it in items:
-            run(it)
-    e1.record()
-    torch.cuda.synchronize()
-    sec = e0.elapsed_time(e1) * 1e-3 / reps
+        del graph
+        return e0.elapsed_time(e1) * 1e3 / (3 * reps_in_graph)
+
+    per = {it[0]: timed_graph(lambda it=it: run(it), reps) for it in items}
+    sec = timed_graph(lambda: [run(it) for it in items], reps) * 1e-6
     ok = all(B.mq_last_device_status(it[8])[0] == 0 for it in items)
     return {"workload": name, "T": T, "us_per_linear": per, "us_all_seven": sec * 1e6, "tops": total_ops / sec / 1e12,
             "tokens_per_s": T / sec, "status_ok": ok}

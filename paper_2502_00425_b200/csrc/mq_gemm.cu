@@ -822,12 +822,17 @@ Plan make_plan(int T, int K, int N, bool rms = false) {
   const int tn_cap = rms ? 224 : 256;
   int n_tt = (T + tn_cap - 1) / tn_cap;
   int TN = (((T + n_tt - 1) / n_tt) + 15) / 16 * 16;
-  if ((long long)pl.n_tn * n_tt > sms) {  // several tiles per CTA; otherwise the fewest tiles are right
+  // The search runs when a CTA gets several tiles, and when every CTA gets one tile of more than
+  // 192 tokens although smaller tiles would still fit the machine in one round (their MMAs are
+  // cheaper); otherwise the fewest tiles are right.
+  const bool multi_round = (long long)pl.n_tn * n_tt > sms;
+  if (multi_round || TN > 192) {
     double best = 0.0;
     const int n_min = n_tt;
     for (int cand = n_min; cand <= n_min * 4 && cand <= (T + 15) / 16; ++cand) {
       const int tn = (((T + cand - 1) / cand) + 15) / 16 * 16;
       const long long tiles_c = (long long)pl.n_tn * cand;
+      if (!multi_round && tiles_c > sms) break;  // stay within one round
       const long long rounds = (tiles_c + sms - 1) / sms;
       const double mma = tn <= 192 ? 112.0 : (tn <= 224 ? 112.0 + (tn - 192) * 0.25 : 120.0 + (tn - 224) * 0.5);
       const double epi = 25.0 * tn;
@@ -863,6 +868,13 @@ Plan make_plan(int T, int K, int N, bool rms = false) {
     if (ksplit < 1) ksplit = 1;
     const int per = (kb_total + ksplit - 1) / ksplit;
     ksplit = (kb_total + per - 1) / per;  // no empty split
+    // Splitting pays only while the partial sums are small: each split writes a [T,N] int32 slice
+    // that the finalize kernel reads back (about 4 TB/s for the pair), and that kernel costs
+    // about 3 us on top.  Against it stands the main loop, 4 MMAs of ~112 cycles per K block at
+    // ~1.9 GHz.  (Decode shapes split; a prefill-sized T with few output channels does not.)
+    const double loop_us = kb_total * 4.0 * 112.0 / 1900.0;
+    const double slices_us = (ksplit + 0.5) * (double)T * N * 4.0 * 2.0 / 4.0e6 + 3.0;
+    if (loop_us / ksplit + slices_us >= loop_us) ksplit = 1;
   }
   pl.ksplit = ksplit;
   // shared memory: as many activation stages as fit beside a minimum of 4 weight stages, then
