@@ -134,6 +134,36 @@ class W4A8DecoderBlock:
         tr.tensors[name + ".in"], tr.tensors[name + ".out"] = x, y
         return y
 
+    def linear_group(self, names, x: torch.Tensor, tr: BlockTrace, calibrate: bool):
+        """Linears that read the same input (q/k/v, gate/up; no rotation): the input is quantized
+        once with mq_fwht_quant_i8 and every linear of the group multiplies the same int8 codes."""
+        first = self.w[names[0]]
+        assert all(self.w[n].rot_block == 0 and self.w[n].K == first.K for n in names)
+        T = x.shape[0]
+        if calibrate:
+            state = torch.zeros(2, dtype=torch.int32, device=x.device)
+            sv = torch.zeros(1, dtype=torch.float32, device=x.device)
+            st = torch.zeros(1, dtype=torch.float32, device=x.device)
+            B.mq_calibrate_static_scales(x, tr.seg, 0, state, sv, st)
+            for n in names:
+                self.w[n].s_vis, self.w[n].s_txt = float(sv.item()), float(st.item())
+        if T <= 4:  # the few-token kernel quantizes inside: nothing to share
+            return [self.linear(n, x, tr, False) for n in names]
+        codes = torch.empty((T, first.K), dtype=torch.int8, device=x.device)
+        B.mq_fwht_quant_i8(x, tr.seg, first.s_vis, first.s_txt, 0, codes, None)
+        outs = []
+        for n in names:
+            lw = self.w[n]
+            key = (n + ".i8", T)
+            if key not in self._ws:
+                self._ws[key] = B.new_workspace(T, lw.K, lw.N, 0, B.MQ_FLAG_X_IS_INT8)
+            y = torch.empty((T, lw.N), dtype=torch.bfloat16, device=x.device)
+            B.mq_w4a8_msq_linear(codes, tr.seg, lw.s_vis, lw.s_txt, lw.layout, lw.s_w, y, self._ws[key], lw.N,
+                                 bias=lw.bias)
+            tr.tensors[n + ".in"], tr.tensors[n + ".out"] = x, y
+            outs.append(y)
+        return outs
+
     # ---- the block ---------------------------------------------------------------------
     def forward(self, emb: torch.Tensor, is_visual: torch.Tensor, calibrate: bool = False):
         """emb: bf16 [L, hidden] in the original token order; is_visual: uint8 [L].
@@ -152,9 +182,7 @@ class W4A8DecoderBlock:
         t["emb_u"] = x0
         h = rmsnorm(x0, self.g_attn)
         t["attn_norm"] = h
-        q = self.linear("q_proj", h, tr, calibrate)
-        k = self.linear("k_proj", h, tr, calibrate)
-        v = self.linear("v_proj", h, tr, calibrate)
+        q, k, v = self.linear_group(["q_proj", "k_proj", "v_proj"], h, tr, calibrate)
         qr = torch.cat([rope(q[bd[b]:bd[b + 1]], tr.pos_us[b], sh.n_q_heads) for b in range(n_seq)])
         kr = torch.cat([rope(k[bd[b]:bd[b + 1]], tr.pos_us[b], sh.n_kv_heads) for b in range(n_seq)])
         t["q_rope"], t["k_rope"] = qr, kr
@@ -166,8 +194,7 @@ class W4A8DecoderBlock:
         t["resid1"] = x1
         h2 = rmsnorm(x1, self.g_mlp)
         t["mlp_norm"] = h2
-        gate = self.linear("gate_proj", h2, tr, calibrate)
-        up = self.linear("up_proj", h2, tr, calibrate)
+        gate, up = self.linear_group(["gate_proj", "up_proj"], h2, tr, calibrate)
         act = (torch.nn.functional.silu(gate.float()) * up.float()).to(torch.bfloat16)
         t["act"] = act
         down = self.linear("down_proj", act, tr, calibrate)
