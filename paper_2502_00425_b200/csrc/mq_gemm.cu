@@ -836,7 +836,9 @@ Plan make_plan(int T, int K, int N, bool rms = false) {
       const long long rounds = (tiles_c + sms - 1) / sms;
       const double mma = tn <= 192 ? 112.0 : (tn <= 224 ? 112.0 + (tn - 192) * 0.25 : 120.0 + (tn - 224) * 0.5);
       const double epi = 25.0 * tn;
-      const bool two_acc = !rms && tn <= 192;
+      // two accumulators: always up to 192 tokens; up to 224 tokens (448 columns, which leaves two
+      // weight slots) when a CTA runs several tiles and the hidden epilogue is worth the shallower ring
+      const bool two_acc = !rms && (tn <= 192 || (tn <= 224 && rounds > 1));
       const double main_loop = 4.0 * mma * kb_total;
       const double est = two_acc ? rounds * main_loop + epi : rounds * (main_loop + epi);
       if (cand == n_min || est < best * 0.995) {
@@ -848,8 +850,9 @@ Plan make_plan(int T, int K, int N, bool rms = false) {
   }
   pl.TN = TN;
   pl.n_tt = n_tt;
-  pl.d_stride = TN <= 128 ? 128 : (TN <= 192 ? 192 : 256);
-  pl.num_d = pl.d_stride <= 192 ? 2 : 1;
+  const bool several_tiles = (long long)pl.n_tn * n_tt > sms;
+  pl.d_stride = TN <= 128 ? 128 : (TN <= 192 ? 192 : ((TN <= 224 && several_tiles) ? 224 : 256));
+  pl.num_d = pl.d_stride <= 224 ? 2 : 1;
   pl.a_base = pl.num_d * pl.d_stride;
   if (rms) {
     pl.d_stride = (TN + 31) / 32 * 32;  // here: columns from the accumulator to its split accumulator
