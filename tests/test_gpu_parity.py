@@ -282,6 +282,24 @@ def test_linear_gemv_shapes(T_vis, T_txt, K, N, rot):
     _check_linear(c)
 
 
+@pytest.mark.parametrize("T_vis,T_txt,K,N,rot", [
+    (0, 1, 131040, 16, 32),    # the largest K the 16x accumulators allow, one token: GEMV with 1024 K blocks
+    (2, 2, 131040, 16, 0),     # four tokens: too long for the GEMV's shared memory, quantizer + split-K GEMM instead
+    (5, 4, 131040, 32, 32),    # nine tokens at the largest K
+])
+def test_linear_maximum_k(T_vis, T_txt, K, N, rot):
+    c = synth.small_linear(900 + T_vis + T_txt, T_vis, T_txt, K, N, rot, calib_vis=4, calib_txt=4)
+    _check_linear(c)
+
+
+def test_linear_sixty_four_segments():
+    # a batch of 32 short sequences after per-sequence AIFS: 64 alternating segments in one call
+    row_mod = synth.interleaved_modality([(1, 5), (0, 3)] * 32)
+    c = synth.heavy_tail_linear("many_segments", 78, 0, 0, 256, 64, 64, calib_vis=8, calib_txt=8, row_mod=row_mod)
+    assert c.seg.n_seg == 64
+    _check_linear(c)
+
+
 def test_linear_many_segments_without_aifs():
     # MSQ without AIFS: interleaved spans, one segment per span, boundary inside a token tile
     row_mod = synth.interleaved_modality([(0, 5), (1, 130), (0, 17), (1, 64), (0, 40), (1, 33), (0, 11)])
