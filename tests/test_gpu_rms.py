@@ -79,6 +79,8 @@ def test_rms_pack_matches_oracle(N, K, rot):
     (3, 5, 4096, 256, 128, True),      # T = 8: the small-T GEMM path underneath, 32 blocks
     (150, 60, 160, 144, 32, True),     # five blocks of 32, two token tiles of the main GEMM
     (0, 9, 2048, 64, 1024, False),     # two blocks of 1024
+    (0, 1, 1152, 272, 128, True),      # one token: the split path keeps the tensor-core kernel (no GEMV variant)
+    (1, 2, 13696, 144, 128, False),    # three tokens at the decode row length, split-K with the split accumulator's slice
     (300, 33, 2304, 528, 128, True),   # 18 blocks, five channel tiles, two token tiles
 ])
 def test_rms_linear_matches_oracle(T_vis, T_txt, K, N, rot, with_bias):
