@@ -308,6 +308,17 @@ int mq_w4a8_msq_linear_rms(const mq_linear_desc* d, const void* X, int64_t ldx, 
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
   uint8_t* wsb = static_cast<uint8_t*>(ws);
   const int sk = rms_side_k(d->K, d->rot_block);
+  if (gemv_applies(d->T, d->K, d->N, sk)) {
+    // one to four tokens: rotation, quantizer, both products and the epilogue in one GEMV kernel
+    GemmArgs g{};
+    g.T = d->T; g.K = d->K; g.N = d->N;
+    g.Xb = X; g.ldx = ldx; g.rot_block = d->rot_block; g.seg = st; g.s_vis = s_vis; g.s_txt = s_txt;
+    g.W_layout = W_layout; g.s_w = s_w; g.bias = bias; g.Y = Y; g.ldy = ldy;
+    g.y_is_f32 = (d->flags & MQ_FLAG_Y_IS_F32) ? 1 : 0;
+    g.acc_out = acc_out;
+    g.side_k = sk; g.side_layout = side_layout; g.s_w_side = s_w_side; g.acc_side_out = acc_side_out;
+    return launch_gemv(g, cs);
+  }
   int8_t* qx = reinterpret_cast<int8_t*>(wsb + wl.qx_off);
   int8_t* xs = reinterpret_cast<int8_t*>(wsb + wl.xs_off);
 

@@ -64,6 +64,14 @@ struct GemvParams {
   int y_is_f32;
   int32_t* acc_out;
   const float* row_scales;  // optional [T]: per-token activation scales (int8 input only)
+  // split part of the rotation-magnitude-suppression linear (Sec. 3.2), bf16 input only: the codes of
+  // the first channel of every rotation block times side_kb extra weight tiles per channel tile,
+  // with their own scale, added before the bias
+  const uint8_t* side_layout;  // nullptr: none
+  const float* s_w_side;
+  int side_kb;                 // K blocks (of 128 split codes) per channel tile
+  int side_cols;               // K / rot_block: split codes per row
+  int32_t* acc_side_out;
 };
 
 __device__ __forceinline__ uint4 ldg_stream(const uint4* p) {
@@ -97,6 +105,22 @@ __device__ __forceinline__ void stage_rows(const GemvParams& p, uint8_t* xs, int
       if (off < p.K) *reinterpret_cast<uint2*>(xs + (size_t)row * p.kpad + off) = quant_chunk_s8(v[i], inv);
     }
   }
+}
+
+// One 16-byte piece of packed weights (32 codes of this lane's channel) against the 32 activation
+// codes at xp (two 16-byte broadcast reads) of one token.
+__device__ __forceinline__ int dot_piece(const uint4& w, const uint4* xp, int acc) {
+  const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+  const uint4 xa = xp[0], xb = xp[1];
+  const uint32_t xw[8] = {xa.x, xa.y, xa.z, xa.w, xb.x, xb.y, xb.z, xb.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int lo = (int)((ww[i] << 4) & 0xF0F0F0F0u);  // codes k0 .. k0+3, each x16
+    const int hi = (int)(ww[i] & 0xF0F0F0F0u);         // codes k0+4 .. k0+7, each x16
+    acc = __dp4a(lo, (int)xw[2 * i], acc);
+    acc = __dp4a(hi, (int)xw[2 * i + 1], acc);
+  }
+  return acc;
 }
 
 template <int TT>
@@ -181,21 +205,8 @@ w4a8_gemv_kernel(const GemvParams p) {
   auto multiply = [&](const uint4 (&w)[4], int k) {
 #pragma unroll
     for (int jj = 0; jj < 4; ++jj) {
-      const uint32_t ww[4] = {w[jj].x, w[jj].y, w[jj].z, w[jj].w};
 #pragma unroll
-      for (int t = 0; t < TT; ++t) {
-        // the 32 codes of token t that meet this piece: two 16-byte broadcast reads
-        const uint4* xp = xs + (size_t)t * chunks + k * 8 + jj * 2;
-        const uint4 xa = xp[0], xb = xp[1];
-        const uint32_t xw[8] = {xa.x, xa.y, xa.z, xa.w, xb.x, xb.y, xb.z, xb.w};
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const int lo = (int)((ww[i] << 4) & 0xF0F0F0F0u);  // codes k0 .. k0+3, each x16
-          const int hi = (int)(ww[i] & 0xF0F0F0F0u);         // codes k0+4 .. k0+7, each x16
-          acc[t] = __dp4a(lo, (int)xw[2 * i], acc[t]);
-          acc[t] = __dp4a(hi, (int)xw[2 * i + 1], acc[t]);
-        }
-      }
+      for (int t = 0; t < TT; ++t) acc[t] = dot_piece(w[jj], xs + (size_t)t * chunks + k * 8 + jj * 2, acc[t]);
     }
   };
   if (kTwoInFlight) {
@@ -218,8 +229,34 @@ w4a8_gemv_kernel(const GemvParams p) {
 
 #pragma unroll
   for (int t = 0; t < TT; ++t) red[(warp * TT + t) * 32 + lane] = acc[t];
+  // split part: its activation codes are those at the first channel of every rotation block;
+  // gather them side by side (zero-padded to whole K blocks) behind the partial sums
+  uint4* xside = reinterpret_cast<uint4*>(red + warps * TT * 32);
+  const int side_pad = p.side_kb * MQ_W_TILE_K;
+  if (p.side_layout) {
+    const int8_t* xb8 = reinterpret_cast<const int8_t*>(xs);
+    int8_t* dst = reinterpret_cast<int8_t*>(xside);
+    for (int i = threadIdx.x; i < TT * side_pad; i += blockDim.x) {
+      const int t = i / side_pad, b = i - t * side_pad;
+      dst[i] = b < p.side_cols ? xb8[(size_t)t * p.kpad + (size_t)b * p.rot_block] : (int8_t)0;
+    }
+  }
   __syncthreads();
   if (warp != 0 || n >= p.N) return;
+  int acc_s[TT];
+#pragma unroll
+  for (int t = 0; t < TT; ++t) acc_s[t] = 0;
+  float sws = 0.0f;
+  if (p.side_layout) {
+    // a few hundred multiply-adds per channel: the first warp does them on its way out
+    const uint4* ssrc = reinterpret_cast<const uint4*>(p.side_layout + (size_t)tn * p.side_kb * 8192) + r;
+    for (int c = 0; c < p.side_kb * 4; ++c) {
+      const uint4 w = ldg_stream(ssrc + (size_t)c * 128);
+#pragma unroll
+      for (int t = 0; t < TT; ++t) acc_s[t] = dot_piece(w, xside + (size_t)t * (side_pad >> 4) + c * 2, acc_s[t]);
+    }
+    sws = p.s_w_side[n];
+  }
   const float sw = p.s_w[n];
   const float bs = p.bias ? p.bias[n] : 0.0f;
 #pragma unroll
@@ -232,6 +269,11 @@ w4a8_gemv_kernel(const GemvParams p) {
     const float st = p.row_scales ? p.row_scales[t]
                                   : (thread_row_modality(p.seg, t) == MQ_VISUAL ? p.s_vis : p.s_txt);
     float y = __fmul_rn((float)a, __fmul_rn(st, sw));
+    if (p.side_layout) {
+      const int as = acc_s[t] >> 4;
+      if (p.acc_side_out) p.acc_side_out[(size_t)t * p.N + n] = as;
+      y = __fadd_rn(y, __fmul_rn((float)as, __fmul_rn(st, sws)));
+    }
     if (p.bias) y = __fadd_rn(y, bs);
     if (p.y_is_f32) static_cast<float*>(p.Y)[(size_t)t * p.ldy + n] = y;
     else static_cast<__nv_bfloat16*>(p.Y)[(size_t)t * p.ldy + n] = __float2bfloat16_rn(y);
@@ -249,17 +291,18 @@ int gemv_sm_count() {
   return n;
 }
 
-size_t gemv_smem(int T, int K, int warps) {
+size_t gemv_smem(int T, int K, int warps, int side_k = 0) {
   const int tt = T <= 1 ? 1 : (T <= 2 ? 2 : 4);
   const size_t kpad = (size_t)((K + MQ_W_TILE_K - 1) / MQ_W_TILE_K) * MQ_W_TILE_K;
-  return (size_t)tt * kpad + (size_t)warps * tt * 32 * sizeof(int32_t);
+  const size_t side_pad = (size_t)((side_k + MQ_W_TILE_K - 1) / MQ_W_TILE_K) * MQ_W_TILE_K;
+  return (size_t)tt * kpad + (size_t)warps * tt * 32 * sizeof(int32_t) + (size_t)tt * side_pad;
 }
 
 }  // namespace
 
-bool gemv_applies(int T, int K, int N) {
+bool gemv_applies(int T, int K, int N, int side_k) {
   if (T < 1 || T > kGemvMaxT || K <= 0 || N <= 0) return false;
-  return gemv_smem(T, K, kGemvMaxWarps) <= (size_t)kGemvSmemLimit;
+  return gemv_smem(T, K, kGemvMaxWarps, side_k) <= (size_t)kGemvSmemLimit;
 }
 
 int launch_gemv(const GemmArgs& a, cudaStream_t st) {
@@ -277,13 +320,21 @@ int launch_gemv(const GemmArgs& a, cudaStream_t st) {
   p.W_layout = static_cast<const uint8_t*>(a.W_layout);
   p.s_w = a.s_w; p.bias = a.bias; p.Y = a.Y; p.ldy = a.ldy; p.y_is_f32 = a.y_is_f32; p.acc_out = a.acc_out;
   p.row_scales = a.row_scales;
+  if (a.side_layout) {
+    if (a.Qx || !a.rot_block) return MQ_ERR_INVALID_ARG;
+    p.side_layout = static_cast<const uint8_t*>(a.side_layout);
+    p.s_w_side = a.s_w_side;
+    p.side_kb = (a.side_k + MQ_W_TILE_K - 1) / MQ_W_TILE_K;
+    p.side_cols = a.K / a.rot_block;
+    p.acc_side_out = a.acc_side_out;
+  }
   const int n_tn = (a.N + MQ_W_TILE_N - 1) / MQ_W_TILE_N;
   const int ctas = n_tn * 4;
   int warps = (gemv_sm_count() * kGemvWarpsPerSm + ctas - 1) / ctas;
   if (warps > kGemvMaxWarps) warps = kGemvMaxWarps;
   if (warps > p.kb_total) warps = p.kb_total;
   if (warps < 1) warps = 1;
-  const size_t smem = gemv_smem(a.T, a.K, warps);
+  const size_t smem = gemv_smem(a.T, a.K, warps, a.side_layout ? a.side_k : 0);
   auto kernel = a.T <= 1 ? w4a8_gemv_kernel<1> : (a.T <= 2 ? w4a8_gemv_kernel<2> : w4a8_gemv_kernel<4>);
   static bool attr_set[3] = {false, false, false};
   const int ki = a.T <= 1 ? 0 : (a.T <= 2 ? 1 : 2);
