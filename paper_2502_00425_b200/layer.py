@@ -58,11 +58,34 @@ def rope(x: torch.Tensor, pos: torch.Tensor, n_heads: int, base: float = 10000.0
     L, width = x.shape
     D = width // n_heads
     xf = x.float().view(L, n_heads, D // 2, 2)
-    theta = base ** (-2.0 * torch.arange(D // 2, device=x.device, dtype=torch.float64) / D)
-    ang = pos.to(torch.float64)[:, None] * theta[None, :]
-    c, s = torch.cos(ang).float()[:, None, :], torch.sin(ang).float()[:, None, :]
+    # float32 angles: positions are exact, the product is off by ~1e-4 rad at a few thousand tokens
+    theta = (base ** (-2.0 * torch.arange(D // 2, device=x.device, dtype=torch.float64) / D)).float()
+    ang = pos.to(torch.float32)[:, None] * theta[None, :]
+    c, s = torch.cos(ang)[:, None, :], torch.sin(ang)[:, None, :]
     out = torch.stack((xf[..., 0] * c - xf[..., 1] * s, xf[..., 0] * s + xf[..., 1] * c), dim=-1)
     return out.view(L, width).to(torch.bfloat16)
+
+
+def gqa_attention_unpermuted(q, k, v, perm, n_q_heads: int, n_kv_heads: int) -> torch.Tensor:
+    """The same attention without a dense mask, for sequences without pads: the unified mask is the
+    causal mask of the ORIGINAL order (Eq. 5), so the rows are put back in that order, a plain
+    causal attention runs (which the library's fused kernels support), and the result returns to
+    AIFS order.  Mathematically identical to gqa_attention with the unified mask."""
+    L = q.shape[0]
+    D = q.shape[1] // n_q_heads
+    group = n_q_heads // n_kv_heads
+    idx = perm.long()
+
+    def to_orig(x, heads):
+        out = torch.empty_like(x)
+        out[idx] = x
+        return out.view(L, heads, D).transpose(0, 1)
+
+    qh = to_orig(q, n_q_heads)
+    kh = to_orig(k, n_kv_heads).repeat_interleave(group, dim=0)
+    vh = to_orig(v, n_kv_heads).repeat_interleave(group, dim=0)
+    o = torch.nn.functional.scaled_dot_product_attention(qh[None], kh[None], vh[None], is_causal=True)
+    return o[0].transpose(0, 1).reshape(L, n_q_heads * D)[idx].contiguous()
 
 
 def gqa_attention(q, k, v, mask, n_q_heads: int, n_kv_heads: int) -> torch.Tensor:
@@ -84,6 +107,9 @@ class W4A8DecoderBlock:
                  g_mlp: torch.Tensor, device="cuda"):
         self.shape, self.w, self.g_attn, self.g_mlp, self.device = shape, weights, g_attn, g_mlp, device
         self._ws: Dict[Tuple[str, int], torch.Tensor] = {}
+        # True: attention in the original order with a plain causal mask instead of the dense unified
+        # mask (same result, much faster glue); the dense mask is still produced and kept in the trace
+        self.causal_glue = False
 
     # ---- pieces ------------------------------------------------------------------------
     def aifs(self, embs, is_visuals, tr: BlockTrace) -> torch.Tensor:
@@ -186,8 +212,12 @@ class W4A8DecoderBlock:
         qr = torch.cat([rope(q[bd[b]:bd[b + 1]], tr.pos_us[b], sh.n_q_heads) for b in range(n_seq)])
         kr = torch.cat([rope(k[bd[b]:bd[b + 1]], tr.pos_us[b], sh.n_kv_heads) for b in range(n_seq)])
         t["q_rope"], t["k_rope"] = qr, kr
-        a = torch.cat([gqa_attention(qr[bd[b]:bd[b + 1]], kr[bd[b]:bd[b + 1]], v[bd[b]:bd[b + 1]], tr.masks[b],
-                                     sh.n_q_heads, sh.n_kv_heads) for b in range(n_seq)])
+        if self.causal_glue:
+            a = torch.cat([gqa_attention_unpermuted(qr[bd[b]:bd[b + 1]], kr[bd[b]:bd[b + 1]], v[bd[b]:bd[b + 1]],
+                                                    tr.perms[b], sh.n_q_heads, sh.n_kv_heads) for b in range(n_seq)])
+        else:
+            a = torch.cat([gqa_attention(qr[bd[b]:bd[b + 1]], kr[bd[b]:bd[b + 1]], v[bd[b]:bd[b + 1]], tr.masks[b],
+                                         sh.n_q_heads, sh.n_kv_heads) for b in range(n_seq)])
         t["attn"] = a
         o = self.linear("o_proj", a, tr, calibrate)
         x1 = (x0.float() + o.float()).to(torch.bfloat16)

@@ -152,3 +152,18 @@ def test_batched_block_with_eight_segments():
     # another attention kernel for another shape, hence a tolerance rather than equality)
     out_single, _ = blk.forward(bf16_to_dev(embs[1]), torch.from_numpy(seqs[1]).to(DEV))
     assert _close_rowmax(bf16_from_dev(out_single), bf16_from_dev(outs[1]))
+
+
+def test_causal_glue_matches_the_unified_mask():
+    """Attention invariance (Eq. 5) at the level of the block: running the glue attention in the
+    original order with a plain causal mask gives the same block output as the dense unified mask."""
+    shape = synth.LayerShape(hidden=256, n_q_heads=4, n_kv_heads=2, head_dim=64, mlp=512)
+    is_visual = synth.interleaved_modality([(0, 9), (1, 70), (0, 15), (1, 40), (0, 21)])
+    blk, _, _, _ = _make_block(shape, 61)
+    emb = bf16_to_dev(synth.embedding_rows(62, is_visual.shape[0], shape.hidden, is_visual))
+    vis = torch.from_numpy(is_visual).to(DEV)
+    out_mask, tr_mask = blk.forward(emb, vis, calibrate=True)
+    blk.causal_glue = True
+    out_causal, tr_causal = blk.forward(emb, vis)
+    assert _close_rowmax(bf16_from_dev(tr_causal.tensors["attn"]), bf16_from_dev(tr_mask.tensors["attn"]))
+    assert _close_rowmax(bf16_from_dev(out_causal), bf16_from_dev(out_mask))
