@@ -7,15 +7,19 @@
  *  - Every function returns an int status (MQ_OK = 0, negative = error) and never
  *    throws.  mq_status_string() names a status.
  *  - Unless a parameter says "host", every pointer is DEVICE memory owned by the
- *    caller.  The library never allocates, frees or keeps device memory; scratch
- *    comes from a caller-provided workspace sized by mq_workspace_bytes().
+ *    caller.  The library never allocates or frees device memory; scratch comes
+ *    from a caller-provided workspace sized by mq_workspace_bytes().  The one piece
+ *    of device memory the library itself holds is the fixed MQ_NOALLOC_WS_BYTES
+ *    array behind mq_w4a8_msq_linear_noalloc (part of its device image).
  *  - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls
  *    enqueue work on it and return without synchronising, except
  *    mq_last_device_status(), which waits for the stream.
  *  - Activations are row-major [rows, cols] with a leading dimension `ld*` counted
  *    in ELEMENTS.  bf16 activations are the usual upper-16-bits-of-float32 format.
- *    Base pointers must be 16-byte aligned and row pitches multiples of 16 bytes,
- *    otherwise MQ_ERR_ALIGNMENT.
+ *    Base pointers must be 16-byte aligned and the row pitches of X and Q
+ *    multiples of 16 bytes, otherwise MQ_ERR_ALIGNMENT.  A bf16 Y whose row pitch is
+ *    not a multiple of 16 bytes is accepted; it is written with 2-byte instead of
+ *    16-byte stores.
  *  - Weights are W[N,K] (output channel x input channel), so Y = X . W^T.
  *  - Token modality is given by a segment table (Sec. 3.1, Eq. 3: the text and
  *    visual spans of the sequence each use their own static scale): row t has the
@@ -344,6 +348,34 @@ size_t mq_dynamic_workspace_bytes(const mq_linear_desc* d);
 int mq_w4a8_dynamic_linear(const mq_linear_desc* d, const void* X, int64_t ldx, const void* W_layout,
                            const float* s_w, const float* bias, void* Y, int64_t ldy, int32_t* acc_out,
                            float* s_rows_out, void* ws, size_t ws_bytes, void* stream);
+
+/* ---- Measurement and self-test aids (the paper has no counterpart) ------------------------- */
+
+/*
+ * Issue-rate microbenchmark of the int8 tensor-core instruction the GEMM is built on
+ * (tcgen05.mma kind::i8, 128 x n_tok x 32 per instruction), with fixed operands and no loads: the
+ * denominator "what the tensor pipe can do on this machine at the clock it holds" next to the
+ * nominal and the bf16-derived figures.  `ctas` CTAs (one per SM up to the SM count) each issue
+ * n_mma MMAs rotating over n_acc accumulators of n_tok columns (n_acc * n_tok <= 480); A comes
+ * from tensor memory (a_from_smem = 0, as in the GEMM) or from shared memory (1).
+ *   cycles_out  device uint64 [ctas]: SM clock cycles from the first issue to the completion of
+ *               the last MMA (0 if the bounded wait gave up)
+ *   status      device int32 [2], zeroed by the caller: MQ_ERR_TIMEOUT + site if a wait gave up
+ * int8 operations per clock and SM = 2 * 128 * n_tok * 32 * n_mma / cycles.
+ */
+int mq_ubench_mma_i8(int32_t n_tok, int32_t n_mma, int32_t n_acc, int32_t a_from_smem, int32_t ctas,
+                     uint64_t* cycles_out, int32_t* status, void* stream);
+
+/*
+ * Exercises the bounded wait that every kernel of the library uses on its mbarriers, on a barrier
+ * that nothing arrives at: after limit_ns (1 .. 1e9) the wait gives up, writes
+ * {MQ_ERR_TIMEOUT, site} to status (device int32 [2], zeroed by the caller) and raises the CTA's
+ * abort flag; a second wait then returns at once.  The kernel returns normally: nothing faults.
+ *   waited_ns_out  device uint64 [4]: {ns the first wait lasted, 1 if it (wrongly) succeeded,
+ *                  ns the second wait lasted, 1 if it (wrongly) succeeded}
+ */
+int mq_selftest_bounded_wait(uint64_t limit_ns, int32_t site, int32_t* status, uint64_t* waited_ns_out,
+                             void* stream);
 
 /* Waits for `stream`, then returns the status word kernels left in the workspace
  * (MQ_OK or MQ_ERR_TIMEOUT) and, if site_out != NULL (host), where the wait gave up. */

@@ -86,6 +86,8 @@ def load(build_if_missing: bool = False):
         "mq_dynamic_quant_i8": (C.c_int, [vp, i32, i32, i64, i32, vp, i64, vp, vp]),
         "mq_dynamic_workspace_bytes": (sz, [descp]),
         "mq_w4a8_dynamic_linear": (C.c_int, [descp, vp, i64, vp, vp, vp, vp, i64, vp, vp, vp, sz, vp]),
+        "mq_ubench_mma_i8": (C.c_int, [i32, i32, i32, i32, i32, vp, vp, vp]),
+        "mq_selftest_bounded_wait": (C.c_int, [C.c_uint64, i32, vp, vp, vp]),
         "mq_last_device_status": (C.c_int, [vp, vp, C.POINTER(C.c_int32)]),
         "mq_reset_device_status": (C.c_int, [vp, vp]),
     }
@@ -101,7 +103,8 @@ EXPORTED = ["mq_version", "mq_status_string", "mq_workspace_bytes", "mq_w4_layou
             "mq_calibrate_static_scales", "mq_pack_w4", "mq_repack_w4", "mq_unpack_w4", "mq_aifs_reorder",
             "mq_attn_mask_remap", "mq_fwht_quant_i8", "mq_w4a8_msq_linear", "mq_w4a8_msq_linear_noalloc", "mq_last_device_status",
             "mq_reset_device_status", "mq_rms_side_ld", "mq_rms_detect", "mq_pack_w4_rms", "mq_rms_workspace_bytes",
-            "mq_w4a8_msq_linear_rms", "mq_dynamic_quant_i8", "mq_dynamic_workspace_bytes", "mq_w4a8_dynamic_linear"]
+            "mq_w4a8_msq_linear_rms", "mq_dynamic_quant_i8", "mq_dynamic_workspace_bytes", "mq_w4a8_dynamic_linear",
+            "mq_ubench_mma_i8", "mq_selftest_bounded_wait"]
 
 
 def status_string(status: int) -> str:
@@ -341,6 +344,20 @@ def mq_w4a8_dynamic_linear(x, w_layout, s_w, y, ws, N, rot_block=0, bias=None, a
     _check(load().mq_w4a8_dynamic_linear(C.byref(d), _ptr(x), _ld(x), _ptr(w_layout), _ptr(s_w), _ptr(bias), _ptr(y),
                                          _ld(y), _ptr(acc_out), _ptr(s_rows_out), _ptr(ws), ws.numel(), _stream()),
            "mq_w4a8_dynamic_linear")
+
+
+def mq_ubench_mma_i8(n_tok, n_mma, n_acc, a_from_smem, ctas, cycles_out, status):
+    """Issue-rate microbenchmark of tcgen05.mma kind::i8; cycles_out int64 [ctas], status int32 [2] (zeroed)."""
+    assert cycles_out.dtype == torch.int64 and cycles_out.numel() >= ctas and status.dtype == torch.int32
+    _check(load().mq_ubench_mma_i8(n_tok, n_mma, n_acc, int(a_from_smem), ctas, _ptr(cycles_out), _ptr(status),
+                                   _stream()), "mq_ubench_mma_i8")
+
+
+def mq_selftest_bounded_wait(limit_ns, site, status, waited_ns_out):
+    """Bounded mbarrier wait on a barrier nobody arrives at; status int32 [2] (zeroed), waited_ns_out int64 [4]."""
+    assert status.dtype == torch.int32 and waited_ns_out.dtype == torch.int64 and waited_ns_out.numel() >= 4
+    _check(load().mq_selftest_bounded_wait(int(limit_ns), int(site), _ptr(status), _ptr(waited_ns_out), _stream()),
+           "mq_selftest_bounded_wait")
 
 
 def mq_last_device_status(ws):

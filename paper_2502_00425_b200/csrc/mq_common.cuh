@@ -5,6 +5,7 @@
 #include <stdint.h>
 
 #include "mq.h"
+#include "mq_device_table.h"
 
 namespace mq {
 
@@ -44,7 +45,41 @@ __device__ __forceinline__ int thread_row_modality(const SegTable& seg, int t) {
   return MQ_TEXT;
 }
 
-inline int cuda_status(cudaError_t e) { return e == cudaSuccess ? MQ_OK : MQ_ERR_CUDA; }
+// A failed runtime call also leaves its error in the runtime's per-thread "last error" slot, where the
+// next launcher's cudaGetLastError() would find it: clear it when reporting the failure.
+inline int cuda_status(cudaError_t e) {
+  if (e == cudaSuccess) return MQ_OK;
+  (void)cudaGetLastError();
+  return MQ_ERR_CUDA;
+}
+
+// ---- per-device host state ------------------------------------------------------------
+// SM count of the CURRENT device (148 if the query fails), cached per device.
+inline int sm_count() {
+  static PerDeviceTable<int> table;
+  int dev = -1, n = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) dev = -1;
+  const bool ok = table.get(dev, [](int d, int* out) {
+    return d >= 0 && cudaDeviceGetAttribute(out, cudaDevAttrMultiProcessorCount, d) == cudaSuccess && *out > 0;
+  }, &n);
+  return ok ? n : 148;
+}
+
+// Raises `kernel`'s dynamic shared-memory limit to `bytes` on the current device, once per device
+// (function attributes belong to the device's context, not to the process).  `table` is the
+// caller's static table for that kernel.
+template <typename Kernel>
+inline bool ensure_dynamic_smem(PerDeviceTable<char>& table, Kernel kernel, int bytes) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) dev = -1;
+  char done = 0;
+  const bool ok = table.get(dev, [&](int, char* out) {
+    *out = 1;
+    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess;
+  }, &done);
+  if (!ok) (void)cudaGetLastError();
+  return ok;
+}
 
 // ---- programmatic dependent launch ----------------------------------------------------
 // The hot-path kernels follow one another on a stream, each a few tens of microseconds long,

@@ -27,9 +27,10 @@
 // MMA sees 16*q_w; the accumulator is therefore exactly 16x the true one (|16 acc| <=
 // 128*8*16*K < 2^31 for K <= 131071) and the epilogue shifts it back, exactly.
 //
-// Warp roles (384 threads): warp 0 activation TMA producer, warp 1 MMA issuer, warp 2
-// tensor-memory allocator, warp 3 weight bulk-copy producer, warps 4-7 weight expanders
-// (one per 32-lane quarter of tensor memory), warps 8-11 epilogue.
+// Warp roles (512 threads): warp 0 activation TMA producer, warp 1 MMA issuer, warp 2
+// tensor-memory allocator, warp 3 weight bulk-copy producer, warps 4-11 weight expanders (two
+// groups of four that take alternate K blocks; within a group one warp per 32-lane quarter of
+// tensor memory), warps 12-15 epilogue.
 //
 // Every wait on an mbarrier is bounded: after ~2 s without progress the waiting thread
 // records MQ_ERR_TIMEOUT and its site in the status word, raises a CTA-wide abort flag,
@@ -38,6 +39,7 @@
 #include <cuda_bf16.h>
 
 #include "mq_common.cuh"
+#include "mq_sm100.cuh"
 
 namespace mq {
 namespace {
@@ -49,7 +51,6 @@ constexpr int kBlockK = MQ_W_TILE_K;   // K per pipeline stage
 constexpr int kWTileBytes = 8192;      // packed int4 tile 128 x 128
 constexpr int kMaxStages = 8;    // main ring: activation tiles in shared memory
 constexpr int kMaxWStages = 16;  // packed-weight tiles in shared memory
-constexpr unsigned long long kTimeoutNs = 2000000000ull;
 constexpr int kSmemBudget = 226 * 1024;  // of the 227 KB a CTA may use
 
 struct KernelParams {
@@ -100,170 +101,6 @@ struct __align__(16) Barriers {
   uint32_t tmem_base;
   int abort_flag;
 };
-
-// ------------------------------------------------------------------------------ PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-// Arrive that cannot be issued before `dep` is available in a register.  Used to release a
-// shared-memory stage after reading it: `dep` is computed from every load of the stage, so the
-// loads have returned their data (not merely been issued) when the producer is told to overwrite it.
-__device__ __forceinline__ void mbar_arrive_after(uint64_t* bar, uint32_t dep) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];  // after %1" ::"r"(smem_u32(bar)), "r"(dep) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
-               : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-__device__ __forceinline__ unsigned long long globaltimer_ns() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
-
-// Bounded wait.  Returns false if the CTA is aborting (this wait or another one expired).
-__device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, Barriers* sh,
-                                            int32_t* status, int site) {
-  const unsigned long long t0 = globaltimer_ns();
-  unsigned spins = 0;
-  while (true) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((++spins & 63u) == 0u) {
-      if (*reinterpret_cast<volatile int*>(&sh->abort_flag)) return false;
-      if (globaltimer_ns() - t0 > kTimeoutNs) {
-        *reinterpret_cast<volatile int*>(&sh->abort_flag) = 1;
-        if (atomicCAS(status, MQ_OK, MQ_ERR_TIMEOUT) == MQ_OK) status[1] = site;
-        __threadfence();
-        return false;
-      }
-    }
-  }
-}
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, Barriers* sh,
-                                          int32_t* status, int site) {
-  if (mbar_try_wait(bar, parity)) return true;
-  return mbar_wait_slow(bar, parity, sh, status, site);
-}
-
-// Wait used while a CTA winds down after an abort: ignores the abort flag, gives up quietly
-// after `limit_ns` (asynchronous copies and MMAs already issued get that long to finish).
-__device__ __noinline__ void mbar_wait_drain(uint64_t* bar, uint32_t parity, unsigned long long limit_ns) {
-  const unsigned long long t0 = globaltimer_ns();
-  unsigned spins = 0;
-  while (!mbar_try_wait(bar, parity)) {
-    if ((++spins & 15u) == 0u && globaltimer_ns() - t0 > limit_ns) return;
-  }
-}
-
-__device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* tmap, int x, int y,
-                                            uint64_t* bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-      ::"r"(smem_u32(smem_dst)), "l"(tmap), "r"(smem_u32(bar)), "r"(x), "r"(y)
-      : "memory");
-}
-__device__ __forceinline__ void bulk_load_1d(void* smem_dst, const void* gsrc, uint32_t bytes,
-                                             uint64_t* bar) {
-  asm volatile(
-      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-      ::"r"(smem_u32(smem_dst)), "l"(gsrc), "r"(bytes), "r"(smem_u32(bar))
-      : "memory");
-}
-
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-__device__ __forceinline__ void tmem_alloc(uint32_t* smem_dst, uint32_t ncols) {
-  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_dst)),
-               "r"(ncols)
-               : "memory");
-}
-__device__ __forceinline__ void tmem_relinquish() {
-  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
-  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
-}
-
-// D[tmem] (+)= A[tmem] * B[smem], int8 x int8 -> int32, one CTA.
-__device__ __forceinline__ void mma_i8_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
-                                          uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::i8 [%0], [%1], %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-// Arrive on an mbarrier once all tcgen05 operations issued so far by this thread are done.
-__device__ __forceinline__ void tc_commit(uint64_t* bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
-               : "memory");
-}
-
-__device__ __forceinline__ void tmem_st_x32(uint32_t taddr, const uint32_t (&r)[32]) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
-      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
-      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
-      "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
-      "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
-      "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
-      : "memory");
-}
-__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void tmem_ld_x16(uint32_t taddr, uint32_t (&r)[16]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-      : "r"(taddr)
-      : "memory");
-}
-__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// True in exactly one lane of a converged warp.
-__device__ __forceinline__ bool elect_one() {
-  uint32_t pred;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "elect.sync _|p, 0xffffffff;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(pred));
-  return pred != 0;
-}
-
-// Warp-uniform verdict of a bounded wait, so that .sync.aligned instructions stay converged.
-__device__ __forceinline__ bool warp_all(bool ok) { return __all_sync(0xffffffffu, ok) != 0; }
-
-// K-major, 128-byte-swizzled shared-memory operand: rows of 128 bytes, 8-row groups 1024 B apart.
-__device__ __forceinline__ uint64_t make_b_desc(uint32_t smem_addr) {
-  return (uint64_t)((smem_addr >> 4) & 0x3FFFu) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
-}
-// kind::i8: D = s32 (bits 4-5 = 2), A = B = signed 8-bit (bits 7-9, 10-12 = 1), both K-major,
-// N >> 3 at bits 17-22, M >> 4 at bits 24-28.
-__device__ __forceinline__ uint32_t make_idesc(int n) {
-  return (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileN >> 4) << 24);
-}
 
 // Tile t of the launch is (channel tile, token tile, K split) = (t % n_tn, (t / n_tn) % n_tt,
 // t / (n_tn * n_tt)); CTA b owns tiles b, b + grid, b + 2 grid, ...  The first one is decoded
@@ -518,7 +355,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const __grid_cons
         const int row0 = c.tt * p.TN;
         if (RMS && c.ks == 0) {
           for (int sb = 0; sb < p.side_kb; ++sb, ++it) {
-            if (wrapped && !(ok = mbar_wait(&sh->done[s], ph ^ 1u, sh, p.status, 1))) break;
+            if (wrapped && !(ok = mbar_wait(&sh->done[s], ph ^ 1u, &sh->abort_flag, p.status, 1))) break;
             mbar_arrive_expect_tx(&sh->full[s], act_stage_bytes);
             tma_load_2d(act_smem + (size_t)s * act_stage_bytes, &tmap_side, sb * kBlockK, row0, &sh->full[s]);
             if (++s == p.stages) { s = 0; ph ^= 1u; wrapped = true; }
@@ -526,7 +363,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const __grid_cons
           if (!ok) break;
         }
         for (int kb = c.kb0(p), kb_end = c.kb1(p); kb < kb_end; ++kb, ++it) {
-          if (wrapped && !(ok = mbar_wait(&sh->done[s], ph ^ 1u, sh, p.status, 1))) break;
+          if (wrapped && !(ok = mbar_wait(&sh->done[s], ph ^ 1u, &sh->abort_flag, p.status, 1))) break;
           mbar_arrive_expect_tx(&sh->full[s], act_stage_bytes);
           tma_load_2d(act_smem + (size_t)s * act_stage_bytes, &tmap_act, kb * kBlockK, row0, &sh->full[s]);
           if (++s == p.stages) { s = 0; ph ^= 1u; wrapped = true; }
@@ -552,7 +389,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const __grid_cons
         if (RMS && c.ks == 0) {
           const uint8_t* ssrc = p.side_layout + (size_t)c.tn * p.side_kb * kWTileBytes;
           for (int sb = 0; sb < p.side_kb; ++sb, ++it, ssrc += kWTileBytes) {
-            if (wrapped && !(ok = mbar_wait(&sh->w_empty[s], ph ^ 1u, sh, p.status, 2))) break;
+            if (wrapped && !(ok = mbar_wait(&sh->w_empty[s], ph ^ 1u, &sh->abort_flag, p.status, 2))) break;
             mbar_arrive_expect_tx(&sh->w_full[s], kWTileBytes);
             bulk_load_1d(w_smem + (size_t)s * kWTileBytes, ssrc, kWTileBytes, &sh->w_full[s]);
             if (++s == p.w_stages) { s = 0; ph ^= 1u; wrapped = true; }
@@ -561,7 +398,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const __grid_cons
         }
         const uint8_t* wsrc = p.W_layout + ((size_t)c.tn * p.kb_total + c.kb0(p)) * kWTileBytes;
         for (int kb = c.kb0(p), kb_end = c.kb1(p); kb < kb_end; ++kb, ++it, wsrc += kWTileBytes) {
-          if (wrapped && !(ok = mbar_wait(&sh->w_empty[s], ph ^ 1u, sh, p.status, 2))) break;
+          if (wrapped && !(ok = mbar_wait(&sh->w_empty[s], ph ^ 1u, &sh->abort_flag, p.status, 2))) break;
           mbar_arrive_expect_tx(&sh->w_full[s], kWTileBytes);
           bulk_load_1d(w_smem + (size_t)s * kWTileBytes, wsrc, kWTileBytes, &sh->w_full[s]);
           if (++s == p.w_stages) { s = 0; ph ^= 1u; wrapped = true; }
@@ -583,7 +420,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const __grid_cons
     uint32_t ph = 0, ph_d = 0;
     bool d_wrapped = false, ok = true;
     for (TileIter c = first; c.valid(p) && ok; c.next(p)) {
-      if (d_wrapped && !(ok = warp_all(mbar_wait(&sh->d_empty[d], ph_d ^ 1u, sh, p.status, 3)))) break;
+      if (d_wrapped && !(ok = warp_all(mbar_wait(&sh->d_empty[d], ph_d ^ 1u, &sh->abort_flag, p.status, 3)))) break;
       tc_fence_after();
       const uint32_t d_tmem = tmem_base + (uint32_t)(d * p.d_stride);
       uint32_t accumulate = 0;
@@ -591,7 +428,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const __grid_cons
         // the split product first, into its own accumulator
         const uint32_t ds_tmem = d_tmem + (uint32_t)p.side_col;
         for (int sb = 0; sb < p.side_kb; ++sb) {
-          if (!(ok = warp_all(mbar_wait(&sh->full[s], ph, sh, p.status, 4)))) break;
+          if (!(ok = warp_all(mbar_wait(&sh->full[s], ph, &sh->abort_flag, p.status, 4)))) break;
           tc_fence_after();
           const uint64_t bdesc = bdesc0 + (uint64_t)((uint32_t)s * bdesc_step);
           const uint32_t a_tmem = tmem_base + (uint32_t)(p.a_base + a * 32);
@@ -609,7 +446,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const __grid_cons
         accumulate = 0;
       }
       for (int kb = c.kb0(p), kb_end = c.kb1(p); kb < kb_end; ++kb) {
-        if (!(ok = warp_all(mbar_wait(&sh->full[s], ph, sh, p.status, 4)))) break;
+        if (!(ok = warp_all(mbar_wait(&sh->full[s], ph, &sh->abort_flag, p.status, 4)))) break;
         tc_fence_after();
         // operands are computed by the whole (converged) warp so that they stay warp-uniform
         const uint64_t bdesc = bdesc0 + (uint64_t)((uint32_t)s * bdesc_step);
@@ -648,7 +485,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const __grid_cons
     uint32_t ph_w = 0, ph = 0;
     bool ok = true;
     for (int it = grp; it < total_it && ok; it += p.groups) {
-      if (!(ok = warp_all(mbar_wait(&sh->w_full[sw], ph_w, sh, p.status, 6)))) break;
+      if (!(ok = warp_all(mbar_wait(&sh->w_full[sw], ph_w, &sh->abort_flag, p.status, 6)))) break;
       const uint4* src = reinterpret_cast<const uint4*>(w_smem + (size_t)sw * kWTileBytes) + r;
       uint32_t regs[32];
 #pragma unroll
@@ -668,7 +505,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const __grid_cons
         // stage and parity of block it - num_a, derived from those of block it
         const int fs = s >= p.num_a ? s - p.num_a : s - p.num_a + p.stages;
         const uint32_t fph = s >= p.num_a ? ph : ph ^ 1u;
-        if (!(ok = warp_all(mbar_wait(&sh->done[fs], fph, sh, p.status, 7)))) break;
+        if (!(ok = warp_all(mbar_wait(&sh->done[fs], fph, &sh->abort_flag, p.status, 7)))) break;
       }
       tc_fence_after();
       tmem_st_x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(p.a_base + a * 32), regs);
@@ -703,7 +540,7 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const __grid_cons
         else stok[j] = (t < p.T && thread_row_modality(p.seg, t) == MQ_VISUAL) ? p.s_vis : p.s_txt;
       }
       __syncwarp();
-      if (!(ok = warp_all(mbar_wait(&sh->d_full[d], ph_d, sh, p.status, 8)))) break;
+      if (!(ok = warp_all(mbar_wait(&sh->d_full[d], ph_d, &sh->abort_flag, p.status, 8)))) break;
       tc_fence_after();
       const int n = c.tn * kTileN + q * 32 + lane;
       const bool n_ok = n < p.N;
@@ -793,17 +630,6 @@ struct Plan {
   int TN, n_tt, n_tn, ksplit, num_d, d_stride, a_base, num_a, stages, w_stages, grid, groups;
   size_t smem;
 };
-
-int sm_count() {
-  static int n = 0;
-  if (!n) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
-      n = 148;
-  }
-  return n;
-}
 
 // rms: the launch carries a split accumulator next to every accumulator (rotation magnitude
 // suppression), so a token tile may use at most 224 of the 512 tensor-memory columns twice over,
@@ -942,12 +768,8 @@ int launch_gemm(const GemmArgs& a, cudaStream_t st) {
   }
 
   auto kernel = rms ? w4a8_gemm_kernel<true> : w4a8_gemm_kernel<false>;
-  static bool attr_set[2] = {false, false};
-  if (!attr_set[rms ? 1 : 0]) {
-    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget) != cudaSuccess)
-      return MQ_ERR_CUDA;
-    attr_set[rms ? 1 : 0] = true;
-  }
+  static PerDeviceTable<char> attr_set[2];
+  if (!ensure_dynamic_smem(attr_set[rms ? 1 : 0], kernel, kSmemBudget)) return MQ_ERR_CUDA;
 
   KernelParams p{};
   p.T = a.T; p.K = a.K; p.N = a.N;
@@ -975,15 +797,17 @@ int launch_gemm(const GemmArgs& a, cudaStream_t st) {
   }
 
   if (pl.ksplit > 1 && !a.splitk_acc) return MQ_ERR_WORKSPACE;
-  if (launch_pdl(kernel, dim3(pl.grid), dim3((8 + 4 * pl.groups) * 32), pl.smem, st, tmap, tmap_side, p) != cudaSuccess)
+  if (cuda_status(launch_pdl(kernel, dim3(pl.grid), dim3((8 + 4 * pl.groups) * 32), pl.smem, st, tmap, tmap_side, p)) != MQ_OK)
     return MQ_ERR_CUDA;
   if (pl.ksplit > 1) {
     const int64_t n = (int64_t)a.T * a.N;
     if (launch_pdl(splitk_finalize_kernel, dim3((unsigned)((n + 255) / 256)), dim3(256), 0, st,
                    static_cast<const int32_t*>(a.splitk_acc), pl.ksplit, a.T, a.N, a.seg, a.s_vis, a.s_txt, a.s_w, a.bias, a.Y,
                    a.ldy, a.y_is_f32, a.acc_out, static_cast<const int32_t*>(side_slice), a.s_w_side,
-                   a.acc_side_out, a.row_scales) != cudaSuccess)
+                   a.acc_side_out, a.row_scales) != cudaSuccess) {
+      (void)cudaGetLastError();
       return MQ_ERR_CUDA;
+    }
   }
   return MQ_OK;
 }

@@ -280,17 +280,6 @@ w4a8_gemv_kernel(const GemvParams p) {
   }
 }
 
-int gemv_sm_count() {
-  static int n = 0;
-  if (!n) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
-      n = 148;
-  }
-  return n;
-}
-
 size_t gemv_smem(int T, int K, int warps, int side_k = 0) {
   const int tt = T <= 1 ? 1 : (T <= 2 ? 2 : 4);
   const size_t kpad = (size_t)((K + MQ_W_TILE_K - 1) / MQ_W_TILE_K) * MQ_W_TILE_K;
@@ -330,19 +319,15 @@ int launch_gemv(const GemmArgs& a, cudaStream_t st) {
   }
   const int n_tn = (a.N + MQ_W_TILE_N - 1) / MQ_W_TILE_N;
   const int ctas = n_tn * 4;
-  int warps = (gemv_sm_count() * kGemvWarpsPerSm + ctas - 1) / ctas;
+  int warps = (sm_count() * kGemvWarpsPerSm + ctas - 1) / ctas;
   if (warps > kGemvMaxWarps) warps = kGemvMaxWarps;
   if (warps > p.kb_total) warps = p.kb_total;
   if (warps < 1) warps = 1;
   const size_t smem = gemv_smem(a.T, a.K, warps, a.side_layout ? a.side_k : 0);
   auto kernel = a.T <= 1 ? w4a8_gemv_kernel<1> : (a.T <= 2 ? w4a8_gemv_kernel<2> : w4a8_gemv_kernel<4>);
-  static bool attr_set[3] = {false, false, false};
+  static PerDeviceTable<char> attr_set[3];
   const int ki = a.T <= 1 ? 0 : (a.T <= 2 ? 1 : 2);
-  if (!attr_set[ki]) {
-    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGemvSmemLimit) != cudaSuccess)
-      return MQ_ERR_CUDA;
-    attr_set[ki] = true;
-  }
+  if (!ensure_dynamic_smem(attr_set[ki], kernel, kGemvSmemLimit)) return MQ_ERR_CUDA;
   return cuda_status(launch_pdl(kernel, dim3(ctas), dim3(warps * 32), smem, st, p));
 }
 

@@ -42,17 +42,22 @@ def gpu_pack(w: np.ndarray):
     return packed, s_w, layout
 
 
-def gpu_linear(case, s_vis, s_txt, layout, s_w, bias=None, y_dtype=torch.bfloat16, x_codes=None, want_acc=True):
-    """Runs mq_w4a8_msq_linear on a synth.LinearCase; returns (y, acc, status)."""
+def gpu_linear(case, s_vis, s_txt, layout, s_w, bias=None, y_dtype=torch.bfloat16, x_codes=None, want_acc=True,
+               y_pad=0):
+    """Runs mq_w4a8_msq_linear on a synth.LinearCase; returns (y, acc, status).  y_pad > 0 makes Y a
+    view of a wider array (row pitch N + y_pad elements); the padding must come back untouched."""
     T, K, N = case.T, case.K, case.N
     x = x_codes if x_codes is not None else bf16_to_dev(case.x)
     flags = B.MQ_FLAG_X_IS_INT8 if x_codes is not None else 0
     rot = 0 if x_codes is not None else case.rot_block
     ws = B.new_workspace(T, K, N, rot, flags)
-    y = torch.full((T, N), float("nan"), dtype=y_dtype, device=DEV)
+    y_full = torch.full((T, N + y_pad), float("nan"), dtype=y_dtype, device=DEV)
+    y = y_full[:, :N] if y_pad else y_full
     acc = torch.full((T, N), -(2 ** 31), dtype=torch.int32, device=DEV) if want_acc else None
     bias_d = None if bias is None else torch.from_numpy(bias).to(DEV)
     B.mq_w4a8_msq_linear(x, dev_segments(case.seg), s_vis, s_txt, layout, s_w, y, ws, N, rot_block=rot,
                          bias=bias_d, acc_out=acc)
     st = B.mq_last_device_status(ws)
+    if y_pad:
+        assert bool(torch.isnan(y_full[:, N:]).all())
     return y, acc, st

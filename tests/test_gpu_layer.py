@@ -112,14 +112,12 @@ def test_config3_block_full_size_sampled():
     _check_block(shape, is_visual, seed=34, rows=rows)
 
 
-def test_batched_block_with_eight_segments():
-    """Config-4 style batch at a reduced size: four sequences reordered one by one, their rows
-    stacked for the linears (eight segments), attention per sequence."""
-    shape = synth.LayerShape(hidden=256, n_q_heads=4, n_kv_heads=2, head_dim=64, mlp=512)
-    blk, ref_w, g1, g2 = _make_block(shape, 41)
-    seqs = [synth.interleaved_modality(sp) for sp in ([(0, 5), (1, 60), (0, 12)], [(1, 40), (0, 9)],
-                                                      [(0, 3), (1, 30), (0, 4), (1, 20), (0, 6)], [(0, 25)])]
-    embs = [synth.embedding_rows(50 + i, s_.shape[0], shape.hidden, s_) for i, s_ in enumerate(seqs)]
+def _check_batched_block(shape, seqs, seed, rows=None):
+    """A batch of sequences reordered one by one, their rows stacked for the linears (two segments per
+    sequence), attention per sequence.  `rows` (indices into the stacked rows) limits the oracle's
+    work on the linears and the attention to a sample; None checks every row."""
+    blk, ref_w, g1, g2 = _make_block(shape, seed)
+    embs = [synth.embedding_rows(seed + 9 + i, s_.shape[0], shape.hidden, s_) for i, s_ in enumerate(seqs)]
     outs, tr = blk.forward_batch([bf16_to_dev(e) for e in embs], [torch.from_numpy(s_).to(DEV) for s_ in seqs],
                                  calibrate=True)
     assert blk.device_status_ok()
@@ -132,26 +130,71 @@ def test_batched_block_with_eight_segments():
         seg_mod += list(m)
         off += s_.shape[0]
     seg_end, seg_mod = np.array(seg_end, np.int32), np.array(seg_mod, np.uint8)
+    total = off
     assert np.array_equal(tr.seg.seg_end.cpu().numpy(), seg_end) and np.array_equal(tr.seg.seg_mod.cpu().numpy(), seg_mod)
     assert np.array_equal(t["emb_u"], np.concatenate([O.aifs_gather(e, p_) for e, p_ in zip(embs, perms)]))
+    sel = np.arange(total) if rows is None else np.asarray(rows)
+    sub_end = np.searchsorted(sel, seg_end).astype(np.int32)
     for name, K, N, rot in shape.linears():
         x_in = t[name + ".in"]
         s_v, s_t = O.calibrate_static_scales(x_in, seg_end, seg_mod, rot)
         assert (np.float32(blk.w[name].s_vis), np.float32(blk.w[name].s_txt)) == (s_v, s_t), name
         qw, s_w = ref_w[name]
-        ref = O.linear_w4a8_msq(x_in, seg_end, seg_mod, s_v, s_t, rot, qw, s_w)
-        assert np.array_equal(t[name + ".out"], ref["y_bf16"]), name
+        ref = O.linear_w4a8_msq(x_in[sel], sub_end, seg_mod, s_v, s_t, rot, qw, s_w)
+        assert np.array_equal(t[name + ".out"][sel], ref["y_bf16"]), name
     bd = tr.bounds
+    D = shape.head_dim
+    assert _close_rowmax(t["attn_norm"], O.rmsnorm(t["emb_u"], g1))
     for b, (s_, p_) in enumerate(zip(seqs, perms)):
         sl = slice(bd[b], bd[b + 1])
-        ref_attn = O.gqa_attention(t["q_rope"][sl], t["k_rope"][sl], t["v_proj.out"][sl], O.unified_mask(p_),
+        assert np.array_equal(tr.perms[b].cpu().numpy(), p_)
+        pos = O.remap_positions(p_)
+        assert np.array_equal(tr.pos_us[b].cpu().numpy(), pos)
+        allowed = O.unified_mask(p_)
+        assert np.array_equal(tr.masks[b].cpu().numpy(), allowed)
+        for nm, src, heads in (("q_rope", "q_proj.out", shape.n_q_heads), ("k_rope", "k_proj.out", shape.n_kv_heads)):
+            ref = np.concatenate([O.rope(t[src][sl][:, h * D:(h + 1) * D], pos) for h in range(heads)], axis=1)
+            assert _close_rowmax(t[nm][sl], ref), nm
+        local = sel[(sel >= bd[b]) & (sel < bd[b + 1])] - bd[b]      # sampled query rows of this sequence
+        ref_attn = O.gqa_attention(t["q_rope"][sl][local], t["k_rope"][sl], t["v_proj.out"][sl], allowed[local],
                                    shape.n_q_heads, shape.n_kv_heads)
-        assert _close_rowmax(t["attn"][sl], ref_attn)
+        assert _close_rowmax(t["attn"][sl][local], ref_attn)
         assert np.array_equal(bf16_from_dev(outs[b]), O.aifs_scatter(t["resid2"][sl], p_))
+    assert _close_rowmax(t["resid1"], t["emb_u"].astype(np.float64) + t["o_proj.out"])
+    assert _close_rowmax(t["mlp_norm"], O.rmsnorm(t["resid1"], g2))
+    assert _close_rowmax(t["act"], O.swiglu(t["gate_proj.out"], t["up_proj.out"]))
+    assert _close_rowmax(t["resid2"], t["resid1"].astype(np.float64) + t["down_proj.out"])
+    return blk, embs, outs
+
+
+def test_batched_block_with_eight_segments():
+    """Config-4 style batch at a reduced size: four sequences reordered one by one, their rows
+    stacked for the linears (eight segments), attention per sequence."""
+    shape = synth.LayerShape(hidden=256, n_q_heads=4, n_kv_heads=2, head_dim=64, mlp=512)
+    seqs = [synth.interleaved_modality(sp) for sp in ([(0, 5), (1, 60), (0, 12)], [(1, 40), (0, 9)],
+                                                      [(0, 3), (1, 30), (0, 4), (1, 20), (0, 6)], [(0, 25)])]
+    blk, embs, outs = _check_batched_block(shape, seqs, 41)
     # a sequence run alone with the same scales gives what it gave inside the batch (the glue may pick
     # another attention kernel for another shape, hence a tolerance rather than equality)
     out_single, _ = blk.forward(bf16_to_dev(embs[1]), torch.from_numpy(seqs[1]).to(DEV))
     assert _close_rowmax(bf16_from_dev(out_single), bf16_from_dev(outs[1]))
+
+
+def test_config4_block_full_size_sampled():
+    """The 8B-shaped block of config 4 at full size: four sequences of [32 text][2304 visual][96 text],
+    9728 stacked rows with eight segments.  The linears and the attention are checked on the rows next
+    to every segment boundary, the first and last rows of the 192-token tiles around them and an even
+    spread (every 512th row); the element-wise glue on every row."""
+    shape = synth.LLAMA_8B
+    seqs = [synth.config4_sequence()] * 4
+    L = seqs[0].shape[0]
+    rows = set(range(0, 4 * L, 512)) | {4 * L - 1}
+    for b in range(4):
+        for e in (b * L, b * L + 2304, (b + 1) * L):
+            rows |= {r for r in (e - 2, e - 1, e, e + 1) if 0 <= r < 4 * L}
+    for t0 in range(0, 4 * L, 192 * 8):
+        rows |= {t0, min(4 * L - 1, t0 + 191)}
+    _check_batched_block(shape, seqs, 71, rows=np.array(sorted(rows)))
 
 
 def test_causal_glue_matches_the_unified_mask():

@@ -225,12 +225,18 @@ def _check_linear(case, bias=None, clipping_expected=None):
     mag = np.abs(O.dequant(ref["acc"], ref["s_rows"], sw_ref)) + (0 if bias is None else np.abs(bias)[None, :])
     nz = mag > 0
     assert (np.abs(y32 - ref["y64"])[nz] / mag[nz]).max() <= 1e-5
-    # bf16 out (the product configuration): within 1e-2 of float64, and equal to the oracle's bf16
+    # bf16 out with the accumulator dump: within 1e-2 of float64, and equal to the oracle's bf16
     yb, acc2, st = gpu_linear(case, s_v, s_t, layout, s_w, bias, torch.bfloat16)
     assert st == (B.MQ_OK, 0)
     yb = bf16_from_dev(yb)
     assert np.array_equal(yb, ref["y_bf16"])
     assert (np.abs(yb - ref["y64"])[nz] / mag[nz]).max() <= 1e-2
+    # the product configuration (bf16 out, no dump: the epilogue with 16-byte stores), and the same
+    # with a row pitch that is not a multiple of 16 bytes (falls back to per-element stores)
+    for y_pad in (0, 4):
+        yp, _, st = gpu_linear(case, s_v, s_t, layout, s_w, bias, torch.bfloat16, want_acc=False, y_pad=y_pad)
+        assert st == (B.MQ_OK, 0)
+        assert np.array_equal(bf16_from_dev(yp), ref["y_bf16"]), y_pad
     # pre-quantized entry (X already int8) gives the same accumulators
     y3, acc3, st = gpu_linear(case, s_v, s_t, layout, s_w, bias, torch.bfloat16, x_codes=q)
     assert st == (B.MQ_OK, 0) and torch.equal(acc3, acc2)
@@ -251,12 +257,12 @@ def test_config1_full():
     (70, 0, 256, 128, 64),         # no text rows
     (1, 0, 32, 16, 32),            # the smallest legal problem
     (250, 263, 160, 144, 32),      # K not a multiple of the K block; two token tiles
-    (3, 5, 4096, 256, 128),        # T = 8: streaming variant (tokens as MMA rows), split-K slices
-    (5, 8, 160, 144, 32),          # T = 13: streaming, ragged K block, one half-empty 256-channel tile
-    (0, 27, 1152, 272, 128),       # T = 27: streaming, two channel tiles, the second one ragged
-    (20, 13, 2048, 128, 0),        # T = 33: streaming, tokens in two epilogue warps
-    (100, 28, 4096, 512, 1024),    # T = 128: the largest streaming problem, split-K
-    (100, 29, 1024, 384, 0),       # T = 129: smallest problem of the channel-row variant
+    (3, 5, 4096, 256, 128),        # T = 8: one 16-token tile, split-K slices + finalize kernel
+    (5, 8, 160, 144, 32),          # T = 13: ragged K block, second channel tile mostly empty
+    (0, 27, 1152, 272, 128),       # T = 27: three channel tiles, the last one ragged
+    (20, 13, 2048, 128, 0),        # T = 33: a 48-token tile, three 16-column epilogue chunks
+    (100, 28, 4096, 512, 1024),    # T = 128: the largest decode-shaped problem, split-K
+    (100, 29, 1024, 384, 0),       # T = 129: just past the decode-shaped range
 ])
 def test_linear_edge_shapes(T_vis, T_txt, K, N, rot):
     c = synth.small_linear(100 + K + N, T_vis, T_txt, K, N, rot, calib_vis=24, calib_txt=8)
@@ -318,6 +324,24 @@ def test_linear_clipping_variant():
     # calibration without the massive tokens: the quantizer must saturate on them
     c = synth.config2(seed=1, T_vis=96, T_txt=32, K=1024, N=128, clipping_variant=True)
     _check_linear(c, clipping_expected=True)
+
+
+def test_config2_clipping_variant_full_size_sampled():
+    """The clipping variant at the size of config 2: the calibration draw has no massive-activation
+    token, so the two massive rows of the batch saturate; codes of the whole batch against the
+    oracle, the product on the sampled rows (which include both massive rows)."""
+    c = synth.config2(clipping_variant=True)
+    s_v, s_t = gpu_calibrate(c.x_calib, c.seg_calib, c.rot_block)
+    o_v, o_t = O.calibrate_static_scales(c.x_calib, c.seg_calib.seg_end, c.seg_calib.seg_mod, c.rot_block)
+    assert (s_v, s_t) == (o_v, o_t)
+    q = torch.empty((c.T, c.K), dtype=torch.int8, device=DEV)
+    B.mq_fwht_quant_i8(bf16_to_dev(c.x), dev_segments(c.seg), s_v, s_t, c.rot_block, q, None)
+    q_ref = O.quantize_act_int8(O.fwht_blocks(c.x, c.rot_block, np.float32),
+                                O.row_scales(c.T, c.seg.seg_end, c.seg.seg_mod, s_v, s_t))
+    assert np.array_equal(q.cpu().numpy(), q_ref)
+    sat = (q_ref == -128) | (q_ref == 127)
+    assert sat.any() and set(np.flatnonzero(sat.any(axis=1)).tolist()) >= set(c.meta["massive_rows"])
+    _check_full_size_sampled(c, tile_rows=224)
 
 
 @pytest.mark.parametrize("T,K,N", [(128, 13696, 512), (8, 4096, 1024), (600, 2048, 640), (3, 13696, 4096)])
@@ -388,6 +412,9 @@ def test_config2_full_size_sampled():
     assert _rel(bf16_from_dev(yb)[rows], ref["y64"])[nz].max() <= 1e-2
     # property that holds at any size: every accumulator obeys |acc| <= 128 * 8 * K
     assert int(acc.abs().max()) <= 128 * 8 * c.K
+    # the launch the benchmark times (no accumulator dump: 16-byte stores) writes the same bits everywhere
+    yp, _, st = gpu_linear(c, s_v, s_t, layout, s_w, None, torch.bfloat16, want_acc=False)
+    assert st == (B.MQ_OK, 0) and torch.equal(yp.view(torch.int16), yb.view(torch.int16))
 
 
 def _check_full_size_sampled(c, tile_rows, n_sample=24):
@@ -423,6 +450,9 @@ def _check_full_size_sampled(c, tile_rows, n_sample=24):
     nz = np.abs(ref["y64"]) > 0
     assert _rel(bf16_from_dev(yb)[rows], ref["y64"])[nz].max() <= 1e-2
     assert int(acc.abs().max()) <= 128 * 8 * c.K
+    # the launch the benchmark times (no accumulator dump: 16-byte stores) writes the same bits everywhere
+    yp, _, st = gpu_linear(c, s_v, s_t, layout, s_w, None, torch.bfloat16, want_acc=False)
+    assert st == (B.MQ_OK, 0) and torch.equal(yp.view(torch.int16), yb.view(torch.int16))
 
 
 @pytest.mark.parametrize("which", ["k_proj", "down_proj"])
@@ -432,11 +462,12 @@ def test_config3_linears_full_size_sampled(which):
     _check_full_size_sampled(synth.config3_linear(which), tile_rows=192)
 
 
-@pytest.mark.parametrize("which", ["q_proj", "down_proj"])
+@pytest.mark.parametrize("which", ["q_proj", "k_proj", "v_proj", "o_proj", "gate_proj", "up_proj", "down_proj"])
 def test_config4_linears_full_size_sampled(which):
-    """8B-shaped block, batch of 4 sequences flattened to 9728 rows with 8 segments."""
+    """8B-shaped block, batch of 4 sequences flattened to 9728 rows with 8 segments: all seven linears
+    (gate / up are the deepest persistent loop: 112 channel tiles x 51 token tiles)."""
     c = synth.config4_linear(which)
-    assert c.seg.n_seg == 8
+    assert c.seg.n_seg == 8 and c.T == 9728
     _check_full_size_sampled(c, tile_rows=192)
 
 
