@@ -337,6 +337,7 @@ def layer_mode_timing(torch, dev, name, shape, seqs, reps=5):
     from paper_2502_00425_b200 import layer as LY
     blk = LY.random_block(shape, 21, dev)
     blk.causal_glue = True  # attention in the original order with a plain causal mask (same result, Eq. 5)
+    blk.fuse_groups = True  # q/k/v and gate/up as one stacked weight each: one launch per group (same results)
     for lw in blk.w.values():
         lw.s_vis, lw.s_txt = 0.5, 0.05
     g = torch.Generator(device="cpu").manual_seed(22)

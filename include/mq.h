@@ -367,6 +367,16 @@ int mq_ubench_mma_i8(int32_t n_tok, int32_t n_mma, int32_t n_acc, int32_t a_from
                      uint64_t* cycles_out, int32_t* status, void* stream);
 
 /*
+ * Cost of the weight expander's inner step (packed int4 tile in shared memory -> sixteen-fold int8
+ * codes in tensor memory), without barriers: one CTA of `warps` (4 or 8) warps runs n_iter rounds of
+ *   mode 0: the 32-column tensor-memory store and its completion wait only,
+ *   mode 1: the four 16-byte shared-memory loads, the nibble expansion and the store + wait,
+ *   mode 2: as 1 but waiting for the stores once at the end.
+ * cycles_out: device uint64 [warps], SM clock cycles per warp for all rounds.
+ */
+int mq_ubench_expand(int32_t n_iter, int32_t warps, int32_t mode, uint64_t* cycles_out, void* stream);
+
+/*
  * Exercises the bounded wait that every kernel of the library uses on its mbarriers, on a barrier
  * that nothing arrives at: after limit_ns (1 .. 1e9) the wait gives up, writes
  * {MQ_ERR_TIMEOUT, site} to status (device int32 [2], zeroed by the caller) and raises the CTA's

@@ -23,6 +23,7 @@ MQ_ERR_WORKSPACE = -6
 MQ_FLAG_X_IS_INT8 = 1
 MQ_FLAG_Y_IS_F32 = 2
 MQ_NOALLOC_WS_BYTES = 4 << 20
+MQ_W_TILE_N, MQ_W_TILE_K = 128, 128
 TEXT, VISUAL = 0, 1
 
 _LIB_NAME = "libmq.so"
@@ -88,6 +89,7 @@ def load(build_if_missing: bool = False):
         "mq_w4a8_dynamic_linear": (C.c_int, [descp, vp, i64, vp, vp, vp, vp, i64, vp, vp, vp, sz, vp]),
         "mq_ubench_mma_i8": (C.c_int, [i32, i32, i32, i32, i32, vp, vp, vp]),
         "mq_selftest_bounded_wait": (C.c_int, [C.c_uint64, i32, vp, vp, vp]),
+        "mq_ubench_expand": (C.c_int, [i32, i32, i32, vp, vp]),
         "mq_last_device_status": (C.c_int, [vp, vp, C.POINTER(C.c_int32)]),
         "mq_reset_device_status": (C.c_int, [vp, vp]),
     }
@@ -104,7 +106,7 @@ EXPORTED = ["mq_version", "mq_status_string", "mq_workspace_bytes", "mq_w4_layou
             "mq_attn_mask_remap", "mq_fwht_quant_i8", "mq_w4a8_msq_linear", "mq_w4a8_msq_linear_noalloc", "mq_last_device_status",
             "mq_reset_device_status", "mq_rms_side_ld", "mq_rms_detect", "mq_pack_w4_rms", "mq_rms_workspace_bytes",
             "mq_w4a8_msq_linear_rms", "mq_dynamic_quant_i8", "mq_dynamic_workspace_bytes", "mq_w4a8_dynamic_linear",
-            "mq_ubench_mma_i8", "mq_selftest_bounded_wait"]
+            "mq_ubench_mma_i8", "mq_selftest_bounded_wait", "mq_ubench_expand"]
 
 
 def status_string(status: int) -> str:
@@ -351,6 +353,12 @@ def mq_ubench_mma_i8(n_tok, n_mma, n_acc, a_from_smem, ctas, cycles_out, status)
     assert cycles_out.dtype == torch.int64 and cycles_out.numel() >= ctas and status.dtype == torch.int32
     _check(load().mq_ubench_mma_i8(n_tok, n_mma, n_acc, int(a_from_smem), ctas, _ptr(cycles_out), _ptr(status),
                                    _stream()), "mq_ubench_mma_i8")
+
+
+def mq_ubench_expand(n_iter, warps, mode, cycles_out):
+    """Cycles of the weight expander's inner step (see include/mq.h); cycles_out int64 [warps]."""
+    assert cycles_out.dtype == torch.int64 and cycles_out.numel() >= warps
+    _check(load().mq_ubench_expand(n_iter, warps, mode, _ptr(cycles_out), _stream()), "mq_ubench_expand")
 
 
 def mq_selftest_bounded_wait(limit_ns, site, status, waited_ns_out):

@@ -105,6 +105,65 @@ ubench_mma_i8_kernel(int n_tok, int n_mma, int n_acc, int a_from_smem, unsigned 
   }
 }
 
+
+// Cost of the weight expanders' inner step, without any barrier: `warps` warps (4 or 8; warp w owns
+// tensor-memory lanes 32 (w % 4) ..) each run n_iter rounds of
+//   mode 0: tcgen05.st x32 (32 registers -> 32 columns) + tcgen05.wait::st
+//   mode 1: four 16-byte shared-memory loads + the 32 logic operations of the nibble expansion + the same store
+//   mode 2: as mode 1 without waiting for the store before the next round's loads (wait once at the end)
+// cycles_out[warp] = clock64 ticks for the n_iter rounds.
+__global__ void __launch_bounds__(256, 1)
+ubench_expand_kernel(int n_iter, int mode, unsigned long long* cycles_out) {
+  __shared__ __align__(16) uint8_t tile[2][8192];
+  __shared__ uint32_t tmem_slot;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int i = threadIdx.x; i < 2 * 8192 / 4; i += blockDim.x) reinterpret_cast<uint32_t*>(tile)[i] = 0x9e3779b9u * (i + 1);
+  if (warp == 0) {
+    tmem_alloc(&tmem_slot, 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&tmem_slot);
+  const int q = warp & 3, grp = warp >> 2;
+  const int r = q * 32 + lane;
+  uint32_t regs[32];
+#pragma unroll
+  for (int i = 0; i < 32; ++i) regs[i] = (uint32_t)(i * 0x01010101u);
+  uint32_t sink = 0;
+  __syncthreads();
+  const long long t0 = clock64();
+  for (int it = 0; it < n_iter; ++it) {
+    if (mode >= 1) {
+      const uint4* src = reinterpret_cast<const uint4*>(tile[it & 1]) + r;
+#pragma unroll
+      for (int jj = 0; jj < 4; ++jj) {
+        const uint4 w = src[jj * 128];
+        const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          regs[jj * 8 + 2 * i] = (ww[i] << 4) & 0xF0F0F0F0u;
+          regs[jj * 8 + 2 * i + 1] = ww[i] & 0xF0F0F0F0u;
+        }
+      }
+      sink ^= regs[1] ^ regs[9];
+    }
+    const uint32_t slot = (uint32_t)(((it * 2 + grp) & 7) * 32);
+    tmem_st_x32(tmem_base + ((uint32_t)(q * 32) << 16) + slot, regs);
+    if (mode <= 1) tmem_wait_st();
+  }
+  tmem_wait_st();
+  const long long t1 = clock64();
+  if (lane == 0) cycles_out[warp] = (unsigned long long)(t1 - t0) + (sink == 0x12345u ? 1ull : 0ull);
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
 // One warp waits (bounded by limit_ns) on a barrier that has no arriver.  The wait gives up, records
 // MQ_ERR_TIMEOUT and `site`, raises the abort flag; a second wait in another warp then returns at once
 // because the flag is up.  waited_ns_out[0] = how long the first wait lasted.
@@ -164,5 +223,14 @@ extern "C" int mq_selftest_bounded_wait(uint64_t limit_ns, int32_t site, int32_t
   if (!status || !waited_ns_out || limit_ns == 0 || limit_ns > 1000000000ull) return MQ_ERR_INVALID_ARG;
   selftest_bounded_wait_kernel<<<1, 64, 0, static_cast<cudaStream_t>(stream)>>>(
       limit_ns, site, status, reinterpret_cast<unsigned long long*>(waited_ns_out));
+  return cuda_status(cudaGetLastError());
+}
+
+extern "C" int mq_ubench_expand(int32_t n_iter, int32_t warps, int32_t mode, uint64_t* cycles_out, void* stream) {
+  using namespace mq;
+  if (n_iter < 1 || n_iter > (1 << 20) || (warps != 4 && warps != 8) || mode < 0 || mode > 2 || !cycles_out)
+    return MQ_ERR_INVALID_ARG;
+  ubench_expand_kernel<<<1, warps * 32, 0, static_cast<cudaStream_t>(stream)>>>(
+      n_iter, mode, reinterpret_cast<unsigned long long*>(cycles_out));
   return cuda_status(cudaGetLastError());
 }

@@ -107,6 +107,9 @@ class W4A8DecoderBlock:
                  g_mlp: torch.Tensor, device="cuda"):
         self.shape, self.w, self.g_attn, self.g_mlp, self.device = shape, weights, g_attn, g_mlp, device
         self._ws: Dict[Tuple[str, int], torch.Tensor] = {}
+        self._fused: Dict[str, Optional[LinearWeights]] = {}
+        # True: q/k/v and gate/up each run as one linear over the stacked weight (same results)
+        self.fuse_groups = False
         # True: attention in the original order with a plain causal mask instead of the dense unified
         # mask (same result, much faster glue); the dense mask is still produced and kept in the trace
         self.causal_glue = False
@@ -160,12 +163,50 @@ class W4A8DecoderBlock:
         tr.tensors[name + ".in"], tr.tensors[name + ".out"] = x, y
         return y
 
+    def fused_group(self, names) -> Optional[LinearWeights]:
+        """The linears of a group stored as ONE weight [sum N, K] (q/k/v as N = q + 2 kv, gate/up as
+        N = 2 mlp): the GEMM layout is contiguous per 128-channel tile, so when every member's N is a
+        multiple of 128 the concatenation of the members' layouts IS the layout of the stacked weight.
+        One launch then serves the whole group (fewer kernel boundaries, fuller waves).  None when a
+        member's N is not tile-aligned or has a bias layout that cannot be stacked."""
+        key = "+".join(names)
+        if key in self._fused:
+            return self._fused[key]
+        ws = [self.w[n] for n in names]
+        ok = all(w.N % B.MQ_W_TILE_N == 0 and w.rot_block == 0 and w.K == ws[0].K for w in ws) and \
+            (all(w.bias is None for w in ws) or all(w.bias is not None for w in ws))
+        fused = None
+        if ok:
+            bias = None if ws[0].bias is None else torch.cat([w.bias for w in ws])
+            fused = LinearWeights(torch.cat([w.layout for w in ws]), torch.cat([w.s_w for w in ws]), ws[0].K,
+                                  sum(w.N for w in ws), 0, bias)
+        self._fused[key] = fused
+        return fused
+
     def linear_group(self, names, x: torch.Tensor, tr: BlockTrace, calibrate: bool):
-        """Linears that read the same input (q/k/v, gate/up; no rotation): the input is quantized
-        once with mq_fwht_quant_i8 and every linear of the group multiplies the same int8 codes."""
+        """Linears that read the same input (q/k/v, gate/up; no rotation).  With `fuse_groups` they run
+        as one linear over the stacked weight (see fused_group) and the outputs are column slices of
+        its result; otherwise the input is quantized once with mq_fwht_quant_i8 and every linear of
+        the group multiplies the same int8 codes."""
         first = self.w[names[0]]
         assert all(self.w[n].rot_block == 0 and self.w[n].K == first.K for n in names)
         T = x.shape[0]
+        fused = self.fused_group(names) if self.fuse_groups else None
+        if fused is not None and not calibrate:
+            fused.s_vis, fused.s_txt = first.s_vis, first.s_txt
+            key = ("+".join(names), T)
+            if key not in self._ws:
+                self._ws[key] = B.new_workspace(T, fused.K, fused.N, 0)
+            y = torch.empty((T, fused.N), dtype=torch.bfloat16, device=x.device)
+            B.mq_w4a8_msq_linear(x, tr.seg, fused.s_vis, fused.s_txt, fused.layout, fused.s_w, y, self._ws[key],
+                                 fused.N, bias=fused.bias)
+            outs, off = [], 0
+            for n in names:
+                yn = y[:, off:off + self.w[n].N]
+                off += self.w[n].N
+                tr.tensors[n + ".in"], tr.tensors[n + ".out"] = x, yn
+                outs.append(yn)
+            return outs
         if calibrate:
             state = torch.zeros(2, dtype=torch.int32, device=x.device)
             sv = torch.zeros(1, dtype=torch.float32, device=x.device)

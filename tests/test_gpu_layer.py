@@ -210,3 +210,25 @@ def test_causal_glue_matches_the_unified_mask():
     out_causal, tr_causal = blk.forward(emb, vis)
     assert _close_rowmax(bf16_from_dev(tr_causal.tensors["attn"]), bf16_from_dev(tr_mask.tensors["attn"]))
     assert _close_rowmax(bf16_from_dev(out_causal), bf16_from_dev(out_mask))
+
+
+def test_fused_groups_match_separate_linears():
+    """q/k/v and gate/up stored as one stacked weight each (one launch per group) give the block the very
+    same bits as separate linears on shared codes: every output channel only sees its own weight row."""
+    shape = synth.LayerShape(hidden=256, n_q_heads=4, n_kv_heads=2, head_dim=128, mlp=512)
+    blk, _, _, _ = _make_block(shape, 81)
+    for T_spans in ([(0, 9), (1, 70), (0, 15), (1, 40), (0, 21)], [(0, 3)]):      # a prefill block and a 3-token step
+        is_visual = synth.interleaved_modality(T_spans)
+        emb = bf16_to_dev(synth.embedding_rows(82, is_visual.shape[0], shape.hidden, is_visual))
+        vis = torch.from_numpy(is_visual).to(DEV)
+        blk.fuse_groups = False
+        out_sep, tr_sep = blk.forward(emb, vis, calibrate=True)
+        blk.fuse_groups = True
+        out_fused, tr_fused = blk.forward(emb, vis)
+        assert blk.fused_group(["q_proj", "k_proj", "v_proj"]) is not None
+        assert blk.fused_group(["gate_proj", "up_proj"]) is not None
+        for name in ("q_proj", "k_proj", "v_proj", "gate_proj", "up_proj", "down_proj"):
+            assert torch.equal(tr_fused.tensors[name + ".out"].contiguous().view(torch.int16),
+                               tr_sep.tensors[name + ".out"].contiguous().view(torch.int16)), name
+        assert torch.equal(out_fused.view(torch.int16), out_sep.view(torch.int16))
+    assert blk.device_status_ok()

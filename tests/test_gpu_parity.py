@@ -328,8 +328,8 @@ def test_linear_clipping_variant():
 
 def test_config2_clipping_variant_full_size_sampled():
     """The clipping variant at the size of config 2: the calibration draw has no massive-activation
-    token, so the two massive rows of the batch saturate; codes of the whole batch against the
-    oracle, the product on the sampled rows (which include both massive rows)."""
+    token, so the quantizer saturates; codes of the whole batch against the oracle, the product on
+    the sampled rows (which include both massive rows)."""
     c = synth.config2(clipping_variant=True)
     s_v, s_t = gpu_calibrate(c.x_calib, c.seg_calib, c.rot_block)
     o_v, o_t = O.calibrate_static_scales(c.x_calib, c.seg_calib.seg_end, c.seg_calib.seg_mod, c.rot_block)
@@ -339,12 +339,19 @@ def test_config2_clipping_variant_full_size_sampled():
     q_ref = O.quantize_act_int8(O.fwht_blocks(c.x, c.rot_block, np.float32),
                                 O.row_scales(c.T, c.seg.seg_end, c.seg.seg_mod, s_v, s_t))
     assert np.array_equal(q.cpu().numpy(), q_ref)
-    sat = (q_ref == -128) | (q_ref == 127)
-    assert sat.any() and set(np.flatnonzero(sat.any(axis=1)).tolist()) >= set(c.meta["massive_rows"])
+    # with the massive tokens left out of the calibration draw both clamp branches are taken (the rotation
+    # spreads a massive channel over its block, so it is not necessarily the massive rows that saturate)
+    assert (q_ref == -128).any() and (q_ref == 127).any()
     _check_full_size_sampled(c, tile_rows=224)
 
 
-@pytest.mark.parametrize("T,K,N", [(128, 13696, 512), (8, 4096, 1024), (600, 2048, 640), (3, 13696, 4096)])
+@pytest.mark.parametrize("T,K,N", [(128, 13696, 512), (8, 4096, 1024), (600, 2048, 640), (3, 13696, 4096),
+                                   # the decode shapes of config 5 (gate / up and down) over the decode range of T
+                                   (5, 4096, 13696), (16, 4096, 13696), (64, 4096, 13696), (128, 4096, 13696),
+                                   (5, 13696, 4096), (16, 13696, 4096), (64, 13696, 4096), (128, 13696, 4096),
+                                   (8, 4096, 27392),      # gate and up as one weight: more channel tiles than SMs
+                                   (24, 96, 4096),        # one K block per channel tile
+                                   (16, 13696, 256)])     # two channel tiles, 107 K blocks: many K splits
 def test_repeated_launches_give_identical_accumulators(T, K, N):
     """A race in the producer / expander / MMA pipeline shows as a result that changes from launch
     to launch.  Exact integer reference (int8 x int4 codes, float64 matmul is exact here), the
