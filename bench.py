@@ -461,7 +461,7 @@ class BufferSet:
 # dram__bytes_read.sum + dram__bytes_write.sum of one w4a8_gemm_kernel launch on this workload
 # (ncu capture summarised in profiles/); None once the kernel has changed since the capture.
 GEMM_TRAFFIC_BYTES = 57.43e6
-LAUNCHES_PER_STEP = 5  # index scan, row gather, remap, rotation+quantizer, GEMM
+LAUNCHES_PER_STEP = 4  # fused AIFS index + gather, remap, rotation + quantizer, GEMM
 
 
 def run_ours(args, info):
@@ -520,16 +520,41 @@ def run_ours(args, info):
 
     kernels = [k_aifs, k_remap, k_quant, k_gemm]
 
+    branch = torch.cuda.Stream()
+
+    def k_index(s):
+        B.mq_aifs_reorder(None, None, s.is_vis, None, s.perm, s.inv, s.n_first, 0, L=case.T)
+
+    def k_gather(s):  # X_out[inv[i]] = X[i], i.e. X_out[j] = X[perm[j]]: the gather, from the finished index arrays
+        B.mq_aifs_reorder(s.emb, s.emb_u, None, None, s.inv, None, None, 1)
+
     def step(s, events=None):
         """One pass of the hot path.  The linear is issued as its two kernels (the quantizer into
         a caller-owned code buffer, then the GEMM on the codes), which is exactly what
-        mq_w4a8_msq_linear does with its workspace, so that events can sit between them."""
-        for i, k in enumerate(kernels):
+        mq_w4a8_msq_linear does with its workspace, so that events can sit between them.
+        Dependencies: the quantizer reads the segment table that the remap writes, and the remap
+        reads the permutation; the row gather of the embeddings needs the permutation only.  The
+        timed step therefore issues index -> remap -> quantizer -> GEMM in line and the row gather
+        as a second branch behind the index kernel (fork and join with events; in a captured graph
+        a parallel branch).  With timing events between the kernels (or --serial-step) the fused
+        index + gather kernel runs in line instead: four launches."""
+        if events is not None or args.serial_step:
+            for i, k in enumerate(kernels):
+                if events is not None:
+                    events[i].record()
+                k(s)
             if events is not None:
-                events[i].record()
-            k(s)
-        if events is not None:
-            events[len(kernels)].record()
+                events[len(kernels)].record()
+            return
+        main = torch.cuda.current_stream()
+        k_index(s)
+        branch.wait_stream(main)
+        with torch.cuda.stream(branch):
+            k_gather(s)
+        k_remap(s)
+        k_quant(s)
+        k_gemm(s)
+        main.wait_stream(branch)
 
     # ---- CUDA graphs: one per buffer set, so that the host only replays.  A second family of
     # graphs of the same step carries timing events recorded as graph nodes ("external" events)
@@ -746,13 +771,15 @@ def run_ours(args, info):
             "scaling": "weak", "vs_baseline": None, "dtype": "int8xint4->int32", "data": "synthetic",
             "config": {"workload": WORKLOAD, "launch": launch_mode,
                        "l2": "inputs larger than L2: %d buffer sets, %.0f MB cycled" % (n_sets, footprint / 1e6),
-                       "step": "aifs_reorder + mask_remap + fwht_quant_i8 + w4a8 gemm",
+                       "step": "aifs_reorder + mask_remap + fwht_quant_i8 + w4a8 gemm"
+                               + ("" if args.serial_step else " (index -> remap -> quantizer -> GEMM in line, the row "
+                                  "gather as a parallel branch behind the index kernel)"),
                        "tokens_per_s": (T_VIS + T_TXT) * args.steps * info.world / t_max},
             "clocks": clocks,
             "e2e": {"value": e2e_ops / 1e12, "unit": UNIT, "h2d_bytes_per_step": case.T * case.K * 2,
                     "d2h_bytes_per_step": case.T * case.N * 2, "steps": e2e_steps,
                     "overlap": "copy-in, compute and copy-out of neighbouring steps on three streams"},
-            "gpu_launches": LAUNCHES_PER_STEP * args.steps,
+            "gpu_launches": (LAUNCHES_PER_STEP if args.serial_step else LAUNCHES_PER_STEP + 1) * args.steps,
             "roofline": {"bound": "tensor", "kernel": "w4a8_gemm_kernel", "achieved": gemm_tops, "peak": peak,
                          "unit": "TOP/s", "frac": gemm_tops / peak,
                          "peak_kind": "2 x measured bf16 %s (%s)" % ("sustained" if sustained else "burst",
@@ -789,6 +816,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--buffer-sets", type=int, default=4)
     ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--serial-step", action="store_true",
+                    help="issue the four kernels of a step in one line instead of two parallel branches")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-decode", action="store_true")
     ap.add_argument("--decode-only", action="store_true",

@@ -285,6 +285,105 @@ def linear_w4a8_msq(x, seg_end, seg_mod, s_vis, s_txt, rot_block, qw, s_w, bias=
             "y_bf16": bf16_rne(y32)}
 
 
+# ----------------------------------------------------------------------------- other bit widths and weight groups
+def quantize_weight_sym(w, bits: int = 4, group: int = 0):
+    """Eq. 2 with z = 0 for a general weight bit-width b and scale granularity: qmax = 2^(b-1) - 1,
+    s = max|w| / qmax over one output channel (group = 0) or over each run of `group` consecutive
+    input channels of it (the group-wise W4 of the weight-only comparison, App. A.12: g = 128),
+    codes clamp to [-2^(b-1), qmax]; literal division (offline).  W8 is the weight side of the W8A8
+    rows of the main results table (Sec. 4.1).
+    Returns (codes int8 [N, K], scales float32 [N] or [N, K / group])."""
+    w = np.asarray(w, dtype=np.float32)
+    N, K = w.shape
+    qmax = np.float32(2 ** (bits - 1) - 1)
+    if group:
+        assert K % group == 0
+        blocks = w.reshape(N, K // group, group)
+        m = np.max(np.abs(blocks), axis=2).astype(np.float32)
+        s = np.where(m > 0, m / qmax, np.float32(1.0)).astype(np.float32)
+        q = np.rint((blocks / s[:, :, None]).astype(np.float32)).reshape(N, K)
+    else:
+        m = np.max(np.abs(w), axis=1).astype(np.float32)
+        s = np.where(m > 0, m / qmax, np.float32(1.0)).astype(np.float32)
+        q = np.rint((w / s[:, None]).astype(np.float32))
+    return np.clip(q, -(2 ** (bits - 1)), 2 ** (bits - 1) - 1).astype(np.int8), s
+
+
+def quantize_act_sym(r, s_rows, bits: int = 8) -> np.ndarray:
+    """quantize_act_int8 for a general activation bit-width: same reciprocal-multiply and
+    round-half-even, clamp to [-2^(b-1), 2^(b-1) - 1].  b = 4 is the activation side of the
+    W4A4 rows of the main results table (Sec. 4.1); the codes still travel as int8."""
+    r = np.asarray(r, dtype=np.float32)
+    s_rows = np.asarray(s_rows, dtype=np.float32).reshape(-1, 1)
+    inv = (np.float32(1.0) / s_rows).astype(np.float32)
+    with np.errstate(invalid="ignore", over="ignore"):
+        q = np.rint((r * inv).astype(np.float32))
+    q = np.where(np.isnan(q), 0.0, q)
+    return np.clip(q, -(2 ** (bits - 1)), 2 ** (bits - 1) - 1).astype(np.int8)
+
+
+def calibrate_static_scales_bits(x_calib, seg_end, seg_mod, rot_block: int, bits: int = 8):
+    """calibrate_static_scales with Eq. 2's denominator 2^(b-1) - 1 for b-bit activations."""
+    x_calib = np.asarray(x_calib, dtype=np.float32)
+    r = fwht_blocks(x_calib, rot_block, np.float32)
+    mod = row_modality(x_calib.shape[0], seg_end, seg_mod)
+    qmax = 2 ** (bits - 1) - 1
+    return static_scale(r[mod == VISUAL], qmax), static_scale(r[mod == TEXT], qmax)
+
+
+def int_gemm_grouped(qx, qw, group: int) -> np.ndarray:
+    """Partial sums per weight group: acc[t, n, g] = sum over the group's input channels."""
+    qx = np.asarray(qx)
+    qw = np.asarray(qw)
+    T, K = qx.shape
+    N = qw.shape[0]
+    G = K // group
+    out = np.empty((T, N, G), dtype=np.int32)
+    for g in range(G):
+        out[:, :, g] = int_gemm(qx[:, g * group:(g + 1) * group], qw[:, g * group:(g + 1) * group])
+    return out
+
+
+def dequant_grouped(acc_g, s_rows, s_wg, bias=None, dtype=np.float64) -> np.ndarray:
+    """y[t,n] = sum_g acc[t,n,g] * (s_a(t) * s_w[n,g]) (+ bias[n]).  dtype=float32 fixes the rounding
+    order: for g = 0, 1, ...: y <- fl(y + fl(float(acc_g) * fl(s_a * s_w[n,g]))), so that one group
+    reproduces dequant() bit for bit."""
+    acc_g = np.asarray(acc_g)
+    T, N, G = acc_g.shape
+    s_rows = np.asarray(s_rows, dtype=np.float32).astype(dtype).reshape(-1, 1)
+    s_wg = np.asarray(s_wg, dtype=np.float32).astype(dtype).reshape(N, G)
+    y = np.zeros((T, N), dtype=dtype)
+    for g in range(G):
+        c = (s_rows * s_wg[None, :, g]).astype(dtype)
+        y = (y + (acc_g[:, :, g].astype(dtype) * c).astype(dtype)).astype(dtype)
+    if bias is not None:
+        y = (y + np.asarray(bias, dtype=np.float32).astype(dtype).reshape(1, -1)).astype(dtype)
+    return y
+
+
+def linear_wa_sym(x, seg_end, seg_mod, s_vis, s_txt, rot_block, qw, s_w, act_bits: int = 8, group: int = 0,
+                  bias=None):
+    """linear_w4a8_msq generalised to the neighbouring settings: b-bit static MSQ activations
+    (codes from quantize_act_sym), weight codes of any width (the integer product does not care),
+    and per-channel (group = 0) or group-wise weight scales."""
+    x = np.asarray(x, dtype=np.float32)
+    T = x.shape[0]
+    r = fwht_blocks(x, rot_block, np.float32)
+    s_rows = row_scales(T, seg_end, seg_mod, s_vis, s_txt)
+    qx = quantize_act_sym(r, s_rows, act_bits)
+    if group:
+        acc_g = int_gemm_grouped(qx, qw, group)
+        y64 = dequant_grouped(acc_g, s_rows, s_w, bias, np.float64)
+        y32 = dequant_grouped(acc_g, s_rows, s_w, bias, np.float32)
+        return {"rotated": r, "s_rows": s_rows, "qx": qx, "acc_g": acc_g, "y64": y64, "y32": y32,
+                "y_bf16": bf16_rne(y32)}
+    acc = int_gemm(qx, qw)
+    y64 = dequant(acc, s_rows, s_w, bias, np.float64)
+    y32 = dequant(acc, s_rows, s_w, bias, np.float32)
+    return {"rotated": r, "s_rows": s_rows, "qx": qx, "acc": acc, "y64": y64, "y32": y32,
+            "y_bf16": bf16_rne(y32)}
+
+
 # ----------------------------------------------------------------------------- AIFS
 def aifs_perm(is_visual, is_pad=None) -> np.ndarray:
     """AIFS order (Sec. 3.1; App. A.2: AIFS(1..L) = (m..n, 1..m-1, n+1..L)):

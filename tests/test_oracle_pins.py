@@ -577,3 +577,114 @@ def test_reciprocal_and_literal_division_report():
         print("A4 %(config)s: %(differ)d of %(codes)d codes differ (rows checked: %(rows)d)" % row)
         assert row["max_abs_code_diff"] <= 1
         assert row["differ"] <= 1e-4 * row["codes"]
+
+
+# ----------------------------------------------------------------------------- other bit widths, weight groups
+def test_weight_quantizer_general_reduces_to_the_int4_per_channel_one():
+    rng = np.random.default_rng(21)
+    w = (rng.standard_normal((24, 256)) * 0.03).astype(np.float32)
+    w[5] = 0.0
+    q4, s4 = O.quantize_weight_int4(w)
+    q, s = O.quantize_weight_sym(w, 4, 0)
+    assert np.array_equal(q, q4) and np.array_equal(s, s4)
+    # one group spanning all of K is the per-channel quantizer
+    qg, sg = O.quantize_weight_sym(w, 4, 256)
+    assert np.array_equal(qg, q4) and np.array_equal(sg[:, 0], s4) and sg.shape == (24, 1)
+
+
+def test_grouped_weight_quantizer_hand_rows():
+    # two groups of four with very different ranges: Eq. 2 per group, b = 4 (qmax 7)
+    w = np.array([[7.0, -3.5, 1.0, 0.0, 0.07, -0.035, 0.01, 0.0],
+                  [0.0, 0.0, 0.0, 0.0, -14.0, 14.0, 2.0, 1.0]], np.float32)
+    q, s = O.quantize_weight_sym(w, 4, 4)
+    assert np.array_equal(s, np.array([[1.0, np.float32(0.07) / np.float32(7)], [1.0, 2.0]], np.float32))
+    #  -3.5 / 1 -> tie -> -4 (even);  -0.035 / 0.01 = -3.5 up to rounding of the scale: checked by value below
+    assert q[0, :4].tolist() == [7, -4, 1, 0]
+    assert q[1].tolist() == [0, 0, 0, 0, -7, 7, 1, 0]            # 1 / 2 = 0.5 -> tie -> 0 (even)
+    assert q[0, 4] == 7 and q[0, 6] == 1 and q[0, 7] == 0 and q[0, 5] in (-3, -4)
+    # with one scale per channel the small group collapses to zero codes: the case group scales exist for
+    qc, sc = O.quantize_weight_sym(w, 4, 0)
+    assert qc[0, 4:].tolist() == [0, 0, 0, 0] and sc[0] == 1.0
+    # error bound per group: |q s - w| <= s / 2 wherever the code is not clamped
+    rng = np.random.default_rng(22)
+    w = (rng.standard_normal((16, 512)) * np.repeat(rng.uniform(0.01, 2.0, (16, 4)), 128, axis=1)).astype(np.float32)
+    q, s = O.quantize_weight_sym(w, 4, 128)
+    err = np.abs(q.astype(np.float64) * np.repeat(s, 128, axis=1) - w)
+    assert np.all(err <= np.repeat(s, 128, axis=1) / 2 * (1 + 1e-6))
+    assert np.abs(q).max() <= 7 and (np.abs(q).reshape(16, 4, 128).max(axis=2) == 7).all()
+
+
+def test_w8_and_a4_quantizers_hand_cases():
+    w = np.array([[127.0, -63.5, 0.5, -128.0]], np.float32)   # max 128 -> s = 128 / 127
+    q, s = O.quantize_weight_sym(w, 8, 0)
+    assert s[0] == np.float32(128.0) / np.float32(127.0)
+    assert q[0].tolist() == [126, -63, 0, -127]                 # 127 / s = 126.0078, -63.5 / s = -63.004, 0.5 / s = 0.496
+    # 4-bit activations: clamp to [-8, 7], ties to even, same reciprocal multiply as the 8-bit path
+    r = np.array([[0.0, 0.5, 1.0, 1.5, 2.5, 7.0, 7.6, 100.0, -8.4, -9.0, -100.0, np.nan, np.inf, -np.inf]], np.float32)
+    q = O.quantize_act_sym(r, [1.0], 4)
+    assert q[0].tolist() == [0, 0, 1, 2, 2, 7, 7, 7, -8, -8, -8, 0, 7, -8]
+    rng = np.random.default_rng(23)
+    r = (rng.standard_normal((7, 96)) * 30).astype(np.float32)
+    s_rows = rng.uniform(0.1, 3.0, 7).astype(np.float32)
+    assert np.array_equal(O.quantize_act_sym(r, s_rows, 8), O.quantize_act_int8(r, s_rows))
+    # Eq. 2's scale with b = 4: max / 7; the arg-max element then takes code +-7
+    x = np.array([[0.5, -3.5, 1.0], [2.0, 0.25, -0.9]], np.float32)
+    s_v, s_t = O.calibrate_static_scales_bits(x, [1, 2], [1, 0], 0, 4)
+    assert s_v == np.float32(3.5) / np.float32(7) and s_t == np.float32(2.0) / np.float32(7)
+    assert O.quantize_act_sym(x, [s_v, s_t], 4).tolist() == [[1, -7, 2], [7, 1, -3]]    # 0.25 / (2/7) = 0.875 -> 1; -0.9 -> -3.15 -> -3
+    assert O.calibrate_static_scales_bits(x, [1, 2], [1, 0], 0, 8) == O.calibrate_static_scales(x, [1, 2], [1, 0], 0)
+
+
+def test_grouped_linear_against_plain_definitions():
+    rng = np.random.default_rng(24)
+    T, K, N, g = 9, 512, 20, 128
+    x = np.asarray(rng.standard_t(3.0, (T, K)), np.float32)
+    w = (rng.standard_normal((N, K)) * np.repeat(rng.uniform(0.005, 0.2, (N, K // g)), g, axis=1)).astype(np.float32)
+    seg_end, seg_mod = [5, T], [1, 0]
+    s_v, s_t = O.calibrate_static_scales(x, seg_end, seg_mod, 128)
+    qw, s_wg = O.quantize_weight_sym(w, 4, g)
+    bias = rng.standard_normal(N).astype(np.float32)
+    ref = O.linear_wa_sym(x, seg_end, seg_mod, s_v, s_t, 128, qw, s_wg, 8, g, bias)
+    # the per-group partial sums add up to the ungrouped integer product, and match nested Python loops
+    assert np.array_equal(ref["acc_g"].sum(axis=2), O.int_gemm(ref["qx"], qw))
+    assert np.array_equal(ref["acc_g"][:2, :3, 1], O.int_gemm_loops(ref["qx"][:2, g:2 * g], qw[:3, g:2 * g]))
+    # the plain definition: dequantized activations times dequantized weights, in float64
+    x_hat = ref["qx"].astype(np.float64) * ref["s_rows"].astype(np.float64)[:, None]
+    w_hat = qw.astype(np.float64) * np.repeat(s_wg.astype(np.float64), g, axis=1)
+    want = x_hat @ w_hat.T + bias.astype(np.float64)[None, :]
+    assert np.max(np.abs(ref["y64"] - want)) <= 1e-10 * np.abs(want).max()
+    assert np.max(np.abs(ref["y32"] - want) / (np.abs(x_hat) @ np.abs(w_hat).T + np.abs(bias))) <= 1e-5
+    # one group: bit for bit the per-channel linear
+    q1, s1 = O.quantize_weight_sym(w, 4, K)
+    a = O.linear_wa_sym(x, seg_end, seg_mod, s_v, s_t, 128, q1, s1, 8, K, bias)
+    b = O.linear_w4a8_msq(x, seg_end, seg_mod, s_v, s_t, 128, *O.quantize_weight_int4(w), bias)
+    assert np.array_equal(a["y32"], b["y32"]) and np.array_equal(a["y_bf16"], b["y_bf16"])
+    assert np.array_equal(a["acc_g"][:, :, 0], b["acc"])
+    # on a weight whose groups differ in range, group scales reconstruct the exact product better
+    exact = O.fwht_blocks(x, 128, np.float64) @ w.astype(np.float64).T + bias
+    err_g = np.abs(ref["y64"] - exact).mean()
+    err_c = np.abs(O.linear_w4a8_msq(x, seg_end, seg_mod, s_v, s_t, 128, *O.quantize_weight_int4(w), bias)["y64"] - exact).mean()
+    assert err_g < err_c
+
+
+def test_w8a8_and_w4a4_linears_order_their_errors():
+    # Sec. 4.1 main table: W8A8 is closest to the exact product, W4A8 next, W4A4 last
+    rng = np.random.default_rng(25)
+    T, K, N = 12, 256, 16
+    x = rng.standard_normal((T, K)).astype(np.float32)
+    w = (rng.standard_normal((N, K)) * 0.05).astype(np.float32)
+    seg_end, seg_mod = [T], [0]
+    exact = x.astype(np.float64) @ w.astype(np.float64).T
+    errs = {}
+    for name, wb, ab in (("w8a8", 8, 8), ("w4a8", 4, 8), ("w4a4", 4, 4)):
+        s_v, s_t = O.calibrate_static_scales_bits(x, seg_end, seg_mod, 0, ab)
+        qw, s_w = O.quantize_weight_sym(w, wb, 0)
+        out = O.linear_wa_sym(x, seg_end, seg_mod, s_v, s_t, 0, qw, s_w, ab, 0)
+        assert np.abs(out["qx"]).max() <= 2 ** (ab - 1) and np.abs(qw).max() <= 2 ** (wb - 1)
+        errs[name] = np.abs(out["y64"] - exact).mean()
+    assert errs["w8a8"] < errs["w4a8"] < errs["w4a4"]
+    # W4A8 through the general path is the hot path itself
+    s_v, s_t = O.calibrate_static_scales(x, seg_end, seg_mod, 0)
+    a = O.linear_wa_sym(x, seg_end, seg_mod, s_v, s_t, 0, *O.quantize_weight_int4(w))
+    b = O.linear_w4a8_msq(x, seg_end, seg_mod, s_v, s_t, 0, *O.quantize_weight_int4(w))
+    assert np.array_equal(a["acc"], b["acc"]) and np.array_equal(a["y_bf16"], b["y_bf16"])
