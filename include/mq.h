@@ -62,6 +62,8 @@ extern "C" {
 /* mq_linear_desc.flags */
 #define MQ_FLAG_X_IS_INT8 1u /* X is already int8 codes [T,K]; skip rotation + quantization */
 #define MQ_FLAG_Y_IS_F32 2u  /* write Y as float32 instead of bfloat16 */
+#define MQ_FLAG_A4 4u        /* 4-bit activation codes (W4A4): clamp to [-8,7], scales from max / 7 */
+#define MQ_FLAG_W8 8u        /* 8-bit weights (W8A8): W_layout from mq_pack_w8, s_w = max / 127 */
 
 /* Size of the library-owned scratch array behind mq_w4a8_msq_linear_noalloc (4 MiB). */
 #define MQ_NOALLOC_WS_BYTES 4194304
@@ -81,7 +83,7 @@ typedef struct mq_linear_desc {
   int32_t K;          /* input channels, multiple of 32 */
   int32_t N;          /* output channels, multiple of 16 */
   int32_t rot_block;  /* online Hadamard block: 0 = off, else 32..1024 power of two dividing K */
-  int32_t group_size; /* weight scale group along K: 0 = one scale per output channel */
+  int32_t group_size; /* weight scale group along K: 0 = one scale per output channel, 128 = group-wise */
   uint32_t flags;     /* MQ_FLAG_* */
 } mq_linear_desc;
 
@@ -115,6 +117,13 @@ int mq_calibrate_static_scales(const void* X, int32_t T, int32_t K, int64_t ldx,
                                uint32_t* amax_state, float* s_vis_out, float* s_txt_out,
                                void* stream);
 
+/* mq_calibrate_static_scales for b-bit activations (act_bits 8 or 4): the divisor is 2^(b-1) - 1, i.e.
+ * 7 for the 4-bit activations of the W4A4 setting (Sec. 4.1).  act_bits = 8 is the call above. */
+int mq_calibrate_static_scales_bits(const void* X, int32_t T, int32_t K, int64_t ldx,
+                                    const mq_segments* seg, int32_t rot_block, int32_t act_bits,
+                                    int32_t accumulate, uint32_t* amax_state, float* s_vis_out,
+                                    float* s_txt_out, void* stream);
+
 /*
  * Weight quantization and packing (Eq. 2 with b = 4, z = 0; Algorithm 1 outputs
  * per-channel weight scales; plain round-to-nearest stands in for GPTQ).
@@ -127,10 +136,25 @@ int mq_calibrate_static_scales(const void* X, int32_t T, int32_t K, int64_t ldx,
  *   gemm_layout optional (may be NULL) opaque layout consumed by mq_w4a8_msq_linear,
  *           mq_w4_layout_bytes(N,K) bytes, 128-byte aligned; a pure permutation of the
  *           canonical nibbles, zero-padded to whole 128 x 128 tiles.
- * group_size must be 0 (per output channel); other values MQ_ERR_UNSUPPORTED.
+ * group_size = 128 (group-wise W4, the g = 128 setting of the weight-only comparison, App. A.12):
+ * one scale per output channel AND run of 128 input channels, s = max over the group / 7; s_w is then
+ * float32 [K / 128, N] (group-major: s_w[g * N + n]) and K must be a multiple of 128.  Other non-zero
+ * values MQ_ERR_UNSUPPORTED.
  */
 int mq_pack_w4(const float* W, int32_t N, int32_t K, int64_t ldw, int32_t group_size,
                uint8_t* packed, float* s_w, void* gemm_layout, void* stream);
+
+/*
+ * 8-bit weights for the W8A8 setting (main results table, Sec. 4.1): Eq. 2 with b = 8,
+ *   s_w[n] = max_k |W[n,k]| / 127 (1.0f for an all-zero row), q = clamp(round_half_even(W / s_w), -128, 127).
+ *   q_out       optional int8 [N,K] (leading dimension ldq): the codes, for inspection
+ *   gemm_layout optional, mq_w8_layout_bytes(N,K) bytes, 128-byte aligned: what mq_w4a8_msq_linear reads
+ *               when MQ_FLAG_W8 is set (128 x 128 tiles of 16 KB, zero-padded)
+ * At least one of q_out / gemm_layout must be given.
+ */
+size_t mq_w8_layout_bytes(int32_t N, int32_t K);
+int mq_pack_w8(const float* W, int32_t N, int32_t K, int64_t ldw, int8_t* q_out, int64_t ldq, float* s_w,
+               void* gemm_layout, void* stream);
 
 /* Canonical [N,K/2] bytes -> GEMM weight layout (same permutation as mq_pack_w4). */
 int mq_repack_w4(const uint8_t* packed, int32_t N, int32_t K, void* gemm_layout, void* stream);
@@ -188,6 +212,12 @@ int mq_fwht_quant_i8(const void* X, int32_t T, int32_t K, int64_t ldx, const mq_
                      float s_vis, float s_txt, int32_t rot_block, int8_t* Q, int64_t ldq,
                      float* rotated_out, void* stream);
 
+/* mq_fwht_quant_i8 with b-bit codes (act_bits 8 or 4; one byte per code either way): for 4 bits the
+ * codes clamp to [-8, 7] (Eq. 2 with b = 4).  No rotated dump. */
+int mq_fwht_quant_bits(const void* X, int32_t T, int32_t K, int64_t ldx, const mq_segments* seg,
+                       float s_vis, float s_txt, int32_t rot_block, int32_t act_bits, int8_t* Q,
+                       int64_t ldq, void* stream);
+
 /*
  * The W4A8 MSQ linear (Sec. 3.1 MSQ + Fig. 4(a) + Eq. 2):
  *   Qx  = mq_fwht_quant_i8(X)            (skipped when MQ_FLAG_X_IS_INT8)
@@ -200,6 +230,16 @@ int mq_fwht_quant_i8(const void* X, int32_t T, int32_t K, int64_t ldx, const mq_
  *   acc_out  optional int32 [T,N] (leading dimension N) dump of the accumulators
  *   ws       workspace of at least mq_workspace_bytes(d) bytes, 256-byte aligned
  * T = 0 is a successful no-op.
+ * Neighbouring settings of the main results table (Sec. 4.1) and of the weight-only comparison
+ * (App. A.12) run through the same call:
+ *   MQ_FLAG_A4        W4A4: the quantizer clamps to [-8, 7] (pass scales calibrated with act_bits = 4);
+ *   MQ_FLAG_W8        W8A8: W_layout / s_w from mq_pack_w8;
+ *   group_size = 128  group-wise W4: s_w is [K / 128, N];
+ *                       Y[t,n] = sum_g fl(float(acc_g[t,n]) * fl(s_mod(t) * s_w[g,n])) added in increasing g
+ *                       (+ bias); acc_out, if given, is int32 [K / 128, T, N]: the accumulator of every group.
+ *                       The group sums are folded into float registers after every K block, which costs
+ *                       about half of the per-channel kernel's throughput (see DESIGN notes in the source).
+ * MQ_FLAG_W8 and group_size = 128 exclude each other (MQ_ERR_UNSUPPORTED).
  * Which kernel runs is an internal choice that does not change the result: one to four
  * rows (single-sequence decode, the case the paper times with a W4A8 GEMV kernel,
  * Sec. 4.3) run rotation, quantizer and a CUDA-core GEMV in ONE kernel; more rows run the

@@ -22,6 +22,8 @@ MQ_ERR_TIMEOUT = -5
 MQ_ERR_WORKSPACE = -6
 MQ_FLAG_X_IS_INT8 = 1
 MQ_FLAG_Y_IS_F32 = 2
+MQ_FLAG_A4 = 4
+MQ_FLAG_W8 = 8
 MQ_NOALLOC_WS_BYTES = 4 << 20
 MQ_W_TILE_N, MQ_W_TILE_K = 128, 128
 TEXT, VISUAL = 0, 1
@@ -71,6 +73,10 @@ def load(build_if_missing: bool = False):
         "mq_w4_layout_bytes": (sz, [i32, i32]),
         "mq_calibrate_static_scales": (C.c_int, [vp, i32, i32, i64, segp, i32, i32, vp, vp, vp, vp]),
         "mq_pack_w4": (C.c_int, [vp, i32, i32, i64, i32, vp, vp, vp, vp]),
+        "mq_calibrate_static_scales_bits": (C.c_int, [vp, i32, i32, i64, segp, i32, i32, i32, vp, vp, vp, vp]),
+        "mq_w8_layout_bytes": (sz, [i32, i32]),
+        "mq_pack_w8": (C.c_int, [vp, i32, i32, i64, vp, i64, vp, vp, vp]),
+        "mq_fwht_quant_bits": (C.c_int, [vp, i32, i32, i64, segp, f32, f32, i32, i32, vp, i64, vp]),
         "mq_repack_w4": (C.c_int, [vp, i32, i32, vp, vp]),
         "mq_unpack_w4": (C.c_int, [vp, vp, i32, i32, vp, i64, vp]),
         "mq_aifs_reorder": (C.c_int, [vp, vp, i32, i32, i64, i64, vp, vp, vp, vp, vp, i32, vp]),
@@ -106,7 +112,8 @@ EXPORTED = ["mq_version", "mq_status_string", "mq_workspace_bytes", "mq_w4_layou
             "mq_attn_mask_remap", "mq_fwht_quant_i8", "mq_w4a8_msq_linear", "mq_w4a8_msq_linear_noalloc", "mq_last_device_status",
             "mq_reset_device_status", "mq_rms_side_ld", "mq_rms_detect", "mq_pack_w4_rms", "mq_rms_workspace_bytes",
             "mq_w4a8_msq_linear_rms", "mq_dynamic_quant_i8", "mq_dynamic_workspace_bytes", "mq_w4a8_dynamic_linear",
-            "mq_ubench_mma_i8", "mq_selftest_bounded_wait", "mq_ubench_expand"]
+            "mq_ubench_mma_i8", "mq_selftest_bounded_wait", "mq_ubench_expand", "mq_calibrate_static_scales_bits",
+            "mq_w8_layout_bytes", "mq_pack_w8", "mq_fwht_quant_bits"]
 
 
 def status_string(status: int) -> str:
@@ -155,8 +162,8 @@ def _ld(t: torch.Tensor) -> int:
 
 
 # ----------------------------------------------------------------------------- calls (same names as the C ABI)
-def mq_workspace_bytes(T, K, N, rot_block=0, flags=0) -> int:
-    d = mq_linear_desc(T, K, N, rot_block, 0, flags)
+def mq_workspace_bytes(T, K, N, rot_block=0, flags=0, group_size=0) -> int:
+    d = mq_linear_desc(T, K, N, rot_block, group_size, flags)
     return int(load().mq_workspace_bytes(C.byref(d)))
 
 
@@ -164,9 +171,9 @@ def mq_w4_layout_bytes(N, K) -> int:
     return int(load().mq_w4_layout_bytes(N, K))
 
 
-def new_workspace(T, K, N, rot_block=0, flags=0, device="cuda") -> torch.Tensor:
+def new_workspace(T, K, N, rot_block=0, flags=0, device="cuda", group_size=0) -> torch.Tensor:
     """Allocates (with torch) and clears a workspace for mq_w4a8_msq_linear."""
-    n = mq_workspace_bytes(T, K, N, rot_block, flags)
+    n = mq_workspace_bytes(T, K, N, rot_block, flags, group_size)
     if n == 0:
         raise MqError(MQ_ERR_INVALID_ARG, "mq_workspace_bytes")
     ws = torch.empty(n, dtype=torch.uint8, device=device)
@@ -174,9 +181,15 @@ def new_workspace(T, K, N, rot_block=0, flags=0, device="cuda") -> torch.Tensor:
     return ws
 
 
-def mq_calibrate_static_scales(x, seg: Segments, rot_block, amax_state, s_vis_out, s_txt_out, accumulate=False):
+def mq_calibrate_static_scales(x, seg: Segments, rot_block, amax_state, s_vis_out, s_txt_out, accumulate=False,
+                               act_bits=8):
     assert x.dtype == torch.bfloat16
     T, K = x.shape
+    if act_bits != 8:
+        _check(load().mq_calibrate_static_scales_bits(_ptr(x), T, K, _ld(x), seg.ref(), rot_block, act_bits,
+                                                      int(accumulate), _ptr(amax_state), _ptr(s_vis_out),
+                                                      _ptr(s_txt_out), _stream()), "mq_calibrate_static_scales_bits")
+        return
     _check(load().mq_calibrate_static_scales(_ptr(x), T, K, _ld(x), seg.ref(), rot_block, int(accumulate),
                                             _ptr(amax_state), _ptr(s_vis_out), _ptr(s_txt_out), _stream()),
            "mq_calibrate_static_scales")
@@ -187,6 +200,25 @@ def mq_pack_w4(w, packed=None, s_w=None, gemm_layout=None, group_size=0):
     N, K = w.shape
     _check(load().mq_pack_w4(_ptr(w), N, K, _ld(w), group_size, _ptr(packed), _ptr(s_w), _ptr(gemm_layout),
                              _stream()), "mq_pack_w4")
+
+
+def mq_w8_layout_bytes(N, K) -> int:
+    return int(load().mq_w8_layout_bytes(N, K))
+
+
+def mq_pack_w8(w, q_out=None, s_w=None, gemm_layout=None):
+    """8-bit per-channel weight quantizer (W8A8): codes int8 [N,K], scales max/127, GEMM layout."""
+    assert w.dtype == torch.float32
+    N, K = w.shape
+    _check(load().mq_pack_w8(_ptr(w), N, K, _ld(w), _ptr(q_out), _ld(q_out) if q_out is not None else 0, _ptr(s_w),
+                             _ptr(gemm_layout), _stream()), "mq_pack_w8")
+
+
+def mq_fwht_quant_bits(x, seg: Segments, s_vis, s_txt, rot_block, act_bits, q_out):
+    assert x.dtype == torch.bfloat16 and q_out.dtype == torch.int8
+    T, K = x.shape
+    _check(load().mq_fwht_quant_bits(_ptr(x), T, K, _ld(x), seg.ref(), float(s_vis), float(s_txt), rot_block,
+                                     act_bits, _ptr(q_out), _ld(q_out), _stream()), "mq_fwht_quant_bits")
 
 
 def mq_repack_w4(packed, N, K, gemm_layout):
@@ -226,10 +258,11 @@ def mq_fwht_quant_i8(x, seg: Segments, s_vis, s_txt, rot_block, q_out, rotated_o
 
 
 def mq_w4a8_msq_linear(x, seg: Segments, s_vis, s_txt, w_layout, s_w, y, ws, N, rot_block=0, bias=None,
-                       acc_out=None):
-    """x: bf16 [T,K] (rotated + quantized inside) or int8 [T,K] codes; y: bf16 or float32 [T,N]."""
+                       acc_out=None, group_size=0, extra_flags=0):
+    """x: bf16 [T,K] (rotated + quantized inside) or int8 [T,K] codes; y: bf16 or float32 [T,N].
+    extra_flags: MQ_FLAG_A4 / MQ_FLAG_W8; group_size: 0 or 128 (see include/mq.h)."""
     T, K = x.shape
-    flags = 0
+    flags = extra_flags
     if x.dtype == torch.int8:
         flags |= MQ_FLAG_X_IS_INT8
     else:
@@ -238,7 +271,7 @@ def mq_w4a8_msq_linear(x, seg: Segments, s_vis, s_txt, w_layout, s_w, y, ws, N, 
         flags |= MQ_FLAG_Y_IS_F32
     else:
         assert y.dtype == torch.bfloat16
-    d = mq_linear_desc(T, K, N, rot_block, 0, flags)
+    d = mq_linear_desc(T, K, N, rot_block, group_size, flags)
     _check(load().mq_w4a8_msq_linear(C.byref(d), _ptr(x), _ld(x), seg.ref(), float(s_vis), float(s_txt),
                                      _ptr(w_layout), _ptr(s_w), _ptr(bias), _ptr(y), _ld(y), _ptr(acc_out),
                                      _ptr(ws), ws.numel(), _stream()), "mq_w4a8_msq_linear")

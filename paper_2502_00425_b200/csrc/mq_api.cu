@@ -40,8 +40,11 @@ int check_desc(const mq_linear_desc* d) {
   if (d->T < 0 || d->K <= 0 || d->N <= 0) return MQ_ERR_INVALID_ARG;
   if (d->K % 32 || d->N % 16) return MQ_ERR_INVALID_ARG;
   if (d->K > 131040) return MQ_ERR_UNSUPPORTED;  // 16x accumulators must stay below 2^31
-  if (d->group_size != 0) return MQ_ERR_UNSUPPORTED;
-  if (d->flags & ~(MQ_FLAG_X_IS_INT8 | MQ_FLAG_Y_IS_F32)) return MQ_ERR_INVALID_ARG;
+  if (d->group_size < 0) return MQ_ERR_INVALID_ARG;
+  if (d->group_size != 0 && d->group_size != MQ_W_TILE_K) return MQ_ERR_UNSUPPORTED;  // a group is one K block
+  if (d->group_size && d->K % MQ_W_TILE_K) return MQ_ERR_INVALID_ARG;
+  if (d->flags & ~(MQ_FLAG_X_IS_INT8 | MQ_FLAG_Y_IS_F32 | MQ_FLAG_A4 | MQ_FLAG_W8)) return MQ_ERR_INVALID_ARG;
+  if ((d->flags & MQ_FLAG_W8) && d->group_size) return MQ_ERR_UNSUPPORTED;
   if (d->flags & MQ_FLAG_X_IS_INT8) {
     if (d->rot_block != 0) return MQ_ERR_INVALID_ARG;
     return MQ_OK;
@@ -57,7 +60,7 @@ WsLayout ws_layout(const mq_linear_desc* d) {
   w.qx_off = kStatusBytes;
   w.qx_bytes = (d->flags & MQ_FLAG_X_IS_INT8) ? 0 : align_up((size_t)d->T * d->K, 256);
   w.splitk_off = w.qx_off + w.qx_bytes;
-  w.splitk_bytes = align_up(gemm_splitk_bytes(d->T, d->K, d->N), 256);
+  w.splitk_bytes = align_up(gemm_splitk_bytes(d->T, d->K, d->N, false, d->group_size, (d->flags & MQ_FLAG_W8) ? 8 : 4), 256);
   w.total = w.splitk_off + w.splitk_bytes;
   return w;
 }
@@ -108,13 +111,41 @@ int mq_calibrate_static_scales(const void* X, int32_t T, int32_t K, int64_t ldx,
                           static_cast<cudaStream_t>(stream));
 }
 
+int mq_calibrate_static_scales_bits(const void* X, int32_t T, int32_t K, int64_t ldx, const mq_segments* seg,
+                                    int32_t rot_block, int32_t act_bits, int32_t accumulate, uint32_t* amax_state,
+                                    float* s_vis_out, float* s_txt_out, void* stream) {
+  if (act_bits != 4 && act_bits != 8) return MQ_ERR_UNSUPPORTED;
+  if (T < 0 || K <= 0 || K % 32) return MQ_ERR_INVALID_ARG;
+  if (!amax_state || !s_vis_out || !s_txt_out) return MQ_ERR_INVALID_ARG;
+  if (T > 0 && !X) return MQ_ERR_INVALID_ARG;
+  if (ldx < K) return MQ_ERR_INVALID_ARG;
+  if (!aligned16(X) || (ldx * 2) % 16) return MQ_ERR_ALIGNMENT;
+  int rc = check_rot(rot_block, K);
+  if (rc != MQ_OK) return rc;
+  SegTable st;
+  if ((rc = check_seg(seg, &st)) != MQ_OK) return rc;
+  return launch_calibrate(X, T, K, ldx, st, rot_block, accumulate, amax_state, s_vis_out, s_txt_out,
+                          static_cast<cudaStream_t>(stream), act_bits);
+}
+
 int mq_pack_w4(const float* W, int32_t N, int32_t K, int64_t ldw, int32_t group_size, uint8_t* packed, float* s_w,
                void* gemm_layout, void* stream) {
   if (N <= 0 || K <= 0 || !W || !s_w) return MQ_ERR_INVALID_ARG;
-  if (K % 32 || N % 16 || ldw < K) return MQ_ERR_INVALID_ARG;
-  if (group_size != 0) return MQ_ERR_UNSUPPORTED;
+  if (K % 32 || N % 16 || ldw < K || group_size < 0) return MQ_ERR_INVALID_ARG;
+  if (group_size != 0 && group_size != MQ_W_TILE_K) return MQ_ERR_UNSUPPORTED;
+  if (group_size && K % group_size) return MQ_ERR_INVALID_ARG;
   if (gemm_layout && !aligned(gemm_layout, 128)) return MQ_ERR_ALIGNMENT;
-  return launch_pack_w4(W, N, K, ldw, packed, s_w, gemm_layout, static_cast<cudaStream_t>(stream));
+  return launch_pack_w4(W, N, K, ldw, packed, s_w, gemm_layout, static_cast<cudaStream_t>(stream), group_size);
+}
+
+size_t mq_w8_layout_bytes(int32_t N, int32_t K) { return 2 * mq_w4_layout_bytes(N, K); }
+
+int mq_pack_w8(const float* W, int32_t N, int32_t K, int64_t ldw, int8_t* q_out, int64_t ldq, float* s_w,
+               void* gemm_layout, void* stream) {
+  if (N <= 0 || K <= 0 || !W || !s_w || (!q_out && !gemm_layout)) return MQ_ERR_INVALID_ARG;
+  if (K % 32 || N % 16 || ldw < K || (q_out && ldq < K)) return MQ_ERR_INVALID_ARG;
+  if (gemm_layout && !aligned(gemm_layout, 128)) return MQ_ERR_ALIGNMENT;
+  return launch_pack_w8(W, N, K, ldw, q_out, ldq, s_w, gemm_layout, static_cast<cudaStream_t>(stream));
 }
 
 int mq_repack_w4(const uint8_t* packed, int32_t N, int32_t K, void* gemm_layout, void* stream) {
@@ -176,6 +207,22 @@ int mq_fwht_quant_i8(const void* X, int32_t T, int32_t K, int64_t ldx, const mq_
                            static_cast<cudaStream_t>(stream));
 }
 
+int mq_fwht_quant_bits(const void* X, int32_t T, int32_t K, int64_t ldx, const mq_segments* seg, float s_vis,
+                       float s_txt, int32_t rot_block, int32_t act_bits, int8_t* Q, int64_t ldq, void* stream) {
+  if (act_bits != 4 && act_bits != 8) return MQ_ERR_UNSUPPORTED;
+  if (T < 0 || K <= 0 || K % 32) return MQ_ERR_INVALID_ARG;
+  if (T > 0 && (!X || !Q)) return MQ_ERR_INVALID_ARG;
+  if (ldx < K || ldq < K) return MQ_ERR_INVALID_ARG;
+  if (!good_scale(s_vis) || !good_scale(s_txt)) return MQ_ERR_INVALID_ARG;
+  if (!aligned16(X) || !aligned16(Q) || (ldx * 2) % 16 || ldq % 16) return MQ_ERR_ALIGNMENT;
+  int rc = check_rot(rot_block, K);
+  if (rc != MQ_OK) return rc;
+  SegTable st;
+  if ((rc = check_seg(seg, &st)) != MQ_OK) return rc;
+  return launch_fwht_quant(X, T, K, ldx, st, s_vis, s_txt, rot_block, Q, ldq, nullptr,
+                           static_cast<cudaStream_t>(stream), nullptr, 0, act_bits);
+}
+
 int mq_w4a8_msq_linear(const mq_linear_desc* d, const void* X, int64_t ldx, const mq_segments* seg, float s_vis,
                        float s_txt, const void* W_layout, const float* s_w, const float* bias, void* Y, int64_t ldy,
                        int32_t* acc_out, void* ws, size_t ws_bytes, void* stream) {
@@ -200,7 +247,10 @@ int mq_w4a8_msq_linear(const mq_linear_desc* d, const void* X, int64_t ldx, cons
 
   const int8_t* qx;
   int64_t ldq;
-  if (!x_i8 && gemv_applies(d->T, d->K, d->N)) {
+  const int act_bits = (d->flags & MQ_FLAG_A4) ? 4 : 8;
+  const int w_bits = (d->flags & MQ_FLAG_W8) ? 8 : 4;
+  const bool variant = act_bits != 8 || w_bits != 4 || d->group_size != 0;  // neighbours of the hot path
+  if (!variant && !x_i8 && gemv_applies(d->T, d->K, d->N)) {
     // one to four tokens: a single kernel rotates, quantizes and multiplies (mq_gemv.cu)
     GemmArgs g{};
     g.T = d->T; g.K = d->K; g.N = d->N;
@@ -214,13 +264,14 @@ int mq_w4a8_msq_linear(const mq_linear_desc* d, const void* X, int64_t ldx, cons
     ldq = ldx;
   } else {
     int8_t* q = reinterpret_cast<int8_t*>(wsb + wl.qx_off);
-    rc = launch_fwht_quant(X, d->T, d->K, ldx, st, s_vis, s_txt, d->rot_block, q, d->K, nullptr, cs);
+    rc = launch_fwht_quant(X, d->T, d->K, ldx, st, s_vis, s_txt, d->rot_block, q, d->K, nullptr, cs, nullptr, 0, act_bits);
     if (rc != MQ_OK) return rc;
     qx = q;
     ldq = d->K;
   }
   GemmArgs a{};
   a.T = d->T; a.K = d->K; a.N = d->N;
+  a.group_size = d->group_size; a.w_bits = w_bits;
   a.Qx = qx; a.ldq = ldq; a.seg = st; a.s_vis = s_vis; a.s_txt = s_txt;
   a.W_layout = W_layout; a.s_w = s_w; a.bias = bias; a.Y = Y; a.ldy = ldy; a.y_is_f32 = y_f32 ? 1 : 0;
   a.acc_out = acc_out;

@@ -118,16 +118,18 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
 // host launchers implemented in the .cu files -----------------------------------------
 int launch_fwht_quant(const void* X, int T, int K, int64_t ldx, SegTable seg, float s_vis,
                       float s_txt, int rot_block, int8_t* Q, int64_t ldq, float* rotated_out,
-                      cudaStream_t st, int8_t* side_out = nullptr, int side_ld = 0);
+                      cudaStream_t st, int8_t* side_out = nullptr, int side_ld = 0, int act_bits = 8);
 int launch_dyn_quant(const void* X, int T, int K, int64_t ldx, int rot_block, int8_t* Q, int64_t ldq, float* s_rows,
                      cudaStream_t st);
 int launch_calibrate(const void* X, int T, int K, int64_t ldx, SegTable seg, int rot_block,
                      int accumulate, uint32_t* amax_state, float* s_vis_out, float* s_txt_out,
-                     cudaStream_t st);
+                     cudaStream_t st, int act_bits = 8);
 int launch_pack_w4(const float* W, int N, int K, int64_t ldw, uint8_t* packed, float* s_w,
-                   void* layout, cudaStream_t st);
+                   void* layout, cudaStream_t st, int group = 0);
 int launch_pack_codes(const float* W, int N, int K, int64_t ldw, const float* s_w, uint8_t* packed,
-                      void* layout, int skip, cudaStream_t st);
+                      void* layout, int skip, cudaStream_t st, int group = 0);
+int launch_pack_w8(const float* W, int N, int K, int64_t ldw, int8_t* q_out, int64_t ldq, float* s_w, void* layout,
+                   cudaStream_t st);
 int launch_repack_w4(const uint8_t* packed, int N, int K, void* layout, cudaStream_t st);
 int launch_unpack_w4(const uint8_t* packed, const void* layout, int N, int K, int8_t* q,
                      int64_t ldq, cudaStream_t st);
@@ -174,11 +176,16 @@ struct GemmArgs {
   const void* side_layout;
   const float* s_w_side;
   int32_t* acc_side_out;
+  // Variants: group_size = 128 selects group-wise weight scales (s_w is then [K / 128][N]; acc_out, if given,
+  // receives the per-group accumulators [K / 128][T][N]); w_bits = 8 selects 8-bit weights (W_layout from
+  // mq_pack_w8).  0 / 0 is the W4 per-channel hot path.
+  int group_size;
+  int w_bits;
 };
 int launch_gemm(const GemmArgs& a, cudaStream_t st);
 // one to four tokens: CUDA-core GEMV (mq_gemv.cu); launch_gemm routes there when it applies
 bool gemv_applies(int T, int K, int N, int side_k = 0);
 int launch_gemv(const GemmArgs& a, cudaStream_t st);
-size_t gemm_splitk_bytes(int T, int K, int N, bool rms = false);
+size_t gemm_splitk_bytes(int T, int K, int N, bool rms = false, int group_size = 0, int w_bits = 4);
 
 }  // namespace mq

@@ -27,7 +27,8 @@ constexpr int kWarpTile = kFwhtWarpTile;  // channels per warp pass
 // kQuantSide: also writes the code of the first channel of every rotation block to
 // side_out[row, block] -- the activation operand of the split product of rotation
 // magnitude suppression (Sec. 3.2), K-contiguous for the GEMM's tensor map.
-enum Mode { kQuant = 0, kQuantDump = 1, kAbsMax = 2, kQuantSide = 3 };
+// kQuant4: 4-bit codes (clamp to [-8, 7]) for the W4A4 setting.
+enum Mode { kQuant = 0, kQuantDump = 1, kAbsMax = 2, kQuantSide = 3, kQuant4 = 4 };
 
 template <int LOG_TPB, bool ROT, int MODE>
 __global__ void __launch_bounds__(kWarpsPerCta * 32)
@@ -76,7 +77,7 @@ fwht_quant_kernel(const uint16_t* __restrict__ X, int T, int K, int64_t ldx, Seg
       dst[0] = make_float4(v[i][0], v[i][1], v[i][2], v[i][3]);
       dst[1] = make_float4(v[i][4], v[i][5], v[i][6], v[i][7]);
     }
-    const uint2 o = quant_chunk_s8(v[i], inv);
+    const uint2 o = MODE == kQuant4 ? quant_chunk_s4(v[i], inv) : quant_chunk_s8(v[i], inv);
     *reinterpret_cast<uint2*>(qrow + off) = o;
     if (MODE == kQuantSide && i == 0 && j == 0)  // element 0 of the block is in chunk 0 of lane-in-block 0
       side_out[(int64_t)row * side_ld + (blk_start >> (5 + LOG_TPB))] = (int8_t)(o.x & 0xffu);
@@ -87,12 +88,12 @@ __global__ void calib_reset_kernel(uint32_t* amax_state) {
   if (threadIdx.x < 2) amax_state[threadIdx.x] = 0u;
 }
 
-__global__ void calib_finalize_kernel(const uint32_t* amax_state, float* s_vis_out, float* s_txt_out) {
+__global__ void calib_finalize_kernel(const uint32_t* amax_state, float* s_vis_out, float* s_txt_out, float qmax) {
   if (threadIdx.x == 0) {
     const float mt = __uint_as_float(amax_state[MQ_TEXT]);
     const float mv = __uint_as_float(amax_state[MQ_VISUAL]);
-    *s_txt_out = mt > 0.0f ? __fdiv_rn(mt, 127.0f) : 1.0f;
-    *s_vis_out = mv > 0.0f ? __fdiv_rn(mv, 127.0f) : 1.0f;
+    *s_txt_out = mt > 0.0f ? __fdiv_rn(mt, qmax) : 1.0f;
+    *s_vis_out = mv > 0.0f ? __fdiv_rn(mv, qmax) : 1.0f;
   }
 }
 
@@ -129,8 +130,12 @@ int dispatch(const void* X, int T, int K, int64_t ldx, SegTable seg, float inv_v
 
 int launch_fwht_quant(const void* X, int T, int K, int64_t ldx, SegTable seg, float s_vis,
                       float s_txt, int rot_block, int8_t* Q, int64_t ldq, float* rotated_out,
-                      cudaStream_t st, int8_t* side_out, int side_ld) {
+                      cudaStream_t st, int8_t* side_out, int side_ld, int act_bits) {
   const float inv_vis = 1.0f / s_vis, inv_txt = 1.0f / s_txt;
+  if (act_bits == 4) {
+    if (side_out || rotated_out) return MQ_ERR_UNSUPPORTED;
+    return dispatch<kQuant4>(X, T, K, ldx, seg, inv_vis, inv_txt, rot_block, Q, ldq, nullptr, nullptr, st);
+  }
   if (side_out) {
     if (!rot_block || rotated_out) return MQ_ERR_INVALID_ARG;
     return dispatch<kQuantSide>(X, T, K, ldx, seg, inv_vis, inv_txt, rot_block, Q, ldq, nullptr, nullptr, st,
@@ -144,11 +149,11 @@ int launch_fwht_quant(const void* X, int T, int K, int64_t ldx, SegTable seg, fl
 
 int launch_calibrate(const void* X, int T, int K, int64_t ldx, SegTable seg, int rot_block,
                      int accumulate, uint32_t* amax_state, float* s_vis_out, float* s_txt_out,
-                     cudaStream_t st) {
+                     cudaStream_t st, int act_bits) {
   if (!accumulate) calib_reset_kernel<<<1, 32, 0, st>>>(amax_state);
   int rc = dispatch<kAbsMax>(X, T, K, ldx, seg, 1.0f, 1.0f, rot_block, nullptr, 0, nullptr, amax_state, st);
   if (rc != MQ_OK) return rc;
-  calib_finalize_kernel<<<1, 32, 0, st>>>(amax_state, s_vis_out, s_txt_out);
+  calib_finalize_kernel<<<1, 32, 0, st>>>(amax_state, s_vis_out, s_txt_out, act_bits == 4 ? 7.0f : 127.0f);
   return cuda_status(cudaGetLastError());
 }
 

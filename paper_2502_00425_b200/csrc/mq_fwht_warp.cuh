@@ -95,4 +95,16 @@ __device__ __forceinline__ uint2 quant_chunk_s8(const float (&v)[8], float inv) 
   return o;
 }
 
+// The same with 4-bit codes (the activation side of W4A4, Sec. 4.1): clamp to [-8, 7]; the codes still
+// occupy one byte each.
+__device__ __forceinline__ uint2 quant_chunk_s4(const float (&v)[8], float inv) {
+  int q[8];
+#pragma unroll
+  for (int r = 0; r < 8; ++r) q[r] = max(-8, min(7, __float2int_rn(__fmul_rn(v[r], inv))));
+  uint2 o;
+  o.x = pack_sat_s8x4(q[0], q[1], q[2], q[3]);
+  o.y = pack_sat_s8x4(q[4], q[5], q[6], q[7]);
+  return o;
+}
+
 }  // namespace mq

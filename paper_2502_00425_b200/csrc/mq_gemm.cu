@@ -48,10 +48,15 @@ constexpr int kMaxGroups = 2;                       // expander warp groups (4 w
 constexpr int kMaxThreads = (8 + 4 * kMaxGroups) * 32;
 constexpr int kTileN = MQ_W_TILE_N;    // channels per CTA tile (MMA M)
 constexpr int kBlockK = MQ_W_TILE_K;   // K per pipeline stage
-constexpr int kWTileBytes = 8192;      // packed int4 tile 128 x 128
+constexpr int kWTileBytes = 8192;      // packed int4 tile 128 x 128 (an int8 tile is twice that)
 constexpr int kMaxStages = 8;    // main ring: activation tiles in shared memory
 constexpr int kMaxWStages = 16;  // packed-weight tiles in shared memory
 constexpr int kSmemBudget = 226 * 1024;  // of the 227 KB a CTA may use
+
+// Instantiations of the kernel.  kPlain: the W4A8 MSQ linear.  kRms: plus the split product of rotation
+// magnitude suppression.  kGrouped: group-wise weight scales (one per output channel and K block of 128),
+// folded into float sums after every K block.  kW8: 8-bit weights (no nibble expansion, no factor 16).
+enum : int { kPlain = 0, kRms = 1, kGrouped = 2, kW8 = 3 };
 
 struct KernelParams {
   int T, K, N;
@@ -88,6 +93,7 @@ struct KernelParams {
   const float* s_w_side;
   int32_t* acc_side_out;       // optional dump of the split accumulator [T, N]
   int32_t* splitk_side;        // split-K launches: the split accumulator's own [T, N] slice
+  int w_tile_bytes;            // bytes of one 128 x 128 weight tile in W_layout (8192 int4, 16384 int8)
 };
 
 struct __align__(16) Barriers {
@@ -133,7 +139,8 @@ struct TileIter {
 // (bf16 output, with or without bias, and the split-K partial sums) are compiled separately so
 // that their per-element code has no branches; the debug outputs (accumulator dump, float32
 // output) share one generic variant that tests its flags at run time.
-enum : int { kEpiSplitK = 1, kEpiAcc = 2, kEpiF32 = 4, kEpiBias = 8, kEpiGeneric = 16, kEpiStaged = 32 };
+// kEpiNoShift: the accumulator is the true one (8-bit weights), not 16x it.
+enum : int { kEpiSplitK = 1, kEpiAcc = 2, kEpiF32 = 4, kEpiBias = 8, kEpiGeneric = 16, kEpiStaged = 32, kEpiNoShift = 64 };
 
 // bf16 output of a 16 x 32 (token x channel) block held one channel per lane: transpose it
 // through this warp's staging buffer so that every lane stores 16 bytes (8 channels of one
@@ -162,6 +169,7 @@ template <int MODE>
 __device__ __forceinline__ void epilogue_chunk(const KernelParams& p, const uint32_t (&v)[16], int t_first,
                                                int nvalid, int n, bool n_ok, float sw, float bs,
                                                const float* stok, __nv_bfloat16* stage, int ks) {
+  constexpr int SH = (MODE & kEpiNoShift) ? 0 : 4;  // the MMA saw 16 * q_w unless the weights are 8-bit
   if (!(MODE & kEpiStaged) && !n_ok) return;
   if (MODE & kEpiSplitK) {
     // every K split owns a slice [T,N] of the scratch: plain stores, summed by the finalize
@@ -169,13 +177,13 @@ __device__ __forceinline__ void epilogue_chunk(const KernelParams& p, const uint
     int32_t* dst = p.splitk_acc + (size_t)ks * p.T * p.N + (size_t)t_first * p.N + n;
 #pragma unroll
     for (int j = 0; j < 16; ++j)
-      if (j < nvalid) dst[(size_t)j * p.N] = ((int)v[j]) >> 4;  // the MMA saw 16 * q_w
+      if (j < nvalid) dst[(size_t)j * p.N] = ((int)v[j]) >> SH;
     return;
   }
   if (MODE & kEpiGeneric) {
 #pragma unroll 1
     for (int j = 0; j < nvalid; ++j) {
-      const int acc = ((int)v[j]) >> 4;
+      const int acc = ((int)v[j]) >> SH;
       const size_t t = (size_t)(t_first + j);
       if (p.acc_out) p.acc_out[t * p.N + n] = acc;
       float y = __fmul_rn((float)acc, __fmul_rn(stok[j], sw));
@@ -191,7 +199,7 @@ __device__ __forceinline__ void epilogue_chunk(const KernelParams& p, const uint
   float y[16];
 #pragma unroll
   for (int j = 0; j < 16; ++j) {
-    y[j] = __fmul_rn((float)(((int)v[j]) >> 4), __fmul_rn(stok[j], sw));  // the MMA saw 16 * q_w
+    y[j] = __fmul_rn((float)(((int)v[j]) >> SH), __fmul_rn(stok[j], sw));
     if (MODE & kEpiBias) y[j] = __fadd_rn(y[j], bs);
   }
   if (MODE & kEpiStaged) {
@@ -201,7 +209,7 @@ __device__ __forceinline__ void epilogue_chunk(const KernelParams& p, const uint
 #pragma unroll
   for (int j = 0; j < 16; ++j) {
     if (j < nvalid) {
-      if (MODE & kEpiAcc) acc_dst[(size_t)j * p.N] = ((int)v[j]) >> 4;
+      if (MODE & kEpiAcc) acc_dst[(size_t)j * p.N] = ((int)v[j]) >> SH;
       if (MODE & kEpiF32) y32[(size_t)j * p.ldy] = y[j];
       else y16[(size_t)j * p.ldy] = __float2bfloat16_rn(y[j]);
     }
@@ -295,23 +303,27 @@ __device__ __forceinline__ void epilogue_tile_side_slice(const KernelParams& p, 
 }
 
 // ------------------------------------------------------------------------------ the kernel
-// RMS = true is the instantiation behind the rotation-magnitude-suppression linear: every tile
+// MODE = kRms is the instantiation behind the rotation-magnitude-suppression linear: every tile
 // (of K split 0) first runs the split product -- p.side_kb K blocks whose activations come
 // through tmap_side and whose weights come from p.side_layout -- into a second accumulator,
 // then the main product, and the epilogue combines the two.  The K blocks of both products
 // go through the same rings; only the sources and the MMA's destination differ.  A separate
 // instantiation keeps the ordinary kernel's code and register allocation as they were.
-template <bool RMS>
+template <int MODE>
 __global__ void __launch_bounds__(kMaxThreads, 1)
 w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const __grid_constant__ CUtensorMap tmap_side,
                  const KernelParams p) {
+  constexpr bool RMS = MODE == kRms;
+  constexpr bool GROUPED = MODE == kGrouped;
+  constexpr bool W8 = MODE == kW8;
+  constexpr int kTileBytes = W8 ? 2 * kWTileBytes : kWTileBytes;
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   // carve: activation stages (1024-aligned), weight stages, barriers, token scales
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int act_stage_bytes = p.TN * kBlockK;
   uint8_t* act_smem = smem;
   uint8_t* w_smem = act_smem + (size_t)p.stages * act_stage_bytes;
-  Barriers* sh = reinterpret_cast<Barriers*>(w_smem + (size_t)p.w_stages * kWTileBytes);
+  Barriers* sh = reinterpret_cast<Barriers*>(w_smem + (size_t)p.w_stages * kTileBytes);
   float* s_tok = reinterpret_cast<float*>(sh + 1);  // [4 epilogue warps][256], then bf16 staging [4][16 x 32]
 
   const int warp = threadIdx.x >> 5;
@@ -396,11 +408,11 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const __grid_cons
           }
           if (!ok) break;
         }
-        const uint8_t* wsrc = p.W_layout + ((size_t)c.tn * p.kb_total + c.kb0(p)) * kWTileBytes;
-        for (int kb = c.kb0(p), kb_end = c.kb1(p); kb < kb_end; ++kb, ++it, wsrc += kWTileBytes) {
+        const uint8_t* wsrc = p.W_layout + ((size_t)c.tn * p.kb_total + c.kb0(p)) * kTileBytes;
+        for (int kb = c.kb0(p), kb_end = c.kb1(p); kb < kb_end; ++kb, ++it, wsrc += kTileBytes) {
           if (wrapped && !(ok = mbar_wait(&sh->w_empty[s], ph ^ 1u, &sh->abort_flag, p.status, 2))) break;
-          mbar_arrive_expect_tx(&sh->w_full[s], kWTileBytes);
-          bulk_load_1d(w_smem + (size_t)s * kWTileBytes, wsrc, kWTileBytes, &sh->w_full[s]);
+          mbar_arrive_expect_tx(&sh->w_full[s], kTileBytes);
+          bulk_load_1d(w_smem + (size_t)s * kTileBytes, wsrc, kTileBytes, &sh->w_full[s]);
           if (++s == p.w_stages) { s = 0; ph ^= 1u; wrapped = true; }
         }
       }
@@ -445,6 +457,33 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const __grid_cons
         if (!ok) break;
         accumulate = 0;
       }
+      if (GROUPED) {
+        // group-wise weight scales: every K block (= one group of 128 input channels) gets a fresh
+        // accumulator, alternating between the two buffers; the epilogue warps fold it into their float
+        // sums while the next block's MMAs run.  (The tile's first buffer wait happened above.)
+        bool first_block = true;
+        for (int kb = c.kb0(p), kb_end = c.kb1(p); kb < kb_end; ++kb) {
+          if (!first_block && d_wrapped &&
+              !(ok = warp_all(mbar_wait(&sh->d_empty[d], ph_d ^ 1u, &sh->abort_flag, p.status, 3)))) break;
+          first_block = false;
+          if (!(ok = warp_all(mbar_wait(&sh->full[s], ph, &sh->abort_flag, p.status, 4)))) break;
+          tc_fence_after();
+          const uint64_t bdesc = bdesc0 + (uint64_t)((uint32_t)s * bdesc_step);
+          const uint32_t a_tmem = tmem_base + (uint32_t)(p.a_base + a * 32);
+          const uint32_t dg_tmem = tmem_base + (uint32_t)(d * p.d_stride);
+          if (elect_one()) {
+#pragma unroll
+            for (int k4 = 0; k4 < 4; ++k4)
+              mma_i8_ts(dg_tmem, a_tmem + k4 * 8, bdesc + (uint64_t)(k4 * 2), idesc, (uint32_t)k4);
+            tc_commit(&sh->done[s]);
+            tc_commit(&sh->d_full[d]);
+          }
+          if (++s == p.stages) { s = 0; ph ^= 1u; }
+          if (++a == p.num_a) a = 0;
+          if (++d == p.num_d) { d = 0; ph_d ^= 1u; d_wrapped = true; }
+        }
+        continue;
+      }
       for (int kb = c.kb0(p), kb_end = c.kb1(p); kb < kb_end; ++kb) {
         if (!(ok = warp_all(mbar_wait(&sh->full[s], ph, &sh->abort_flag, p.status, 4)))) break;
         tc_fence_after();
@@ -486,16 +525,26 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const __grid_cons
     bool ok = true;
     for (int it = grp; it < total_it && ok; it += p.groups) {
       if (!(ok = warp_all(mbar_wait(&sh->w_full[sw], ph_w, &sh->abort_flag, p.status, 6)))) break;
-      const uint4* src = reinterpret_cast<const uint4*>(w_smem + (size_t)sw * kWTileBytes) + r;
+      const uint4* src = reinterpret_cast<const uint4*>(w_smem + (size_t)sw * kTileBytes) + r;
       uint32_t regs[32];
+      if (W8) {
+        // 8-bit weights: the tile already holds int8 codes, 16-byte piece (c, r) = codes k = 16 c .. + 15 of
+        // channel r; they go to tensor memory as they are
 #pragma unroll
-      for (int jj = 0; jj < 4; ++jj) {
-        const uint4 w = src[jj * 128];
-        const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+        for (int c8 = 0; c8 < 8; ++c8) {
+          const uint4 w = src[c8 * 128];
+          regs[c8 * 4] = w.x; regs[c8 * 4 + 1] = w.y; regs[c8 * 4 + 2] = w.z; regs[c8 * 4 + 3] = w.w;
+        }
+      } else {
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          regs[jj * 8 + 2 * i] = (ww[i] << 4) & 0xF0F0F0F0u;   // codes k0..k0+3, each x16
-          regs[jj * 8 + 2 * i + 1] = ww[i] & 0xF0F0F0F0u;      // codes k0+4..k0+7, each x16
+        for (int jj = 0; jj < 4; ++jj) {
+          const uint4 w = src[jj * 128];
+          const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            regs[jj * 8 + 2 * i] = (ww[i] << 4) & 0xF0F0F0F0u;   // codes k0..k0+3, each x16
+            regs[jj * 8 + 2 * i + 1] = ww[i] & 0xF0F0F0F0u;      // codes k0+4..k0+7, each x16
+          }
         }
       }
       const uint32_t dep = __shfl_xor_sync(0xffffffffu, regs[1] ^ regs[9] ^ regs[17] ^ regs[25], 1);  // all lanes' loads done
@@ -531,7 +580,83 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const __grid_cons
     int d = 0;
     uint32_t ph_d = 0;
     bool ok = true;
-    for (TileIter c = first; c.valid(p) && ok; c.next(p)) {
+    if (GROUPED) {
+      // ---- group-wise weight scales (App. A.12: g = 128 = one K block).  s_w is [K / 128][N].  Per tile the
+      // lane that owns channel n keeps one float sum per token column (TN <= 64) and, after every K block,
+      // adds  fl(float(acc_g) * fl(s_a * s_w[g][n]))  in increasing g -- the order the result is defined in.
+      const bool plain_out = !p.acc_out && !p.y_is_f32 && (p.ldy % 8) == 0;
+      for (TileIter c = first; c.valid(p) && ok; c.next(p)) {
+        const int t0 = c.tt * p.TN;
+        const int ncols = min(p.TN, p.T - t0);
+        const int n = c.tn * kTileN + q * 32 + lane;
+        const bool n_ok = n < p.N;
+        // which token columns of the tile are visual rows: bit j of `vis`
+        const int ta = t0 + lane, tb = t0 + 32 + lane;
+        const unsigned lo = __ballot_sync(0xffffffffu, ta < p.T && thread_row_modality(p.seg, ta) == MQ_VISUAL);
+        const unsigned hi = __ballot_sync(0xffffffffu, tb < p.T && thread_row_modality(p.seg, tb) == MQ_VISUAL);
+        const unsigned long long vis = (unsigned long long)lo | ((unsigned long long)hi << 32);
+        float sum[64];
+#pragma unroll
+        for (int j = 0; j < 64; ++j) sum[j] = 0.0f;
+        const float* swg = p.s_w + n;
+        float sw_next = n_ok ? swg[(size_t)c.kb0(p) * p.N] : 0.0f;
+        for (int kb = c.kb0(p), kb_end = c.kb1(p); kb < kb_end && ok; ++kb) {
+          const float swv = sw_next;
+          if (kb + 1 < kb_end) sw_next = n_ok ? swg[(size_t)(kb + 1) * p.N] : 0.0f;  // in flight during this block
+          const float cv = __fmul_rn(p.s_vis, swv), ct = __fmul_rn(p.s_txt, swv);
+          if (!(ok = warp_all(mbar_wait(&sh->d_full[d], ph_d, &sh->abort_flag, p.status, 8)))) break;
+          tc_fence_after();
+          const uint32_t d_tmem = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(d * p.d_stride);
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            if (h * 32 < ncols) {  // warp-uniform
+              uint32_t v0[16], v1[16];
+              tmem_ld_x16(d_tmem + h * 32, v0);
+              tmem_ld_x16(d_tmem + h * 32 + 16, v1);
+              tmem_wait_ld();
+              if (h == 1 || ncols <= 32) {  // the accumulator has been read: hand it back to the MMA warp
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sh->d_empty[d]);
+              }
+#pragma unroll
+              for (int j = 0; j < 32; ++j) {
+                const int col = h * 32 + j;
+                const int acc = ((int)(j < 16 ? v0[j] : v1[j - 16])) >> 4;  // the MMA saw 16 * q_w
+                if (p.acc_out && n_ok && col < ncols) p.acc_out[((size_t)kb * p.T + t0 + col) * p.N + n] = acc;
+                const float cs = ((vis >> col) & 1ull) ? cv : ct;
+                sum[col] = __fadd_rn(sum[col], __fmul_rn((float)acc, cs));
+              }
+            }
+          }
+          if (++d == p.num_d) { d = 0; ph_d ^= 1u; }
+        }
+        if (!ok) break;
+        const float bs = (n_ok && p.bias) ? p.bias[n] : 0.0f;
+#pragma unroll
+        for (int cc = 0; cc < 64; cc += 16) {
+          if (cc < ncols) {  // warp-uniform
+            float y[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) y[j] = p.bias ? __fadd_rn(sum[cc + j], bs) : sum[cc + j];
+            const int nvalid = min(16, ncols - cc);
+            if (plain_out) {
+              staged_store(p, y, t0 + cc, nvalid, n, stage);
+            } else if (n_ok) {
+#pragma unroll
+              for (int j = 0; j < 16; ++j) {
+                if (j < nvalid) {
+                  const size_t t = (size_t)(t0 + cc + j);
+                  if (p.y_is_f32) static_cast<float*>(p.Y)[t * p.ldy + n] = y[j];
+                  else static_cast<__nv_bfloat16*>(p.Y)[t * p.ldy + n] = __float2bfloat16_rn(y[j]);
+                }
+              }
+            }
+          }
+        }
+      }
+    }
+    for (TileIter c = first; !GROUPED && c.valid(p) && ok; c.next(p)) {
       const int t0 = c.tt * p.TN;
       __syncwarp();
       for (int j = lane; j < p.TN; j += 32) {
@@ -557,11 +682,12 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const __grid_cons
           else epilogue_tile_side<false>(p, d_tmem, t0, n, n_ok, sw, sws, bs, stok, stage);
         }
       } else {
+        constexpr int X = W8 ? kEpiNoShift : 0;
         switch (epi_mode) {
-#define MQ_EPI_CASE(M) case M: epilogue_tile<M>(p, d_tmem, t0, n, n_ok, sw, bs, stok, stage, c.ks); break;
+#define MQ_EPI_CASE(M) case M: epilogue_tile<(M) | X>(p, d_tmem, t0, n, n_ok, sw, bs, stok, stage, c.ks); break;
           MQ_EPI_CASE(kEpiStaged) MQ_EPI_CASE(kEpiStaged | kEpiBias) MQ_EPI_CASE(kEpiSplitK)
 #undef MQ_EPI_CASE
-          default: epilogue_tile<kEpiGeneric>(p, d_tmem, t0, n, n_ok, sw, bs, stok, stage, c.ks); break;
+          default: epilogue_tile<kEpiGeneric | X>(p, d_tmem, t0, n, n_ok, sw, bs, stok, stage, c.ks); break;
         }
       }
       tc_fence_before();
@@ -634,25 +760,30 @@ struct Plan {
 // rms: the launch carries a split accumulator next to every accumulator (rotation magnitude
 // suppression), so a token tile may use at most 224 of the 512 tensor-memory columns twice over,
 // there is a single accumulator pair, and what is left (>= 64 columns) holds the weight slots.
-Plan make_plan(int T, int K, int N, bool rms = false) {
+Plan make_plan(int T, int K, int N, int mode = kPlain) {
   Plan pl{};
+  const bool rms = mode == kRms, grouped = mode == kGrouped;
+  const int wtile = mode == kW8 ? 2 * kWTileBytes : kWTileBytes;
   const int sms = sm_count();
   pl.n_tn = (N + kTileN - 1) / kTileN;
   const int kb_total = (K + kBlockK - 1) / kBlockK;
   // Token tile.  Candidates: T cut into n_tt even tiles (multiple of 16, at most tn_cap tokens).
   // Each is rated with a small model of the kernel: a CTA runs `rounds` tiles one after the
-  // other; a K block costs four MMAs whose duration is flat up to 192 tokens and grows beyond
-  // (measured: 112 cycles up to N = 192, 120 at 224, 136 at 256); the epilogue (~25 cycles per
-  // token column) hides behind the next tile's main loop only when two accumulators fit
-  // (tiles of <= 192 tokens).  The cheapest candidate wins; ties go to the larger tile.
-  const int tn_cap = rms ? 224 : 256;
+  // other; the period of a K block in this kernel was found flat up to 192 tokens and growing beyond
+  // (112 cycles per MMA slot up to 192 tokens, 120 at 224, 136 at 256: an empirical figure of the whole
+  // pipeline -- the MMA alone takes 10 + N / 2 cycles); the epilogue (~25 cycles per token column)
+  // hides behind the next tile's main loop only when two accumulators fit (tiles of <= 192 tokens).
+  // The cheapest candidate wins; ties go to the larger tile.
+  // Group-wise weight scales: the epilogue keeps one float sum per token column in registers, so the
+  // tile is at most 64 tokens; its accumulators alternate per K block.
+  const int tn_cap = grouped ? 64 : (rms ? 224 : 256);
   int n_tt = (T + tn_cap - 1) / tn_cap;
   int TN = (((T + n_tt - 1) / n_tt) + 15) / 16 * 16;
   // The search runs when a CTA gets several tiles, and when every CTA gets one tile of more than
   // 192 tokens although smaller tiles would still fit the machine in one round (their MMAs are
   // cheaper); otherwise the fewest tiles are right.
   const bool multi_round = (long long)pl.n_tn * n_tt > sms;
-  if (multi_round || TN > 192) {
+  if (!grouped && (multi_round || TN > 192)) {
     double best = 0.0;
     const int n_min = n_tt;
     for (int cand = n_min; cand <= n_min * 4 && cand <= (T + 15) / 16; ++cand) {
@@ -685,12 +816,17 @@ Plan make_plan(int T, int K, int N, bool rms = false) {
     pl.num_d = 1;
     pl.a_base = 2 * pl.d_stride;
   }
+  if (grouped) {
+    pl.d_stride = 64;
+    pl.num_d = 2;
+    pl.a_base = 128;
+  }
   pl.num_a = (512 - pl.a_base) / 32;
   if (pl.num_a > kMaxStages) pl.num_a = kMaxStages;
   // split K when the tiles alone cannot fill the machine (small T: weight streaming)
   const long long tiles = (long long)pl.n_tn * n_tt;
   int ksplit = 1;
-  if (tiles * 2 <= sms) {
+  if (!grouped && tiles * 2 <= sms) {  // (group sums are added in K order: no K split)
     ksplit = (int)(sms / tiles);
     const int max_split = kb_total / 4 > 0 ? kb_total / 4 : 1;  // keep >= 4 K blocks per CTA
     if (ksplit > max_split) ksplit = max_split;
@@ -710,14 +846,14 @@ Plan make_plan(int T, int K, int N, bool rms = false) {
   // the rest to the weight ring
   const int act_stage = TN * kBlockK;
   const size_t fixed = 1024 + sizeof(Barriers) + 4 * 256 * sizeof(float) + 4 * 16 * 32 * 2;
-  int stages = (int)((kSmemBudget - fixed - 4 * (size_t)kWTileBytes) / act_stage);
+  int stages = (int)((kSmemBudget - fixed - 4 * (size_t)wtile) / act_stage);
   if (stages > kMaxStages) stages = kMaxStages;
   if (stages < pl.num_a) pl.num_a = stages;
-  int w_stages = (int)((kSmemBudget - fixed - (size_t)stages * act_stage) / kWTileBytes);
+  int w_stages = (int)((kSmemBudget - fixed - (size_t)stages * act_stage) / wtile);
   if (w_stages > kMaxWStages) w_stages = kMaxWStages;
   pl.stages = stages;
   pl.w_stages = w_stages;
-  pl.smem = fixed + (size_t)stages * act_stage + (size_t)w_stages * kWTileBytes;
+  pl.smem = fixed + (size_t)stages * act_stage + (size_t)w_stages * wtile;
   pl.groups = 2;
   if (pl.groups > pl.num_a) pl.groups = pl.num_a;
   if (pl.groups > pl.w_stages) pl.groups = pl.w_stages;
@@ -729,10 +865,15 @@ Plan make_plan(int T, int K, int N, bool rms = false) {
 
 }  // namespace
 
-size_t gemm_splitk_bytes(int T, int K, int N, bool rms) {
+static int mode_of(bool rms, int group_size, int w_bits) {
+  return rms ? kRms : (group_size ? kGrouped : (w_bits == 8 ? kW8 : kPlain));
+}
+
+size_t gemm_splitk_bytes(int T, int K, int N, bool rms, int group_size, int w_bits) {
   if (T <= 0 || K <= 0 || N <= 0) return 0;
-  if (!rms && gemv_applies(T, K, N)) return 0;  // the GEMV path reduces inside its CTAs
-  const Plan pl = make_plan(T, K, N, rms);
+  const int mode = mode_of(rms, group_size, w_bits);
+  if (mode == kPlain && gemv_applies(T, K, N)) return 0;  // the GEMV path reduces inside its CTAs
+  const Plan pl = make_plan(T, K, N, mode);
   // one [T,N] slice per K split, and one more for the split accumulator
   return pl.ksplit > 1 ? (size_t)(pl.ksplit + (rms ? 1 : 0)) * T * N * sizeof(int32_t) : 0;
 }
@@ -740,8 +881,11 @@ size_t gemm_splitk_bytes(int T, int K, int N, bool rms) {
 int launch_gemm(const GemmArgs& a, cudaStream_t st) {
   if (a.T == 0 || a.N == 0) return MQ_OK;
   const bool rms = a.side_layout != nullptr;
-  if (!rms && gemv_applies(a.T, a.K, a.N)) return launch_gemv(a, st);  // one to four tokens: see mq_gemv.cu
-  const Plan pl = make_plan(a.T, a.K, a.N, rms);
+  const int mode = mode_of(rms, a.group_size, a.w_bits);
+  if (rms && (a.group_size || a.w_bits == 8)) return MQ_ERR_UNSUPPORTED;
+  if (a.group_size && (a.group_size != kBlockK || a.K % kBlockK || a.row_scales || a.w_bits == 8)) return MQ_ERR_UNSUPPORTED;
+  if (mode == kPlain && gemv_applies(a.T, a.K, a.N)) return launch_gemv(a, st);  // one to four tokens: see mq_gemv.cu
+  const Plan pl = make_plan(a.T, a.K, a.N, mode);
   EncodeTiledFn encode = get_encode_fn();
   if (!encode) return MQ_ERR_CUDA;
 
@@ -767,9 +911,11 @@ int launch_gemm(const GemmArgs& a, cudaStream_t st) {
       return MQ_ERR_CUDA;
   }
 
-  auto kernel = rms ? w4a8_gemm_kernel<true> : w4a8_gemm_kernel<false>;
-  static PerDeviceTable<char> attr_set[2];
-  if (!ensure_dynamic_smem(attr_set[rms ? 1 : 0], kernel, kSmemBudget)) return MQ_ERR_CUDA;
+  auto kernel = mode == kRms ? w4a8_gemm_kernel<kRms>
+                             : (mode == kGrouped ? w4a8_gemm_kernel<kGrouped>
+                                                 : (mode == kW8 ? w4a8_gemm_kernel<kW8> : w4a8_gemm_kernel<kPlain>));
+  static PerDeviceTable<char> attr_set[4];
+  if (!ensure_dynamic_smem(attr_set[mode], kernel, kSmemBudget)) return MQ_ERR_CUDA;
 
   KernelParams p{};
   p.T = a.T; p.K = a.K; p.N = a.N;

@@ -67,11 +67,14 @@ def test_linear_argument_validation(lib):
     assert call(_desc(K=100)) == B.MQ_ERR_INVALID_ARG
     assert call(_desc(N=100)) == B.MQ_ERR_INVALID_ARG
     assert call(_desc(T=-1)) == B.MQ_ERR_INVALID_ARG
-    assert call(_desc(group=128)) == B.MQ_ERR_UNSUPPORTED
+    assert call(_desc(group=64)) == B.MQ_ERR_UNSUPPORTED                      # a weight group is one K block of 128
+    assert call(_desc(group=-128)) == B.MQ_ERR_INVALID_ARG
+    assert call(_desc(K=160, group=128), ldx=160) == B.MQ_ERR_INVALID_ARG     # K must be whole groups
+    assert call(_desc(group=128, flags=B.MQ_FLAG_W8)) == B.MQ_ERR_UNSUPPORTED
     assert call(_desc(rot=16)) == B.MQ_ERR_UNSUPPORTED
     assert call(_desc(rot=96)) == B.MQ_ERR_INVALID_ARG
     assert call(_desc(K=384, rot=256), ldx=384) == B.MQ_ERR_INVALID_ARG      # rotation block must divide K
-    assert call(_desc(flags=8)) == B.MQ_ERR_INVALID_ARG
+    assert call(_desc(flags=16)) == B.MQ_ERR_INVALID_ARG
     assert call(_desc(rot=128, flags=B.MQ_FLAG_X_IS_INT8)) == B.MQ_ERR_INVALID_ARG
     assert call(_desc(K=1 << 20), ldx=1 << 20) == B.MQ_ERR_UNSUPPORTED
     assert call(_desc(), s_v=0.0) == B.MQ_ERR_INVALID_ARG
@@ -108,7 +111,19 @@ def test_other_entry_points_validate(lib):
     assert c(A, 4, 128, 128, C.byref(seg), 0, 0, None, A, A, None) == B.MQ_ERR_INVALID_ARG
     assert c(A, 4, 128, 128, C.byref(seg), 24, 0, A, A, A, None) == B.MQ_ERR_INVALID_ARG
     p = lib.mq_pack_w4
-    assert p(A, 128, 128, 128, 128, None, A, None, None) == B.MQ_ERR_UNSUPPORTED
+    assert p(A, 128, 128, 128, 64, None, A, None, None) == B.MQ_ERR_UNSUPPORTED
+    assert p(A, 128, 160, 160, 128, None, A, None, None) == B.MQ_ERR_INVALID_ARG
+    p8 = lib.mq_pack_w8
+    assert p8(A, 128, 128, 128, None, 0, A, None, None) == B.MQ_ERR_INVALID_ARG       # neither codes nor layout wanted
+    assert p8(A, 128, 128, 128, A, 64, A, None, None) == B.MQ_ERR_INVALID_ARG         # ldq < K
+    assert p8(A, 128, 128, 128, None, 0, A, A + 16, None) == B.MQ_ERR_ALIGNMENT
+    assert B.mq_w8_layout_bytes(3584, 18944) == 2 * B.mq_w4_layout_bytes(3584, 18944)
+    qb = lib.mq_fwht_quant_bits
+    assert qb(A, 4, 128, 128, C.byref(seg), 1.0, 1.0, 0, 5, A, 128, None) == B.MQ_ERR_UNSUPPORTED
+    assert qb(A, 4, 128, 128, C.byref(seg), 1.0, 0.0, 0, 4, A, 128, None) == B.MQ_ERR_INVALID_ARG
+    cb = lib.mq_calibrate_static_scales_bits
+    assert cb(A, 4, 128, 128, C.byref(seg), 0, 3, 0, A, A, A, None) == B.MQ_ERR_UNSUPPORTED
+    assert cb(A, 4, 128, 128, C.byref(seg), 0, 4, 0, None, A, A, None) == B.MQ_ERR_INVALID_ARG
     assert p(A, 128, 100, 100, 0, None, A, None, None) == B.MQ_ERR_INVALID_ARG
     assert p(A, 128, 128, 128, 0, None, None, None, None) == B.MQ_ERR_INVALID_ARG
     assert p(A, 128, 128, 128, 0, None, A, A + 16, None) == B.MQ_ERR_ALIGNMENT
