@@ -159,6 +159,93 @@ def run_reference(args, info):
     print(json.dumps(line), flush=True)
 
 
+# ------------------------------------------------------------------------------------------ tensor-pipe microbenchmark
+def mma_issue_microbenchmark(torch, B, dev, n_sms):
+    """tcgen05.mma kind::i8 with fixed operands and no loads (the library's own probe): cycles per
+    128 x N x 32 instruction on every SM at once, for the token-tile widths the GEMM uses."""
+    out = {}
+    n_mma = 4096
+    for n_tok in (64, 128, 192, 224, 256):
+        cyc = torch.zeros(n_sms, dtype=torch.int64, device=dev)
+        st = torch.zeros(2, dtype=torch.int32, device=dev)
+        for _ in range(2):
+            B.mq_ubench_mma_i8(n_tok, n_mma, 1, 0, n_sms, cyc, st)
+        torch.cuda.synchronize()
+        per = float(cyc.double().mean()) / n_mma
+        out["N%d" % n_tok] = {"cycles_per_mma": per, "ops_per_clk_sm": 2.0 * 128 * n_tok * 32 / per,
+                              "status_ok": st.tolist() == [0, 0]}
+    return out
+
+
+def gemm_traffic_record():
+    """DRAM bytes of one GEMM launch on the bench workload, from the ncu capture summarised under
+    profiles/: valid only while the kernel source is the one that was captured."""
+    import hashlib
+    path = os.path.join(ROOT, "profiles", "w4a8_gemm_config2_traffic.json")
+    src = os.path.join(ROOT, "paper_2502_00425_b200", "csrc", "mq_gemm.cu")
+    try:
+        with open(path) as f:
+            rec = json.load(f)
+        with open(src, "rb") as f:
+            sha = hashlib.sha256(f.read()).hexdigest()
+    except Exception:
+        return None, None
+    if rec.get("mq_gemm_cu_sha256") != sha:
+        return None, dict(rec, stale="mq_gemm.cu has changed since the capture")
+    return rec.get("dram_bytes_per_launch"), rec
+
+
+def variants_timing(torch, B, dev, T, K, N, rot, n_sets=4, reps=10):
+    """The neighbouring settings on the config-2 shape, each as rotation + quantizer + GEMM (CUDA-graph
+    replays over n_sets rotating copies, larger than L2 in total; random valid weight bytes: timing only,
+    parity is covered by the tests): W4A8 per-channel (the hot path), group-wise W4 (g = 128), W8A8, W4A4."""
+    g = torch.Generator(device="cpu").manual_seed(14)
+    seg = B.Segments.from_host([T - 64, T], [1, 0], dev)
+    G = K // 128
+    sets = []
+    for _ in range(n_sets):
+        x = (torch.randn((T, K), generator=g, dtype=torch.float32) * 2).to(torch.bfloat16).to(dev)
+        lay4 = torch.randint(0, 256, (B.mq_w4_layout_bytes(N, K),), dtype=torch.uint8, generator=g).to(dev)
+        lay8 = torch.randint(0, 256, (B.mq_w8_layout_bytes(N, K),), dtype=torch.uint8, generator=g).to(dev)
+        s_w = (torch.rand(N, generator=g) * 0.01 + 0.001).to(dev)
+        s_wg = (torch.rand((G, N), generator=g) * 0.01 + 0.001).to(dev)
+        y = torch.empty((T, N), dtype=torch.bfloat16, device=dev)
+        sets.append({"x": x, "lay4": lay4, "lay8": lay8, "s_w": s_w, "s_wg": s_wg, "y": y,
+                     "ws": B.new_workspace(T, K, N, rot), "ws_g": B.new_workspace(T, K, N, rot, group_size=128),
+                     "ws_8": B.new_workspace(T, K, N, rot, B.MQ_FLAG_W8), "ws_a4": B.new_workspace(T, K, N, rot, B.MQ_FLAG_A4)})
+    fns = {
+        "w4a8_per_channel_us": lambda s_: B.mq_w4a8_msq_linear(s_["x"], seg, 0.5, 0.05, s_["lay4"], s_["s_w"], s_["y"], s_["ws"], N, rot_block=rot),
+        "w4a8_g128_us": lambda s_: B.mq_w4a8_msq_linear(s_["x"], seg, 0.5, 0.05, s_["lay4"], s_["s_wg"], s_["y"], s_["ws_g"], N, rot_block=rot, group_size=128),
+        "w8a8_us": lambda s_: B.mq_w4a8_msq_linear(s_["x"], seg, 0.5, 0.05, s_["lay8"], s_["s_w"], s_["y"], s_["ws_8"], N, rot_block=rot, extra_flags=B.MQ_FLAG_W8),
+        "w4a4_us": lambda s_: B.mq_w4a8_msq_linear(s_["x"], seg, 0.5, 0.05, s_["lay4"], s_["s_w"], s_["y"], s_["ws_a4"], N, rot_block=rot, extra_flags=B.MQ_FLAG_A4),
+    }
+    out = {}
+    for name, fn in fns.items():
+        for s_ in sets:
+            fn(s_)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            for s_ in sets:
+                fn(s_)
+        graph.replay()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            graph.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        out[name] = e0.elapsed_time(e1) * 1e3 / (reps * n_sets)
+        del graph
+    ok = all(B.mq_last_device_status(s_[k])[0] == 0 for s_ in sets for k in ("ws", "ws_g", "ws_8", "ws_a4"))
+    ops = 2.0 * T * K * N
+    out.update({"workload": "config2 down_proj T=%d K=%d N=%d rot=%d: quantizer + GEMM" % (T, K, N, rot),
+                "tops": {k[:-3]: ops / (v * 1e-6) / 1e12 for k, v in out.items() if k.endswith("_us")},
+                "status_ok": ok})
+    return out
+
+
 # ------------------------------------------------------------------------------------------ decode sweep
 def decode_sweep(torch, B, dev, peaks, n_sets=6, reps=20):
     """Config-5-shaped decode steps: the linears of a 4096 / 13696 SwiGLU MLP (gate, up: 4096 -> 13696;
@@ -210,14 +297,40 @@ def decode_sweep(torch, B, dev, peaks, n_sets=6, reps=20):
             e1.record()
             torch.cuda.synchronize()
             sec = e0.elapsed_time(e1) * 1e-3 / (reps * n_sets)
+            del graph
+            # every linear of the arrangement alone (the same call, rotating weight sets)
+            per_linear = []
+            for j, (K, N, rot) in enumerate(shapes):
+                def one(i, j=j, K=K, N=N, rot=rot):
+                    lay, s_w = weights[i % n_sets][j]
+                    B.mq_w4a8_msq_linear(xs[j], seg, 1.0, 0.05, lay, s_w, ys[j], wss[j], N, rot_block=rot)
+                g1 = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g1):
+                    for i in range(n_sets):
+                        one(i)
+                g1.replay()
+                torch.cuda.synchronize()
+                e0.record()
+                for _ in range(reps):
+                    g1.replay()
+                e1.record()
+                torch.cuda.synchronize()
+                us = e0.elapsed_time(e1) * 1e3 / (reps * n_sets)
+                del g1
+                per_linear.append({"K": K, "N": N, "us": us, "weight_gbs": N * K / 2 / us / 1e3})
             status = [B.mq_last_device_status(w)[0] for w in wss]
             gbs = w_bytes / sec / 1e9
             res["T%d" % T] = {"us_per_mlp": sec * 1e6, "weight_gbs": gbs, "frac_of_measured_hbm": gbs / peaks["hbm_gbs"],
+                              "frac_of_nominal_8tbs": gbs / 8000.0, "per_linear": per_linear,
+                              "kernel": ("w4a8_gemv_kernel (rotation + quantizer + dp4a product in one launch)" if T <= 4 else
+                                         "fwht_quant_kernel + w4a8_gemm_kernel (+ splitk_finalize_kernel when K is split)"),
                               "tokens_per_s": T / sec, "status_ok": all(v == 0 for v in status)}
-            del graph
         out[name] = res
         del weights
         torch.cuda.empty_cache()
+    out["roofline"] = {"bound": "hbm", "bytes": "packed int4 weights of the three linears: %d B per MLP pass" % w_bytes,
+                       "peak_measured_gbs": peaks["hbm_gbs"], "peak_nominal_gbs": 8000.0,
+                       "timing": "CUDA-graph replays of %d MLP passes over rotating weight sets, CUDA events" % n_sets}
     out["workload"] = ("config5: 4096/13696 MLP (gate, up, down with 128-block rotation), %d weight sets of %.0f MB "
                        "cycled" % (n_sets, w_bytes / 1e6))
     return out
@@ -458,9 +571,6 @@ class BufferSet:
         return sum(t.numel() * t.element_size() for t in (self.x, self.layout, self.ws, self.y, self.emb, self.emb_u))
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one w4a8_gemm_kernel launch on this workload
-# (ncu capture summarised in profiles/); None once the kernel has changed since the capture.
-GEMM_TRAFFIC_BYTES = 57.43e6
 LAUNCHES_PER_STEP = 4  # fused AIFS index + gather, remap, rotation + quantizer, GEMM
 
 
@@ -729,7 +839,14 @@ def run_ours(args, info):
     e2e_ops, _ = D.aggregate_throughput(ops_per_step() * e2e_steps, e0.elapsed_time(e1) * 1e-3, dev)
 
     # ---- decode-shaped sweep (rank 0, N = 1 only): the HBM-bound regime of the same path
-    decode, suites, rms_timing, dyn_timing, layers = None, None, None, None, None
+    decode, suites, rms_timing, dyn_timing, layers, var_timing = None, None, None, None, None, None
+    n_sms = torch.cuda.get_device_properties(dev).multi_processor_count
+    ubench = None
+    if info.is_main:
+        try:
+            ubench = mma_issue_microbenchmark(torch, B, dev, n_sms)
+        except Exception:
+            ubench = None
     if info.is_main and info.world == 1 and not args.no_decode:
         del graphs, ev_graphs
         decode = decode_sweep(torch, B, dev, peaks)
@@ -741,6 +858,8 @@ def run_ours(args, info):
                                9728, 2304, 128, 4, synth.LLAMA_8B)]
         rms_timing = rms_linear_timing(torch, B, dev, case.T, case.K, case.N, ROT)
         dyn_timing = dynamic_linear_timing(torch, B, dev, case.T, case.K, case.N, ROT)
+        torch.cuda.empty_cache()
+        var_timing = variants_timing(torch, B, dev, case.T, case.K, case.N, ROT)
         torch.cuda.empty_cache()
         layers = [layer_mode_timing(torch, dev, "config3: Qwen2-7B-shaped block, one sequence of 3360 tokens",
                                     synth.QWEN2_7B, [synth.config3_sequence()]),
@@ -758,13 +877,42 @@ def run_ours(args, info):
         cpu = {"value": ops_per_step() / float(np.median(times)) / 1e12, "unit": UNIT, "cores": host_threads(),
                "kind": "oracle", "sample": "the full config-2 workload (1088 rows), median of 3 passes",
                "seconds_per_pass": float(np.median(times))}
+        try:  # the same oracle confined to one thread, on a 64-row sample (the library matmul is its only threaded step)
+            from threadpoolctl import threadpool_limits
+            sample = oracle_sample_rows()[::4]
+            with threadpool_limits(limits=1):
+                t1 = time_oracle(case, qw, sw_ref, o_v, o_t, sample, 2)
+            cpu["single_thread"] = {"value": ops_per_step(len(sample)) / float(np.min(t1)) / 1e12, "unit": UNIT, "cores": 1,
+                                    "sample": "%d of 1088 rows, best of 2 passes" % len(sample)}
+        except Exception:
+            pass
+        # the reading of x / s (multiply by the float32 reciprocal) against Eq. 2's literal division, on this batch
+        r_rot = O.fwht_blocks(case.x, ROT, np.float32)
+        s_rows = O.row_scales(case.T, case.seg.seg_end, case.seg.seg_mod, o_v, o_t)
+        differ = int((O.quantize_act_int8(r_rot, s_rows) != O.quantize_act_int8_divide(r_rot, s_rows)).sum())
+        cpu["codes_differing_reciprocal_vs_division"] = {"differ": differ, "codes": int(r_rot.size)}
 
     if info.is_main:
         gemm_tops = ops_per_step() / kern["gemm"] / 1e12
+        linear_tops = ops_per_step() / (kern["gemm"] + kern["fwht_quant"]) / 1e12
         timed_s = t_max
         sustained = timed_s > 1.0
         peak = 2.0 * (peaks["bf16_sustained"] if sustained else peaks["bf16_burst"])
         quant_bytes = case.T * case.K * 3
+        traffic, traffic_rec = gemm_traffic_record()
+        # the tensor pipe's own rate on this machine: the issue-only microbenchmark at the widest tile, at
+        # the SM clock sampled during the timed region and at the maximum clock
+        sm_mhz = clocks.get("sm_mhz") or clocks.get("sm_max_mhz") or 1965.0
+        sm_max = clocks.get("sm_max_mhz") or 1965.0
+        ub = ubench["N256"]["ops_per_clk_sm"] if ubench else None
+        ub_sampled = ub * n_sms * sm_mhz * 1e6 / 1e12 if ub else None
+        ub_max = ub * n_sms * sm_max * 1e6 / 1e12 if ub else None
+        denominators = {
+            "measured_bf16_burst_x2": 2.0 * peaks["bf16_burst"], "measured_bf16_sustained_x2": 2.0 * peaks["bf16_sustained"],
+            "nominal_dense_int8": 4500.0, "mma_microbenchmark_at_sampled_clock": ub_sampled,
+            "mma_microbenchmark_at_max_clock": ub_max,
+            "ncu_tensor_pipe_pct_of_elapsed": (traffic_rec or {}).get("sm__pipe_tensor_cycles_active_pct_of_elapsed")}
+        fracs = lambda tops: {k: (tops / v if v else None) for k, v in denominators.items() if k != "ncu_tensor_pipe_pct_of_elapsed"}
         line = {
             "metric": METRIC, "value": value_ops / 1e12, "unit": UNIT, "n_gpus": info.world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": 1e3 * t_max / args.steps, "higher_is_better": True,
@@ -784,7 +932,14 @@ def run_ours(args, info):
                          "unit": "TOP/s", "frac": gemm_tops / peak,
                          "peak_kind": "2 x measured bf16 %s (%s)" % ("sustained" if sustained else "burst",
                                                                       peaks["source"]),
-                         "traffic": GEMM_TRAFFIC_BYTES, "traffic_unit": "bytes per launch (ncu, profiles/)",
+                         "denominators_tops": denominators, "frac_by_denominator": fracs(gemm_tops),
+                         "linear": {"what": "fwht_quant_kernel + w4a8_gemm_kernel (the prefill W4A8 MSQ linear)",
+                                    "achieved": linear_tops, "frac_by_denominator": fracs(linear_tops)},
+                         "step": {"what": "the whole timed step", "achieved": value_ops / 1e12 / info.world,
+                                  "frac_by_denominator": fracs(value_ops / 1e12 / info.world)},
+                         "mma_microbenchmark": ubench,
+                         "traffic": traffic, "traffic_unit": "bytes per launch (ncu, profiles/)",
+                         "traffic_record": traffic_rec,
                          "algorithmic_bytes": case.T * case.K + case.N * case.K // 2 + 4 * case.N
                          + 2 * case.T * case.N,
                          "avg_kernel_us": kern["gemm"] * 1e6,
@@ -800,6 +955,7 @@ def run_ours(args, info):
             "layer_linear_suites": suites,
             "rms_linear": rms_timing,
             "static_vs_dynamic_a8": dyn_timing,
+            "variants": var_timing,
             "layer_mode": layers,
             "device_status": list(status),
             "cpu_baseline": cpu,

@@ -267,10 +267,13 @@ int mq_w4a8_msq_linear(const mq_linear_desc* d, const void* X, int64_t ldx,
  * cudaFree and calls no allocating library routine.
  *
  *  - Limit: mq_workspace_bytes(d) must not exceed MQ_NOALLOC_WS_BYTES, otherwise
- *    MQ_ERR_WORKSPACE is returned and nothing is enqueued.  That covers decode-shaped
- *    problems (for example T = 128, K = 13696, N = 4096); prefill-sized ones need
- *    mq_w4a8_msq_linear.  The array occupies that much memory on every device the
- *    library is used on, until the process exits.
+ *    MQ_ERR_WORKSPACE is returned and nothing is enqueued.  The workspace holds the int8
+ *    codes (T * K bytes) and, where the launch splits K, one [T, N] int32 slice per split,
+ *    so the limit depends on the shape: ask mq_workspace_bytes.  Decode-shaped problems
+ *    fit (for example K = 4096, N = 13696 up to T = 256; K = 13696, N = 4096, which splits
+ *    K four ways, up to T = 48 -- T = 64 there needs 5,071,104 bytes and is refused);
+ *    prefill-sized ones need mq_w4a8_msq_linear.  The array occupies that much memory on
+ *    every device the library is used on, until the process exits.
  *  - Set-up: the first call on each device looks up the array's device address (with that
  *    device current).  Make that first call outside any stream capture.
  *  - Sharing: every call on a device uses the same array, which keeps what the previous

@@ -11,9 +11,11 @@
 // them the scratch lives in a fixed array that is part of this library's device image.
 //
 // Cost and limit.  The array is MQ_NOALLOC_WS_BYTES (4 MiB) of global memory on EVERY
-// device that loads the library, held until the process exits.  It is sized for the
-// decode-shaped calls (a few hundred tokens at most); larger problems are rejected with
-// MQ_ERR_WORKSPACE and must use mq_w4a8_msq_linear with a caller-owned workspace.
+// device that loads the library, held until the process exits.  It is sized for
+// decode-shaped calls: the int8 codes (T * K bytes) plus one [T, N] int32 slice per K split
+// must fit, which admits e.g. K = 4096, N = 13696 up to T = 256 but K = 13696, N = 4096
+// (four K splits) only up to T = 48.  Larger problems are rejected with MQ_ERR_WORKSPACE
+// and must use mq_w4a8_msq_linear with a caller-owned workspace.
 //
 // The array's name is only a handle in host code -- it is not a device address -- so the
 // address is looked up with cudaGetSymbolAddress, once per device, with that device
@@ -63,8 +65,8 @@ extern "C" int mq_w4a8_msq_linear_noalloc(const mq_linear_desc* d, const void* X
   if (!ws) return MQ_ERR_CUDA;
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
   // The array keeps whatever the previous call left.  The status word is sticky, so it must
-  // start from MQ_OK; the activation codes are fully rewritten and the split-K sums are
-  // zeroed by the GEMM launcher itself.
+  // start from MQ_OK; the activation codes are fully rewritten, and every K split overwrites
+  // its own [T, N] slice with plain stores before the finalize kernel reads it.
   if (cudaMemsetAsync(ws, 0, mq::kStatusBytes, cs) != cudaSuccess) return MQ_ERR_CUDA;
   const int rc = mq_w4a8_msq_linear(d, X, ldx, seg, s_vis, s_txt, W_layout, s_w, bias, Y, ldy, acc_out, ws,
                                     (size_t)MQ_NOALLOC_WS_BYTES, stream);

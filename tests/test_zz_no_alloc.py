@@ -28,6 +28,13 @@ def test_noalloc_rejects_oversized_problems_on_the_host():
                                         None, None, None)
     assert rc == B.MQ_ERR_WORKSPACE
     assert B.status_string(rc) == "MQ_ERR_WORKSPACE"
+    # the limits the header documents for the decode shapes of a 4096 / 13696 MLP
+    assert B.mq_workspace_bytes(256, 4096, 13696, 0) <= B.MQ_NOALLOC_WS_BYTES
+    assert B.mq_workspace_bytes(48, 13696, 4096, 128) <= B.MQ_NOALLOC_WS_BYTES
+    assert B.mq_workspace_bytes(64, 13696, 4096, 128) == 5071104 > B.MQ_NOALLOC_WS_BYTES
+    d = B.mq_linear_desc(64, 13696, 4096, 128, 0, 0)
+    assert lib.mq_w4a8_msq_linear_noalloc(C.byref(d), None, 13696, None, 1.0, 1.0, None, None, None, None, 4096,
+                                          None, None, None) == B.MQ_ERR_WORKSPACE
     bad = B.mq_linear_desc(8, 100, 128, 0, 0, 0)     # K % 32 != 0: same verdict as the main entry point
     rc = lib.mq_w4a8_msq_linear_noalloc(C.byref(bad), None, 100, None, 1.0, 1.0, None, None, None, None, 128,
                                         None, None, None)
