@@ -335,7 +335,8 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const __grid_cons
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmap_act)) : "memory");
     for (int i = 0; i < p.stages; ++i) { mbar_init(&sh->full[i], 1 + 4); mbar_init(&sh->done[i], 1); }
     for (int i = 0; i < p.w_stages; ++i) { mbar_init(&sh->w_full[i], 1); mbar_init(&sh->w_empty[i], 4); }
-    for (int i = 0; i < 2; ++i) { mbar_init(&sh->d_full[i], 1); mbar_init(&sh->d_empty[i], 4); }
+    // every epilogue warp arrives on d_empty: four of them, eight in the group-scale instantiation
+    for (int i = 0; i < 2; ++i) { mbar_init(&sh->d_full[i], 1); mbar_init(&sh->d_empty[i], GROUPED ? 8 : 4); }
     mbar_init(&sh->drain, 1);
     sh->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -584,6 +585,11 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const __grid_cons
       // ---- group-wise weight scales (App. A.12: g = 128 = one K block).  s_w is [K / 128][N].  Per tile the
       // lane that owns channel n keeps one float sum per token column (TN <= 64) and, after every K block,
       // adds  fl(float(acc_g) * fl(s_a * s_w[g][n]))  in increasing g -- the order the result is defined in.
+      // Eight warps fold (one expander group only): warp (q, half) owns lane quarter q and the token columns
+      // 32 half .. 32 half + 31 of the tile.  A single warp issues well below one instruction per cycle, so
+      // two per scheduler roughly double the fold rate.
+      const int half = (warp - (4 + 4 * p.groups)) >> 2;
+      if (half == 1) stage = reinterpret_cast<__nv_bfloat16*>(s_tok) + q * (16 * 32);  // the token-scale table is unused here
       const bool plain_out = !p.acc_out && !p.y_is_f32 && (p.ldy % 8) == 0;
       for (TileIter c = first; c.valid(p) && ok; c.next(p)) {
         const int t0 = c.tt * p.TN;
@@ -594,10 +600,13 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const __grid_cons
         const int ta = t0 + lane, tb = t0 + 32 + lane;
         const unsigned lo = __ballot_sync(0xffffffffu, ta < p.T && thread_row_modality(p.seg, ta) == MQ_VISUAL);
         const unsigned hi = __ballot_sync(0xffffffffu, tb < p.T && thread_row_modality(p.seg, tb) == MQ_VISUAL);
-        const unsigned long long vis = (unsigned long long)lo | ((unsigned long long)hi << 32);
-        float sum[64];
+        float sum[32];
 #pragma unroll
-        for (int j = 0; j < 64; ++j) sum[j] = 0.0f;
+        for (int j = 0; j < 32; ++j) sum[j] = 0.0f;
+        const unsigned vis_h = half ? hi : lo;                 // this warp's 32 columns
+        const int ncols_h = max(0, min(32, ncols - half * 32));
+        const unsigned in_h = ncols_h >= 32 ? 0xffffffffu : ((1u << ncols_h) - 1u);
+        const bool uniform_mod = vis_h == 0u || vis_h == in_h;  // (rows past T count as text: no bit there)
         const float* swg = p.s_w + n;
         float sw_next = n_ok ? swg[(size_t)c.kb0(p) * p.N] : 0.0f;
         for (int kb = c.kb0(p), kb_end = c.kb1(p); kb < kb_end && ok; ++kb) {
@@ -606,26 +615,38 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const __grid_cons
           const float cv = __fmul_rn(p.s_vis, swv), ct = __fmul_rn(p.s_txt, swv);
           if (!(ok = warp_all(mbar_wait(&sh->d_full[d], ph_d, &sh->abort_flag, p.status, 8)))) break;
           tc_fence_after();
-          const uint32_t d_tmem = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(d * p.d_stride);
-#pragma unroll
-          for (int h = 0; h < 2; ++h) {
-            if (h * 32 < ncols) {  // warp-uniform
-              uint32_t v0[16], v1[16];
-              tmem_ld_x16(d_tmem + h * 32, v0);
-              tmem_ld_x16(d_tmem + h * 32 + 16, v1);
-              tmem_wait_ld();
-              if (h == 1 || ncols <= 32) {  // the accumulator has been read: hand it back to the MMA warp
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&sh->d_empty[d]);
-              }
+          const uint32_t d_tmem = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(d * p.d_stride + half * 32);
+          uint32_t v0[16], v1[16];
+          if (ncols_h > 0) {  // warp-uniform
+            tmem_ld_x16(d_tmem, v0);
+            tmem_ld_x16(d_tmem + 16, v1);
+            tmem_wait_ld();
+          }
+          // the accumulator has been read (or is not this warp's to read): hand it back to the MMA warp
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&sh->d_empty[d]);
+          if (ncols_h > 0) {
+            if (p.acc_out && n_ok) {  // debug dump of this group's accumulators
 #pragma unroll
               for (int j = 0; j < 32; ++j) {
-                const int col = h * 32 + j;
-                const int acc = ((int)(j < 16 ? v0[j] : v1[j - 16])) >> 4;  // the MMA saw 16 * q_w
-                if (p.acc_out && n_ok && col < ncols) p.acc_out[((size_t)kb * p.T + t0 + col) * p.N + n] = acc;
-                const float cs = ((vis >> col) & 1ull) ? cv : ct;
-                sum[col] = __fadd_rn(sum[col], __fmul_rn((float)acc, cs));
+                if (j < ncols_h)
+                  p.acc_out[((size_t)kb * p.T + t0 + half * 32 + j) * p.N + n] = ((int)(j < 16 ? v0[j] : v1[j - 16])) >> 4;
+              }
+            }
+            // The MMA saw 16 * q_w: float(16 a) * (c / 16) == float(a) * c bit for bit (powers of two), which
+            // saves the shift; a tile within one modality (the usual case after AIFS) also skips the select.
+            const float cv16 = __fmul_rn(cv, 0.0625f), ct16 = __fmul_rn(ct, 0.0625f);
+            if (uniform_mod) {
+              const float cs = vis_h ? cv16 : ct16;
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                sum[j] = __fadd_rn(sum[j], __fmul_rn((float)(int)(j < 16 ? v0[j] : v1[j - 16]), cs));
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; ++j) {
+                const float cs = ((vis_h >> j) & 1u) ? cv16 : ct16;
+                sum[j] = __fadd_rn(sum[j], __fmul_rn((float)(int)(j < 16 ? v0[j] : v1[j - 16]), cs));
               }
             }
           }
@@ -634,19 +655,20 @@ w4a8_gemm_kernel(const __grid_constant__ CUtensorMap tmap_act, const __grid_cons
         if (!ok) break;
         const float bs = (n_ok && p.bias) ? p.bias[n] : 0.0f;
 #pragma unroll
-        for (int cc = 0; cc < 64; cc += 16) {
-          if (cc < ncols) {  // warp-uniform
+        for (int cc = 0; cc < 32; cc += 16) {
+          if (cc < ncols_h) {  // warp-uniform
             float y[16];
 #pragma unroll
             for (int j = 0; j < 16; ++j) y[j] = p.bias ? __fadd_rn(sum[cc + j], bs) : sum[cc + j];
-            const int nvalid = min(16, ncols - cc);
+            const int nvalid = min(16, ncols_h - cc);
+            const int tc0 = t0 + half * 32 + cc;
             if (plain_out) {
-              staged_store(p, y, t0 + cc, nvalid, n, stage);
+              staged_store(p, y, tc0, nvalid, n, stage);
             } else if (n_ok) {
 #pragma unroll
               for (int j = 0; j < 16; ++j) {
                 if (j < nvalid) {
-                  const size_t t = (size_t)(t0 + cc + j);
+                  const size_t t = (size_t)(tc0 + j);
                   if (p.y_is_f32) static_cast<float*>(p.Y)[t * p.ldy + n] = y[j];
                   else static_cast<__nv_bfloat16*>(p.Y)[t * p.ldy + n] = __float2bfloat16_rn(y[j]);
                 }
@@ -854,7 +876,7 @@ Plan make_plan(int T, int K, int N, int mode = kPlain) {
   pl.stages = stages;
   pl.w_stages = w_stages;
   pl.smem = fixed + (size_t)stages * act_stage + (size_t)w_stages * wtile;
-  pl.groups = 2;
+  pl.groups = grouped ? 1 : 2;  // group scales: the second expander group's warps fold accumulators instead
   if (pl.groups > pl.num_a) pl.groups = pl.num_a;
   if (pl.groups > pl.w_stages) pl.groups = pl.w_stages;
   if (pl.groups < 1) pl.groups = 1;
@@ -943,7 +965,7 @@ int launch_gemm(const GemmArgs& a, cudaStream_t st) {
   }
 
   if (pl.ksplit > 1 && !a.splitk_acc) return MQ_ERR_WORKSPACE;
-  if (cuda_status(launch_pdl(kernel, dim3(pl.grid), dim3((8 + 4 * pl.groups) * 32), pl.smem, st, tmap, tmap_side, p)) != MQ_OK)
+  if (cuda_status(launch_pdl(kernel, dim3(pl.grid), dim3((4 + 4 * pl.groups + (mode == kGrouped ? 8 : 4)) * 32), pl.smem, st, tmap, tmap_side, p)) != MQ_OK)
     return MQ_ERR_CUDA;
   if (pl.ksplit > 1) {
     const int64_t n = (int64_t)a.T * a.N;
