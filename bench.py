@@ -706,14 +706,43 @@ def run_ours(args, info):
             launch_mode = "eager (graph capture failed: %s)" % type(e).__name__
             torch.cuda.synchronize()
 
+    # Steps are independent batches on their own buffer sets.  With --steps-in-flight 2 (the default) they are
+    # issued alternately on two streams, so the small kernels at the head of one step (index, remap, quantizer)
+    # can run while the GEMM of the step before occupies the tensor cores; every kernel of a step still waits
+    # for the kernels it depends on (stream order within the step).  A buffer set comes round again on the
+    # stream it was used on before (n_sets is even), so its reuse is ordered.
+    in_flight = max(1, min(args.steps_in_flight, 2))
+    if n_sets % 2:
+        in_flight = 1
+    lanes = [torch.cuda.Stream() for _ in range(in_flight)] if in_flight > 1 else None
+
     def run_step(i):
+        if lanes is not None:
+            with torch.cuda.stream(lanes[i % in_flight]):
+                if graphs is not None:
+                    graphs[i % n_sets].replay()
+                else:
+                    step(sets[i % n_sets])
+            return
         if graphs is not None:
             graphs[i % n_sets].replay()
         else:
             step(sets[i % n_sets])
 
+    def fork_lanes():
+        if lanes is not None:
+            for l_ in lanes:
+                l_.wait_stream(torch.cuda.current_stream())
+
+    def join_lanes():
+        if lanes is not None:
+            for l_ in lanes:
+                torch.cuda.current_stream().wait_stream(l_)
+
+    fork_lanes()
     for i in range(max(args.warmup, 3)):
         run_step(i)
+    join_lanes()
     torch.cuda.synchronize()
 
     # ---- timed region: exactly K steps, device-resident inputs
@@ -723,8 +752,10 @@ def run_ours(args, info):
     torch.cuda.synchronize()
     sampler.start()
     e0.record()
+    fork_lanes()
     for i in range(args.steps):
         run_step(i)
+    join_lanes()
     e1.record()
     torch.cuda.synchronize()
     clocks = sampler.stop()
@@ -922,6 +953,7 @@ def run_ours(args, info):
                        "step": "aifs_reorder + mask_remap + fwht_quant_i8 + w4a8 gemm"
                                + ("" if args.serial_step else " (index -> remap -> quantizer -> GEMM in line, the row "
                                   "gather as a parallel branch behind the index kernel)"),
+                       "steps_in_flight": in_flight,
                        "tokens_per_s": (T_VIS + T_TXT) * args.steps * info.world / t_max},
             "clocks": clocks,
             "e2e": {"value": e2e_ops / 1e12, "unit": UNIT, "h2d_bytes_per_step": case.T * case.K * 2,
@@ -972,6 +1004,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--buffer-sets", type=int, default=4)
     ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--steps-in-flight", type=int, default=2,
+                    help="independent steps issued concurrently (1: one stream; 2: alternate streams)")
     ap.add_argument("--serial-step", action="store_true",
                     help="issue the four kernels of a step in one line instead of two parallel branches")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -23,16 +23,37 @@ __device__ __forceinline__ uint32_t pack_sat_s8x4(int q0, int q1, int q2, int q3
 // Loads this lane's four chunks of the row (zeros past K) and, if ROT, transforms them:
 // butterflies in increasing stride order, one float32 rounding each, then x c_n = 1/sqrt(n).
 // Must be called by all 32 lanes (warp shuffles).
-template <int LOG_TPB, bool ROT>
-__device__ __forceinline__ void fwht_warp_tile(const uint16_t* __restrict__ xrow, int K, int blk_start, int j,
-                                               float c_n, float (&v)[4][8]) {
+// The loads alone: this lane's four 16-byte chunks of the tile (zeros past K), so that a caller can have the
+// loads of a second tile in flight while it transforms the first.
+template <int LOG_TPB>
+__device__ __forceinline__ void fwht_warp_load(const uint16_t* __restrict__ xrow, int K, int blk_start, int j,
+                                               uint4 (&raw)[4]) {
   constexpr int TPB = 1 << LOG_TPB;
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     const int off = blk_start + (i * TPB + j) * 8;
-    uint4 w = make_uint4(0u, 0u, 0u, 0u);
-    if (off < K) w = __ldg(reinterpret_cast<const uint4*>(xrow + off));
-    const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+    raw[i] = make_uint4(0u, 0u, 0u, 0u);
+    if (off < K) raw[i] = __ldg(reinterpret_cast<const uint4*>(xrow + off));
+  }
+}
+
+template <int LOG_TPB, bool ROT>
+__device__ __forceinline__ void fwht_warp_compute(const uint4 (&raw)[4], int j, float c_n, float (&v)[4][8]);
+
+template <int LOG_TPB, bool ROT>
+__device__ __forceinline__ void fwht_warp_tile(const uint16_t* __restrict__ xrow, int K, int blk_start, int j,
+                                               float c_n, float (&v)[4][8]) {
+  uint4 raw[4];
+  fwht_warp_load<LOG_TPB>(xrow, K, blk_start, j, raw);
+  fwht_warp_compute<LOG_TPB, ROT>(raw, j, c_n, v);
+}
+
+// bf16 -> float32 and, if ROT, the transform of one tile from its loaded chunks.
+template <int LOG_TPB, bool ROT>
+__device__ __forceinline__ void fwht_warp_compute(const uint4 (&raw)[4], int j, float c_n, float (&v)[4][8]) {
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const uint32_t ww[4] = {raw[i].x, raw[i].y, raw[i].z, raw[i].w};
 #pragma unroll
     for (int p = 0; p < 4; ++p) {
       v[i][2 * p] = __uint_as_float(ww[p] << 16);
@@ -41,45 +62,59 @@ __device__ __forceinline__ void fwht_warp_tile(const uint16_t* __restrict__ xrow
   }
 
   if (ROT) {
+    // The butterflies run on pairs of float32 values (add / fma .f32x2: two IEEE round-to-nearest results per
+    // instruction, bit-identical to the scalar ones).  A pair holds the same element r of two chunks that
+    // no stage but the last combines: (chunk 0, chunk 2) in pa, (chunk 1, chunk 3) in pb.
+    const float2 minus1 = make_float2(-1.0f, -1.0f);
+    float2 pa[8], pb[8];
+#pragma unroll
+    for (int r = 0; r < 8; ++r) {
+      pa[r] = make_float2(v[0][r], v[2][r]);
+      pb[r] = make_float2(v[1][r], v[3][r]);
+    }
     // strides 1, 2, 4: inside each 8-element chunk
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
+    for (int h = 1; h < 8; h <<= 1) {
 #pragma unroll
-      for (int h = 1; h < 8; h <<= 1) {
-#pragma unroll
-        for (int r = 0; r < 8; ++r) {
-          if ((r & h) == 0) {
-            const float a = v[i][r], b = v[i][r + h];
-            v[i][r] = __fadd_rn(a, b);
-            v[i][r + h] = __fsub_rn(a, b);
-          }
+      for (int r = 0; r < 8; ++r) {
+        if ((r & h) == 0) {
+          const float2 a0 = pa[r], b0 = pa[r + h], a1 = pb[r], b1 = pb[r + h];
+          pa[r] = __fadd2_rn(a0, b0);
+          pa[r + h] = __ffma2_rn(b0, minus1, a0);  // a - b, one rounding
+          pb[r] = __fadd2_rn(a1, b1);
+          pb[r + h] = __ffma2_rn(b1, minus1, a1);
         }
       }
     }
     // strides 8 * 2^b for b < log2(TPB): partner lane j ^ 2^b
 #pragma unroll
     for (int b = 0; b < LOG_TPB; ++b) {
-      const float sgn = ((j >> b) & 1) ? -1.0f : 1.0f;
+      const float sg = ((j >> b) & 1) ? -1.0f : 1.0f;
+      const float2 sgn = make_float2(sg, sg);
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-#pragma unroll
-        for (int r = 0; r < 8; ++r) {
-          const float p = __shfl_xor_sync(0xffffffffu, v[i][r], 1 << b);
-          // lower element: own + partner; upper element: partner - own (one rounding)
-          v[i][r] = __fmaf_rn(v[i][r], sgn, p);
-        }
+      for (int r = 0; r < 8; ++r) {
+        float2 qa, qb;
+        qa.x = __shfl_xor_sync(0xffffffffu, pa[r].x, 1 << b);
+        qa.y = __shfl_xor_sync(0xffffffffu, pa[r].y, 1 << b);
+        qb.x = __shfl_xor_sync(0xffffffffu, pb[r].x, 1 << b);
+        qb.y = __shfl_xor_sync(0xffffffffu, pb[r].y, 1 << b);
+        // lower element: own + partner; upper element: partner - own (one rounding)
+        pa[r] = __ffma2_rn(pa[r], sgn, qa);
+        pb[r] = __ffma2_rn(pb[r], sgn, qb);
       }
     }
     // strides 8 * TPB and 16 * TPB: across the four chunks of this lane
+    const float2 cn2 = make_float2(c_n, c_n);
 #pragma unroll
     for (int r = 0; r < 8; ++r) {
-      float a0 = v[0][r], a1 = v[1][r], a2 = v[2][r], a3 = v[3][r];
-      float b0 = __fadd_rn(a0, a1), b1 = __fsub_rn(a0, a1);
-      float b2 = __fadd_rn(a2, a3), b3 = __fsub_rn(a2, a3);
-      v[0][r] = __fmul_rn(__fadd_rn(b0, b2), c_n);
-      v[1][r] = __fmul_rn(__fadd_rn(b1, b3), c_n);
-      v[2][r] = __fmul_rn(__fsub_rn(b0, b2), c_n);
-      v[3][r] = __fmul_rn(__fsub_rn(b1, b3), c_n);
+      const float2 s02 = __fadd2_rn(pa[r], pb[r]);          // (c0 + c1, c2 + c3)
+      const float2 d02 = __ffma2_rn(pb[r], minus1, pa[r]);  // (c0 - c1, c2 - c3)
+      const float2 o02 = __fmul2_rn(make_float2(__fadd_rn(s02.x, s02.y), __fsub_rn(s02.x, s02.y)), cn2);
+      const float2 o13 = __fmul2_rn(make_float2(__fadd_rn(d02.x, d02.y), __fsub_rn(d02.x, d02.y)), cn2);
+      v[0][r] = o02.x;
+      v[2][r] = o02.y;
+      v[1][r] = o13.x;
+      v[3][r] = o13.y;
     }
   }
 }
@@ -87,8 +122,13 @@ __device__ __forceinline__ void fwht_warp_tile(const uint16_t* __restrict__ xrow
 // Eq. 2 with a reciprocal scale: round-to-nearest-even of v * inv, saturated to int8 (NaN -> 0).
 __device__ __forceinline__ uint2 quant_chunk_s8(const float (&v)[8], float inv) {
   int q[8];
+  const float2 inv2 = make_float2(inv, inv);
 #pragma unroll
-  for (int r = 0; r < 8; ++r) q[r] = __float2int_rn(__fmul_rn(v[r], inv));
+  for (int r = 0; r < 8; r += 2) {
+    const float2 y = __fmul2_rn(make_float2(v[r], v[r + 1]), inv2);  // two IEEE products per instruction
+    q[r] = __float2int_rn(y.x);
+    q[r + 1] = __float2int_rn(y.y);
+  }
   uint2 o;
   o.x = pack_sat_s8x4(q[0], q[1], q[2], q[3]);
   o.y = pack_sat_s8x4(q[4], q[5], q[6], q[7]);
