@@ -83,7 +83,7 @@ def rotate_dense(x, n: int) -> np.ndarray:
     return (blocks @ H).reshape(x.shape)
 
 
-def fwht_blocks(x, n: int, dtype=np.float32) -> np.ndarray:
+def fwht_blocks(x, n: int, dtype=np.float32, normalise: bool = True) -> np.ndarray:
     """Fast Walsh-Hadamard transform of every length-n block of the last axis.
 
     The fast form of App. A.3's Kronecker recursion: log2(n) butterfly stages
@@ -91,7 +91,9 @@ def fwht_blocks(x, n: int, dtype=np.float32) -> np.ndarray:
     (for i with bit h clear) by (v[i] + v[i+h], v[i] - v[i+h]); afterwards one
     multiplication by 1/sqrt(n) (Sec. 3.2: orthonormal H).  In float32 this is
     the canonical rounding order: every add/sub and the final multiply rounds
-    once, the normalisation constant is float32(1/sqrt(n))."""
+    once, the normalisation constant is float32(1/sqrt(n)).  normalise=False
+    stops after the butterflies (the full-width Kronecker rotation normalises
+    once at its very end)."""
     x = np.asarray(x)
     K = x.shape[-1]
     if n == 0:
@@ -107,8 +109,9 @@ def fwht_blocks(x, n: int, dtype=np.float32) -> np.ndarray:
         w[:, :, :, 0, :] = a + b
         w[:, :, :, 1, :] = a - b
         h *= 2
-    c = dtype(1.0) / np.sqrt(dtype(n)) if dtype == np.float64 else np.float32(1.0 / np.sqrt(np.float64(n)))
-    v = v * c
+    if normalise:
+        c = dtype(1.0) / np.sqrt(dtype(n)) if dtype == np.float64 else np.float32(1.0 / np.sqrt(np.float64(n)))
+        v = v * c
     return v.reshape(x.shape).astype(dtype)
 
 
@@ -382,6 +385,108 @@ def linear_wa_sym(x, seg_end, seg_mod, s_vis, s_txt, rot_block, qw, s_w, act_bit
     y32 = dequant(acc, s_rows, s_w, bias, np.float32)
     return {"rotated": r, "s_rows": s_rows, "qx": qx, "acc": acc, "y64": y64, "y32": y32,
             "y_bf16": bf16_rne(y32)}
+
+
+# ----------------------------------------------------------------------------- full-width rotation for K = m * 2^k
+def _gf27_tables():
+    """GF(27) = GF(3)[x] / (x^3 + 2x + 1): elements are base-3 digit triples c0 + 3 c1 + 9 c2."""
+    def mul(a, b):
+        pa = [a % 3, (a // 3) % 3, a // 9]
+        pb = [b % 3, (b // 3) % 3, b // 9]
+        prod = [0] * 5
+        for i in range(3):
+            for j in range(3):
+                prod[i + j] = (prod[i + j] + pa[i] * pb[j]) % 3
+        for d in (4, 3):                       # x^3 = -2x - 1 = x + 2 (mod 3)
+            c = prod[d]
+            prod[d] = 0
+            prod[d - 2] = (prod[d - 2] + c) % 3
+            prod[d - 3] = (prod[d - 3] + 2 * c) % 3
+        return prod[0] + 3 * prod[1] + 9 * prod[2]
+
+    def sub(a, b):
+        return sum((((a // 3 ** d) % 3 - (b // 3 ** d) % 3) % 3) * 3 ** d for d in range(3))
+
+    return mul, sub
+
+
+def _quadratic_character(q: int):
+    """chi(a) for the field of q elements (q an odd prime, or 27): +1 for non-zero squares, -1 for
+    non-squares, 0 for 0, together with the field's subtraction."""
+    if q == 27:
+        mul, sub = _gf27_tables()
+        squares = {mul(a, a) for a in range(1, 27)}
+        assert len(squares) == 13
+        chi = [0] + [1 if a in squares else -1 for a in range(1, 27)]
+        return chi, sub
+    assert q > 2 and all(q % d for d in range(2, int(q ** 0.5) + 1)), "q must be an odd prime (or 27)"
+    chi = [0] + [1 if pow(a, (q - 1) // 2, q) == 1 else -1 for a in range(1, q)]
+    return chi, lambda a, b: (a - b) % q
+
+
+def paley_hadamard(m: int) -> np.ndarray:
+    """A Hadamard matrix of order m (entries +-1, H H^T = m I) by Paley's constructions, for the
+    orders a full-width online rotation of K = m * 2^k needs when K is not a power of two (the paper
+    defines only H_{2^n}, App. A.3; the Kronecker form H_m (x) H_{2^k} is the usual completion):
+      type I,  m = q + 1 with q = 3 (mod 4):  H = I + S,  S = [[0, 1^T], [-1, Q]],  Q[a,b] = chi(a - b);
+      type II, m = 2 (q + 1) with q = 1 (mod 4):  H = [[C + I, C - I], [C - I, -C - I]],
+               C = [[0, 1^T], [1, Q]].
+    q is an odd prime or 27.  m = 28 (K = 14336 = 28 * 512) is type I over GF(27); m = 148
+    (K = 18944 = 148 * 128) is type II with q = 73."""
+    if m in (1, 2):
+        return hadamard_matrix(m)
+    for kind, q in ((1, m - 1), (2, m // 2 - 1)):
+        if kind == 2 and m % 2:
+            continue
+        is_field = q == 27 or (q > 2 and all(q % d for d in range(2, int(q ** 0.5) + 1)))
+        if not is_field or q % 4 != (3 if kind == 1 else 1):
+            continue
+        chi, sub = _quadratic_character(q)
+        Q = np.array([[chi[sub(a, b)] for b in range(q)] for a in range(q)], dtype=np.int64)
+        if kind == 1:
+            S = np.zeros((q + 1, q + 1), dtype=np.int64)
+            S[0, 1:] = 1
+            S[1:, 0] = -1
+            S[1:, 1:] = Q
+            return (np.eye(q + 1, dtype=np.int64) + S).astype(np.int64)
+        C = np.zeros((q + 1, q + 1), dtype=np.int64)
+        C[0, 1:] = 1
+        C[1:, 0] = 1
+        C[1:, 1:] = Q
+        I = np.eye(q + 1, dtype=np.int64)
+        return np.block([[C + I, C - I], [C - I, -C - I]]).astype(np.int64)
+    raise ValueError("no Paley construction for order %d" % m)
+
+
+def kron_rotate_dense(x, h_m, n2: int) -> np.ndarray:
+    """y = x (H_m (x) H_n2) / sqrt(K) in float64, K = m * n2, with the input channels of a row read as
+    an m x n2 array X (channel = i * n2 + j): Y = H_m^T X H_n2 / sqrt(K)."""
+    x = np.asarray(x, dtype=np.float64)
+    h_m = np.asarray(h_m, dtype=np.float64)
+    m = h_m.shape[0]
+    T, K = x.shape
+    assert K == m * n2
+    X = x.reshape(T, m, n2)
+    U = X @ hadamard_matrix(n2).astype(np.float64)
+    Y = np.einsum("ia,tij->taj", h_m, U)
+    return (Y / np.sqrt(np.float64(K))).reshape(T, K)
+
+
+def kron_rotate_f32(x, h_m, n2: int) -> np.ndarray:
+    """The same in float32 with a fixed order: the un-normalised butterflies of fwht_blocks on every
+    run of n2 channels, then for every output (a, j) the sum over i = 0, 1, ... of +-U[i, j] added
+    one at a time, then one multiply by float32(1 / sqrt(K))."""
+    x = np.asarray(x, dtype=np.float32)
+    h_m = np.asarray(h_m)
+    m = h_m.shape[0]
+    T, K = x.shape
+    assert K == m * n2
+    U = (fwht_blocks(x, n2, np.float32, normalise=False) if n2 > 1 else x).reshape(T, m, n2)
+    Y = np.zeros((T, m, n2), dtype=np.float32)
+    for i in range(m):
+        Y = (Y + h_m[i].astype(np.float32)[None, :, None] * U[:, i, None, :]).astype(np.float32)
+    c = np.float32(1.0 / np.sqrt(np.float64(K)))
+    return (Y * c).astype(np.float32).reshape(T, K)
 
 
 # ----------------------------------------------------------------------------- AIFS

@@ -688,3 +688,56 @@ def test_w8a8_and_w4a4_linears_order_their_errors():
     a = O.linear_wa_sym(x, seg_end, seg_mod, s_v, s_t, 0, *O.quantize_weight_int4(w))
     b = O.linear_w4a8_msq(x, seg_end, seg_mod, s_v, s_t, 0, *O.quantize_weight_int4(w))
     assert np.array_equal(a["acc"], b["acc"]) and np.array_equal(a["y_bf16"], b["y_bf16"])
+
+
+# ----------------------------------------------------------------------------- full-width rotation, K = m * 2^k
+@pytest.mark.parametrize("m", [4, 8, 12, 20, 28, 36, 44, 148])
+def test_paley_hadamard_gram_is_m_identity_in_integers(m):
+    H = O.paley_hadamard(m)
+    assert H.shape == (m, m) and set(np.unique(H).tolist()) == {-1, 1}
+    assert np.array_equal(H @ H.T, m * np.eye(m, dtype=np.int64))
+    assert np.array_equal(H.T @ H, m * np.eye(m, dtype=np.int64))
+
+
+def test_paley_hadamard_refuses_orders_it_cannot_build():
+    for m in (107, 428, 16 * 107):            # K = 13696 = 107 * 128: no order-m matrix from these constructions
+        with pytest.raises((ValueError, AssertionError)):
+            O.paley_hadamard(m)
+
+
+def test_gf27_is_a_field():
+    from oracle.mq_oracle import _gf27_tables
+    mul, sub = _gf27_tables()
+    for a in range(1, 27):
+        assert sorted(mul(a, b) for b in range(27)) == list(range(27))      # multiplication by a != 0 permutes the field
+        assert sub(a, a) == 0 and mul(a, 1) == a
+    assert all(mul(a, mul(b, c)) == mul(mul(a, b), c) for a in (2, 5, 11, 26) for b in (3, 7, 13) for c in (4, 9, 20))
+
+
+def test_kronecker_rotation_against_the_dense_kronecker_product():
+    rng = np.random.default_rng(31)
+    m, n2, T = 12, 8, 5
+    K = m * n2
+    Hm = O.paley_hadamard(m)
+    full = np.kron(Hm, O.hadamard_matrix(n2)).astype(np.float64)              # (A (x) B)[i n2 + j, a n2 + b] = A[i,a] B[j,b]
+    assert np.array_equal(full @ full.T, K * np.eye(K))
+    x = rng.standard_normal((T, K))
+    want = x @ full / np.sqrt(K)
+    got = O.kron_rotate_dense(x, Hm, n2)
+    assert np.max(np.abs(got - want)) <= 1e-12
+    # orthonormal: norms are kept and the product with an equally rotated weight is unchanged
+    assert np.allclose(np.linalg.norm(got, axis=1), np.linalg.norm(x, axis=1))
+    w = rng.standard_normal((7, K))
+    assert np.max(np.abs(got @ O.kron_rotate_dense(w, Hm, n2).T - x @ w.T)) <= 1e-10
+    # a transposed H_m or swapped factors would fail the dense comparison (H_12 here is not symmetric)
+    assert not np.array_equal(Hm, Hm.T)
+    # float32 twin: same values within float32 accuracy, exact on small integers
+    x32 = rng.standard_normal((T, K)).astype(np.float32)
+    y32 = O.kron_rotate_f32(x32, Hm, n2)
+    assert np.max(np.abs(y32 - O.kron_rotate_dense(x32, Hm, n2))) <= 1e-5 * np.abs(x32).max() * np.sqrt(K)
+    xi = rng.integers(-8, 9, (T, K)).astype(np.float32)
+    c = np.float32(1.0 / np.sqrt(np.float64(K)))
+    assert np.array_equal(O.kron_rotate_f32(xi, Hm, n2), ((xi.astype(np.float64) @ full).astype(np.float32) * c))
+    # m = 1 is the plain block transform
+    assert np.array_equal(O.kron_rotate_f32(x32[:, :8], np.array([[1]]), 8),
+                          (O.fwht_blocks(x32[:, :8], 8, np.float32, normalise=False) * np.float32(1.0 / np.sqrt(8.0))).astype(np.float32))
