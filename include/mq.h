@@ -212,6 +212,23 @@ int mq_fwht_quant_i8(const void* X, int32_t T, int32_t K, int64_t ldx, const mq_
                      float s_vis, float s_txt, int32_t rot_block, int8_t* Q, int64_t ldq,
                      float* rotated_out, void* stream);
 
+/*
+ * Full-width online rotation for K = m * 2^k, fused with the MSQ int8 quantizer.  App. A.3 defines H_{2^n} only;
+ * for a K that is not a power of two (14336 = 28 * 512, 18944 = 148 * 128) the rotation of Fig. 4(a) is completed
+ * in Kronecker form H_K = H_m (x) H_{K/m} with a Hadamard matrix of order m that the CALLER supplies:
+ *   h_neg   device uint8 [m, m], h_neg[i * m + a] = 1 where H_m[i, a] = -1, 0 where it is +1
+ *   r[t, a * n2 + j] = float32(1 / sqrt(K)) * sum_i H_m[i, a] * U[t, i, j],  n2 = K / m,
+ *       U = the un-normalised butterflies (strides 1, 2, ..., n2 / 2) of every run of n2 channels of row t,
+ *       the sum added one term at a time for i = 0, 1, ..., m - 1 in float32;
+ *   Q as in mq_fwht_quant_i8;  rotated_out optional float32 [T, K] dump of r.
+ * m <= 256, K / m a power of two in [32, 1024], 4 K + m^2 <= 200 KiB (the row is kept in shared memory);
+ * otherwise MQ_ERR_UNSUPPORTED / MQ_ERR_INVALID_ARG.  The codes feed mq_w4a8_msq_linear with
+ * MQ_FLAG_X_IS_INT8; the weight is rotated offline with the same matrix.  Cost: m additions per element.
+ */
+int mq_kron_quant_i8(const void* X, int32_t T, int32_t K, int64_t ldx, const mq_segments* seg, float s_vis,
+                     float s_txt, int32_t m, const uint8_t* h_neg, int8_t* Q, int64_t ldq, float* rotated_out,
+                     void* stream);
+
 /* mq_fwht_quant_i8 with b-bit codes (act_bits 8 or 4; one byte per code either way): for 4 bits the
  * codes clamp to [-8, 7] (Eq. 2 with b = 4).  No rotated dump. */
 int mq_fwht_quant_bits(const void* X, int32_t T, int32_t K, int64_t ldx, const mq_segments* seg,

@@ -77,6 +77,7 @@ def load(build_if_missing: bool = False):
         "mq_w8_layout_bytes": (sz, [i32, i32]),
         "mq_pack_w8": (C.c_int, [vp, i32, i32, i64, vp, i64, vp, vp, vp]),
         "mq_fwht_quant_bits": (C.c_int, [vp, i32, i32, i64, segp, f32, f32, i32, i32, vp, i64, vp]),
+        "mq_kron_quant_i8": (C.c_int, [vp, i32, i32, i64, segp, f32, f32, i32, vp, vp, i64, vp, vp]),
         "mq_repack_w4": (C.c_int, [vp, i32, i32, vp, vp]),
         "mq_unpack_w4": (C.c_int, [vp, vp, i32, i32, vp, i64, vp]),
         "mq_aifs_reorder": (C.c_int, [vp, vp, i32, i32, i64, i64, vp, vp, vp, vp, vp, i32, vp]),
@@ -113,7 +114,7 @@ EXPORTED = ["mq_version", "mq_status_string", "mq_workspace_bytes", "mq_w4_layou
             "mq_reset_device_status", "mq_rms_side_ld", "mq_rms_detect", "mq_pack_w4_rms", "mq_rms_workspace_bytes",
             "mq_w4a8_msq_linear_rms", "mq_dynamic_quant_i8", "mq_dynamic_workspace_bytes", "mq_w4a8_dynamic_linear",
             "mq_ubench_mma_i8", "mq_selftest_bounded_wait", "mq_ubench_expand", "mq_calibrate_static_scales_bits",
-            "mq_w8_layout_bytes", "mq_pack_w8", "mq_fwht_quant_bits"]
+            "mq_w8_layout_bytes", "mq_pack_w8", "mq_fwht_quant_bits", "mq_kron_quant_i8"]
 
 
 def status_string(status: int) -> str:
@@ -219,6 +220,15 @@ def mq_fwht_quant_bits(x, seg: Segments, s_vis, s_txt, rot_block, act_bits, q_ou
     T, K = x.shape
     _check(load().mq_fwht_quant_bits(_ptr(x), T, K, _ld(x), seg.ref(), float(s_vis), float(s_txt), rot_block,
                                      act_bits, _ptr(q_out), _ld(q_out), _stream()), "mq_fwht_quant_bits")
+
+
+def mq_kron_quant_i8(x, seg: Segments, s_vis, s_txt, h_neg, q_out, rotated_out=None):
+    """Full-width rotation H_m (x) H_(K/m) + MSQ quantizer; h_neg: uint8 [m, m], 1 where H_m is -1."""
+    assert x.dtype == torch.bfloat16 and q_out.dtype == torch.int8 and h_neg.dtype == torch.uint8
+    T, K = x.shape
+    m = h_neg.shape[0]
+    _check(load().mq_kron_quant_i8(_ptr(x), T, K, _ld(x), seg.ref(), float(s_vis), float(s_txt), m, _ptr(h_neg),
+                                   _ptr(q_out), _ld(q_out), _ptr(rotated_out), _stream()), "mq_kron_quant_i8")
 
 
 def mq_repack_w4(packed, N, K, gemm_layout):

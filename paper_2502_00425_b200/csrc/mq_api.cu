@@ -207,6 +207,25 @@ int mq_fwht_quant_i8(const void* X, int32_t T, int32_t K, int64_t ldx, const mq_
                            static_cast<cudaStream_t>(stream));
 }
 
+int mq_kron_quant_i8(const void* X, int32_t T, int32_t K, int64_t ldx, const mq_segments* seg, float s_vis, float s_txt,
+                     int32_t m, const uint8_t* h_neg, int8_t* Q, int64_t ldq, float* rotated_out, void* stream) {
+  if (T < 0 || K <= 0 || m < 1 || m > 256 || K % m) return MQ_ERR_INVALID_ARG;
+  const int n2 = K / m;
+  if (n2 & (n2 - 1)) return MQ_ERR_INVALID_ARG;               // K / m must be a power of two
+  if (n2 < 32 || n2 > 1024) return MQ_ERR_UNSUPPORTED;
+  if ((size_t)K * sizeof(float) + (size_t)m * m > 200 * 1024) return MQ_ERR_UNSUPPORTED;  // the row lives in shared memory
+  if (T > 0 && (!X || !Q || !h_neg)) return MQ_ERR_INVALID_ARG;
+  if (ldx < K || ldq < K) return MQ_ERR_INVALID_ARG;
+  if (!good_scale(s_vis) || !good_scale(s_txt)) return MQ_ERR_INVALID_ARG;
+  if (!aligned16(X) || !aligned16(Q) || (ldx * 2) % 16 || ldq % 16) return MQ_ERR_ALIGNMENT;
+  if (rotated_out && !aligned16(rotated_out)) return MQ_ERR_ALIGNMENT;
+  SegTable st;
+  const int rc = check_seg(seg, &st);
+  if (rc != MQ_OK) return rc;
+  return launch_kron_quant(X, T, K, ldx, st, s_vis, s_txt, m, h_neg, Q, ldq, rotated_out,
+                           static_cast<cudaStream_t>(stream));
+}
+
 int mq_fwht_quant_bits(const void* X, int32_t T, int32_t K, int64_t ldx, const mq_segments* seg, float s_vis,
                        float s_txt, int32_t rot_block, int32_t act_bits, int8_t* Q, int64_t ldq, void* stream) {
   if (act_bits != 4 && act_bits != 8) return MQ_ERR_UNSUPPORTED;

@@ -119,6 +119,8 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
 int launch_fwht_quant(const void* X, int T, int K, int64_t ldx, SegTable seg, float s_vis,
                       float s_txt, int rot_block, int8_t* Q, int64_t ldq, float* rotated_out,
                       cudaStream_t st, int8_t* side_out = nullptr, int side_ld = 0, int act_bits = 8);
+int launch_kron_quant(const void* X, int T, int K, int64_t ldx, SegTable seg, float s_vis, float s_txt, int m,
+                      const uint8_t* h_neg, int8_t* Q, int64_t ldq, float* rotated_out, cudaStream_t st);
 int launch_dyn_quant(const void* X, int T, int K, int64_t ldx, int rot_block, int8_t* Q, int64_t ldq, float* s_rows,
                      cudaStream_t st);
 int launch_calibrate(const void* X, int T, int K, int64_t ldx, SegTable seg, int rot_block,

@@ -121,6 +121,12 @@ def test_other_entry_points_validate(lib):
     qb = lib.mq_fwht_quant_bits
     assert qb(A, 4, 128, 128, C.byref(seg), 1.0, 1.0, 0, 5, A, 128, None) == B.MQ_ERR_UNSUPPORTED
     assert qb(A, 4, 128, 128, C.byref(seg), 1.0, 0.0, 0, 4, A, 128, None) == B.MQ_ERR_INVALID_ARG
+    kq = lib.mq_kron_quant_i8
+    assert kq(A, 4, 14336, 14336, C.byref(seg), 1.0, 1.0, 24, A, A, 14336, None, None) == B.MQ_ERR_INVALID_ARG      # 24 does not divide K
+    assert kq(A, 4, 96, 96, C.byref(seg), 1.0, 1.0, 1, A, A, 96, None, None) == B.MQ_ERR_INVALID_ARG               # K / m = 96 is not a power of two
+    assert kq(A, 4, 448, 448, C.byref(seg), 1.0, 1.0, 28, A, A, 448, None, None) == B.MQ_ERR_UNSUPPORTED       # K / m = 16 is below 32
+    assert kq(A, 4, 3584, 3584, C.byref(seg), 1.0, 1.0, 28, None, A, 3584, None, None) == B.MQ_ERR_INVALID_ARG  # no sign table
+    assert kq(A, 4, 3584, 3584, C.byref(seg), 1.0, -1.0, 28, A, A, 3584, None, None) == B.MQ_ERR_INVALID_ARG
     cb = lib.mq_calibrate_static_scales_bits
     assert cb(A, 4, 128, 128, C.byref(seg), 0, 3, 0, A, A, A, None) == B.MQ_ERR_UNSUPPORTED
     assert cb(A, 4, 128, 128, C.byref(seg), 0, 4, 0, None, A, A, None) == B.MQ_ERR_INVALID_ARG
