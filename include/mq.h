@@ -409,6 +409,29 @@ int mq_w4a8_dynamic_linear(const mq_linear_desc* d, const void* X, int64_t ldx, 
                            const float* s_w, const float* bias, void* Y, int64_t ldy, int32_t* acc_out,
                            float* s_rows_out, void* ws, size_t ws_bytes, void* stream);
 
+/* ---- Glue of a decoder block (layer mode) ------------------------------------------------------
+ *
+ * Single-pass bf16 kernels (float32 arithmetic) for what sits between the linears of a block, so that a
+ * sequence can flow through a whole layer on the library's own kernels: RMSNorm (App. A.14), the rotary
+ * embedding on the ORIGINAL token positions that AIFS carries along (App. A.2), SwiGLU in front of the
+ * down-projection (Fig. 4(a)) and the residual add.  Not part of the quantized path; attention itself is
+ * left to the caller (with AIFS it is the causal attention of the original order, Eq. 5).
+ * All tensors bf16 row-major with leading dimensions in elements; rows 16-byte aligned (rotary: 4-byte).
+ */
+/* Y[t,:] = X[t,:] / sqrt(mean(X[t,:]^2) + eps) * gain;  D a multiple of 8, at most 16384. */
+int mq_glue_rmsnorm(const void* X, int32_t T, int32_t D, int64_t ldx, const float* gain, float eps, void* Y,
+                    int64_t ldy, void* stream);
+/* Channel pairs (2i, 2i+1) of each of n_heads heads of width head_dim rotated by pos[t] * base^(-2i/head_dim);
+ * X [L, n_heads * head_dim]; Y may be X (in place). */
+int mq_glue_rope(const void* X, int32_t L, int32_t n_heads, int32_t head_dim, int64_t ldx, const int32_t* pos,
+                 float base, void* Y, int64_t ldy, void* stream);
+/* Y = G / (1 + exp(-G)) * U;  G, U, Y [T, M] (G and U may be column ranges of one wider array); M % 8 == 0. */
+int mq_glue_swiglu(const void* G, int64_t ldg, const void* U, int64_t ldu, int32_t T, int32_t M, void* Y,
+                   int64_t ldy, void* stream);
+/* Y = A + B, one rounding to bf16;  [T, D], D % 8 == 0. */
+int mq_glue_residual_add(const void* A, int64_t lda, const void* Bm, int64_t ldb, int32_t T, int32_t D, void* Y,
+                         int64_t ldy, void* stream);
+
 /* ---- Measurement and self-test aids (the paper has no counterpart) ------------------------- */
 
 /*

@@ -78,6 +78,10 @@ def load(build_if_missing: bool = False):
         "mq_pack_w8": (C.c_int, [vp, i32, i32, i64, vp, i64, vp, vp, vp]),
         "mq_fwht_quant_bits": (C.c_int, [vp, i32, i32, i64, segp, f32, f32, i32, i32, vp, i64, vp]),
         "mq_kron_quant_i8": (C.c_int, [vp, i32, i32, i64, segp, f32, f32, i32, vp, vp, i64, vp, vp]),
+        "mq_glue_rmsnorm": (C.c_int, [vp, i32, i32, i64, vp, f32, vp, i64, vp]),
+        "mq_glue_rope": (C.c_int, [vp, i32, i32, i32, i64, vp, f32, vp, i64, vp]),
+        "mq_glue_swiglu": (C.c_int, [vp, i64, vp, i64, i32, i32, vp, i64, vp]),
+        "mq_glue_residual_add": (C.c_int, [vp, i64, vp, i64, i32, i32, vp, i64, vp]),
         "mq_repack_w4": (C.c_int, [vp, i32, i32, vp, vp]),
         "mq_unpack_w4": (C.c_int, [vp, vp, i32, i32, vp, i64, vp]),
         "mq_aifs_reorder": (C.c_int, [vp, vp, i32, i32, i64, i64, vp, vp, vp, vp, vp, i32, vp]),
@@ -114,7 +118,8 @@ EXPORTED = ["mq_version", "mq_status_string", "mq_workspace_bytes", "mq_w4_layou
             "mq_reset_device_status", "mq_rms_side_ld", "mq_rms_detect", "mq_pack_w4_rms", "mq_rms_workspace_bytes",
             "mq_w4a8_msq_linear_rms", "mq_dynamic_quant_i8", "mq_dynamic_workspace_bytes", "mq_w4a8_dynamic_linear",
             "mq_ubench_mma_i8", "mq_selftest_bounded_wait", "mq_ubench_expand", "mq_calibrate_static_scales_bits",
-            "mq_w8_layout_bytes", "mq_pack_w8", "mq_fwht_quant_bits", "mq_kron_quant_i8"]
+            "mq_w8_layout_bytes", "mq_pack_w8", "mq_fwht_quant_bits", "mq_kron_quant_i8", "mq_glue_rmsnorm", "mq_glue_rope",
+            "mq_glue_swiglu", "mq_glue_residual_add"]
 
 
 def status_string(status: int) -> str:
@@ -409,6 +414,34 @@ def mq_selftest_bounded_wait(limit_ns, site, status, waited_ns_out):
     assert status.dtype == torch.int32 and waited_ns_out.dtype == torch.int64 and waited_ns_out.numel() >= 4
     _check(load().mq_selftest_bounded_wait(int(limit_ns), int(site), _ptr(status), _ptr(waited_ns_out), _stream()),
            "mq_selftest_bounded_wait")
+
+
+def mq_glue_rmsnorm(x, gain, y, eps=1e-6):
+    assert x.dtype == torch.bfloat16 and y.dtype == torch.bfloat16 and gain.dtype == torch.float32
+    T, D = x.shape
+    _check(load().mq_glue_rmsnorm(_ptr(x), T, D, _ld(x), _ptr(gain), float(eps), _ptr(y), _ld(y), _stream()),
+           "mq_glue_rmsnorm")
+
+
+def mq_glue_rope(x, pos, n_heads, y, base=10000.0):
+    assert x.dtype == torch.bfloat16 and y.dtype == torch.bfloat16 and pos.dtype == torch.int32
+    L, width = x.shape
+    _check(load().mq_glue_rope(_ptr(x), L, n_heads, width // n_heads, _ld(x), _ptr(pos), float(base), _ptr(y), _ld(y),
+                               _stream()), "mq_glue_rope")
+
+
+def mq_glue_swiglu(gate, up, y):
+    assert gate.dtype == torch.bfloat16 and up.dtype == torch.bfloat16 and y.dtype == torch.bfloat16
+    T, M = gate.shape
+    _check(load().mq_glue_swiglu(_ptr(gate), _ld(gate), _ptr(up), _ld(up), T, M, _ptr(y), _ld(y), _stream()),
+           "mq_glue_swiglu")
+
+
+def mq_glue_residual_add(a, b, y):
+    assert a.dtype == torch.bfloat16 and b.dtype == torch.bfloat16 and y.dtype == torch.bfloat16
+    T, D = a.shape
+    _check(load().mq_glue_residual_add(_ptr(a), _ld(a), _ptr(b), _ld(b), T, D, _ptr(y), _ld(y), _stream()),
+           "mq_glue_residual_add")
 
 
 def mq_last_device_status(ws):

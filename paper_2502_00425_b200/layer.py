@@ -110,6 +110,9 @@ class W4A8DecoderBlock:
         self._fused: Dict[str, Optional[LinearWeights]] = {}
         # True: q/k/v and gate/up each run as one linear over the stacked weight (same results)
         self.fuse_groups = False
+        # True: RMSNorm, rotary embedding, SwiGLU and the residual adds run as the library's single-pass
+        # kernels (mq_glue_*); False: the plain torch expressions above (float32 temporaries in HBM)
+        self.cuda_glue = True
         # True: attention in the original order with a plain causal mask instead of the dense unified
         # mask (same result, much faster glue); the dense mask is still produced and kept in the trace
         self.causal_glue = False
@@ -247,11 +250,11 @@ class W4A8DecoderBlock:
         t, bd = tr.tensors, tr.bounds
         n_seq = len(embs)
         t["emb_u"] = x0
-        h = rmsnorm(x0, self.g_attn)
+        h = self._rmsnorm(x0, self.g_attn)
         t["attn_norm"] = h
         q, k, v = self.linear_group(["q_proj", "k_proj", "v_proj"], h, tr, calibrate)
-        qr = torch.cat([rope(q[bd[b]:bd[b + 1]], tr.pos_us[b], sh.n_q_heads) for b in range(n_seq)])
-        kr = torch.cat([rope(k[bd[b]:bd[b + 1]], tr.pos_us[b], sh.n_kv_heads) for b in range(n_seq)])
+        qr = self._rope(q, tr, sh.n_q_heads)
+        kr = self._rope(k, tr, sh.n_kv_heads)
         t["q_rope"], t["k_rope"] = qr, kr
         if self.causal_glue:
             a = torch.cat([gqa_attention_unpermuted(qr[bd[b]:bd[b + 1]], kr[bd[b]:bd[b + 1]], v[bd[b]:bd[b + 1]],
@@ -261,15 +264,19 @@ class W4A8DecoderBlock:
                                          sh.n_q_heads, sh.n_kv_heads) for b in range(n_seq)])
         t["attn"] = a
         o = self.linear("o_proj", a, tr, calibrate)
-        x1 = (x0.float() + o.float()).to(torch.bfloat16)
+        x1 = self._add(x0, o)
         t["resid1"] = x1
-        h2 = rmsnorm(x1, self.g_mlp)
+        h2 = self._rmsnorm(x1, self.g_mlp)
         t["mlp_norm"] = h2
         gate, up = self.linear_group(["gate_proj", "up_proj"], h2, tr, calibrate)
-        act = (torch.nn.functional.silu(gate.float()) * up.float()).to(torch.bfloat16)
+        if self.cuda_glue:
+            act = torch.empty((gate.shape[0], gate.shape[1]), dtype=torch.bfloat16, device=gate.device)
+            B.mq_glue_swiglu(gate, up, act)
+        else:
+            act = (torch.nn.functional.silu(gate.float()) * up.float()).to(torch.bfloat16)
         t["act"] = act
         down = self.linear("down_proj", act, tr, calibrate)
-        x2 = (x1.float() + down.float()).to(torch.bfloat16)
+        x2 = self._add(x1, down)
         t["resid2"] = x2
         outs = []
         for b in range(n_seq):
@@ -277,6 +284,30 @@ class W4A8DecoderBlock:
             B.mq_aifs_reorder(x2[bd[b]:bd[b + 1]], out, None, None, tr.perms[b], None, None, direction=1)
             outs.append(out)
         return outs, tr
+
+    # ---- glue: the library's single-pass kernels, or the torch expressions -------------------------
+    def _rmsnorm(self, x, gain):
+        if not self.cuda_glue:
+            return rmsnorm(x, gain)
+        y = torch.empty_like(x)
+        B.mq_glue_rmsnorm(x, gain, y)
+        return y
+
+    def _rope(self, x, tr: BlockTrace, n_heads: int):
+        bd = tr.bounds
+        if not self.cuda_glue:
+            return torch.cat([rope(x[bd[b]:bd[b + 1]], tr.pos_us[b], n_heads) for b in range(len(bd) - 1)])
+        y = torch.empty((x.shape[0], x.shape[1]), dtype=torch.bfloat16, device=x.device)
+        for b in range(len(bd) - 1):
+            B.mq_glue_rope(x[bd[b]:bd[b + 1]], tr.pos_us[b], n_heads, y[bd[b]:bd[b + 1]])
+        return y
+
+    def _add(self, a, b):
+        if not self.cuda_glue:
+            return (a.float() + b.float()).to(torch.bfloat16)
+        y = torch.empty_like(a)
+        B.mq_glue_residual_add(a, b, y)
+        return y
 
     def device_status_ok(self) -> bool:
         return all(B.mq_last_device_status(ws)[0] == B.MQ_OK for ws in self._ws.values())
