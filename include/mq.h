@@ -440,14 +440,15 @@ int mq_glue_residual_add(const void* A, int64_t lda, const void* Bm, int64_t ldb
  * denominator "what the tensor pipe can do on this machine at the clock it holds" next to the
  * nominal and the bf16-derived figures.  `ctas` CTAs (one per SM up to the SM count) each issue
  * n_mma MMAs rotating over n_acc accumulators of n_tok columns (n_acc * n_tok <= 480); A comes
- * from tensor memory (a_from_smem = 0, as in the GEMM) or from shared memory (1).
+ * from tensor memory (a_from_smem = 0, as in the GEMM) or from shared memory (1).  commit_every > 0 adds a
+ * tcgen05.commit to an mbarrier after every commit_every MMAs (the GEMM commits once per K block of four).
  *   cycles_out  device uint64 [ctas]: SM clock cycles from the first issue to the completion of
  *               the last MMA (0 if the bounded wait gave up)
  *   status      device int32 [2], zeroed by the caller: MQ_ERR_TIMEOUT + site if a wait gave up
  * int8 operations per clock and SM = 2 * 128 * n_tok * 32 * n_mma / cycles.
  */
-int mq_ubench_mma_i8(int32_t n_tok, int32_t n_mma, int32_t n_acc, int32_t a_from_smem, int32_t ctas,
-                     uint64_t* cycles_out, int32_t* status, void* stream);
+int mq_ubench_mma_i8(int32_t n_tok, int32_t n_mma, int32_t n_acc, int32_t a_from_smem, int32_t commit_every,
+                     int32_t ctas, uint64_t* cycles_out, int32_t* status, void* stream);
 
 /*
  * Cost of the weight expander's inner step (packed int4 tile in shared memory -> sixteen-fold int8

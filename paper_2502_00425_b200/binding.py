@@ -98,7 +98,7 @@ def load(build_if_missing: bool = False):
         "mq_dynamic_quant_i8": (C.c_int, [vp, i32, i32, i64, i32, vp, i64, vp, vp]),
         "mq_dynamic_workspace_bytes": (sz, [descp]),
         "mq_w4a8_dynamic_linear": (C.c_int, [descp, vp, i64, vp, vp, vp, vp, i64, vp, vp, vp, sz, vp]),
-        "mq_ubench_mma_i8": (C.c_int, [i32, i32, i32, i32, i32, vp, vp, vp]),
+        "mq_ubench_mma_i8": (C.c_int, [i32, i32, i32, i32, i32, i32, vp, vp, vp]),
         "mq_selftest_bounded_wait": (C.c_int, [C.c_uint64, i32, vp, vp, vp]),
         "mq_ubench_expand": (C.c_int, [i32, i32, i32, vp, vp]),
         "mq_last_device_status": (C.c_int, [vp, vp, C.POINTER(C.c_int32)]),
@@ -396,10 +396,10 @@ def mq_w4a8_dynamic_linear(x, w_layout, s_w, y, ws, N, rot_block=0, bias=None, a
            "mq_w4a8_dynamic_linear")
 
 
-def mq_ubench_mma_i8(n_tok, n_mma, n_acc, a_from_smem, ctas, cycles_out, status):
+def mq_ubench_mma_i8(n_tok, n_mma, n_acc, a_from_smem, ctas, cycles_out, status, commit_every=0):
     """Issue-rate microbenchmark of tcgen05.mma kind::i8; cycles_out int64 [ctas], status int32 [2] (zeroed)."""
     assert cycles_out.dtype == torch.int64 and cycles_out.numel() >= ctas and status.dtype == torch.int32
-    _check(load().mq_ubench_mma_i8(n_tok, n_mma, n_acc, int(a_from_smem), ctas, _ptr(cycles_out), _ptr(status),
+    _check(load().mq_ubench_mma_i8(n_tok, n_mma, n_acc, int(a_from_smem), int(commit_every), ctas, _ptr(cycles_out), _ptr(status),
                                    _stream()), "mq_ubench_mma_i8")
 
 

@@ -16,6 +16,7 @@ namespace {
 
 struct ProbeShared {
   uint64_t done;
+  uint64_t tick;  // receives the intermediate commits of the microbenchmark (nobody waits on it)
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -25,8 +26,8 @@ struct ProbeShared {
 // zero-filled operands (the tensor pipe does not look at values).  cycles_out[block] = clock64 ticks
 // from the first issue to the arrival of the commit that follows the last MMA.
 __global__ void __launch_bounds__(128, 1)
-ubench_mma_i8_kernel(int n_tok, int n_mma, int n_acc, int a_from_smem, unsigned long long* cycles_out,
-                     int32_t* status) {
+ubench_mma_i8_kernel(int n_tok, int n_mma, int n_acc, int a_from_smem, int commit_every,
+                     unsigned long long* cycles_out, int32_t* status) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* b_smem = smem;                    // 256 rows x 128 B, K-major, 128-byte swizzle atoms
@@ -38,6 +39,7 @@ ubench_mma_i8_kernel(int n_tok, int n_mma, int n_acc, int a_from_smem, unsigned 
     reinterpret_cast<uint4*>(smem)[i] = make_uint4(0u, 0u, 0u, 0u);
   if (threadIdx.x == 0) {
     mbar_init(&sh->done, 1);
+    mbar_init(&sh->tick, 1);
     sh->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -74,7 +76,7 @@ ubench_mma_i8_kernel(int n_tok, int n_mma, int n_acc, int a_from_smem, unsigned 
     __syncwarp();
     t0 = clock64();
     if (leader) {
-      int acc = 0;
+      int acc = 0, since = 0;
       for (int i = 0; i < n_mma; ++i) {
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * n_tok);
         const int k4 = i & 3;
@@ -89,6 +91,11 @@ ubench_mma_i8_kernel(int n_tok, int n_mma, int n_acc, int a_from_smem, unsigned 
           mma_i8_ts(d_tmem, a_tmem + (uint32_t)(k4 * 8), bdesc + (uint64_t)(k4 * 2), idesc, 1u);
         }
         if (++acc == n_acc) acc = 0;
+        // the GEMM commits once per K block (four MMAs): what that costs the issuing thread
+        if (++since == commit_every) {  // (a counter: an integer modulo per MMA would cost more than the MMA)
+          since = 0;
+          if (i + 1 < n_mma) tc_commit(&sh->tick);
+        }
       }
       tc_commit(&sh->done);
     }
@@ -202,10 +209,10 @@ __global__ void selftest_bounded_wait_kernel(unsigned long long limit_ns, int si
 }  // namespace
 }  // namespace mq
 
-extern "C" int mq_ubench_mma_i8(int32_t n_tok, int32_t n_mma, int32_t n_acc, int32_t a_from_smem, int32_t ctas,
-                                uint64_t* cycles_out, int32_t* status, void* stream) {
+extern "C" int mq_ubench_mma_i8(int32_t n_tok, int32_t n_mma, int32_t n_acc, int32_t a_from_smem, int32_t commit_every,
+                                int32_t ctas, uint64_t* cycles_out, int32_t* status, void* stream) {
   using namespace mq;
-  if (n_tok < 16 || n_tok > 256 || n_tok % 16 || n_mma < 1 || n_mma > (1 << 20) || n_acc < 1 || ctas < 1 ||
+  if (n_tok < 16 || n_tok > 256 || n_tok % 16 || n_mma < 1 || n_mma > (1 << 20) || n_acc < 1 || commit_every < 0 || ctas < 1 ||
       ctas > 4096 || !cycles_out || !status)
     return MQ_ERR_INVALID_ARG;
   if (n_acc * n_tok > 480) return MQ_ERR_INVALID_ARG;  // accumulators share tensor memory with the A slot
@@ -213,7 +220,7 @@ extern "C" int mq_ubench_mma_i8(int32_t n_tok, int32_t n_mma, int32_t n_acc, int
   static PerDeviceTable<char> attr_set;
   if (!ensure_dynamic_smem(attr_set, ubench_mma_i8_kernel, (int)smem)) return MQ_ERR_CUDA;
   ubench_mma_i8_kernel<<<ctas, 128, smem, static_cast<cudaStream_t>(stream)>>>(
-      n_tok, n_mma, n_acc, a_from_smem, reinterpret_cast<unsigned long long*>(cycles_out), status);
+      n_tok, n_mma, n_acc, a_from_smem, commit_every, reinterpret_cast<unsigned long long*>(cycles_out), status);
   return cuda_status(cudaGetLastError());
 }
 
