@@ -414,8 +414,8 @@ int mq_w4a8_dynamic_linear(const mq_linear_desc* d, const void* X, int64_t ldx, 
  * Single-pass bf16 kernels (float32 arithmetic) for what sits between the linears of a block, so that a
  * sequence can flow through a whole layer on the library's own kernels: RMSNorm (App. A.14), the rotary
  * embedding on the ORIGINAL token positions that AIFS carries along (App. A.2), SwiGLU in front of the
- * down-projection (Fig. 4(a)) and the residual add.  Not part of the quantized path; attention itself is
- * left to the caller (with AIFS it is the causal attention of the original order, Eq. 5).
+ * down-projection (Fig. 4(a)) and the residual add.  Not part of the quantized path; attention under the
+ * unified mask is mq_aifs_attention below.
  * All tensors bf16 row-major with leading dimensions in elements; rows 16-byte aligned (rotary: 4-byte).
  */
 /* Y[t,:] = X[t,:] / sqrt(mean(X[t,:]^2) + eps) * gain;  D a multiple of 8, at most 16384. */
@@ -431,6 +431,29 @@ int mq_glue_swiglu(const void* G, int64_t ldg, const void* U, int64_t ldu, int32
 /* Y = A + B, one rounding to bf16;  [T, D], D % 8 == 0. */
 int mq_glue_residual_add(const void* A, int64_t lda, const void* Bm, int64_t ldb, int32_t T, int32_t D, void* Y,
                          int64_t ldy, void* stream);
+
+/* ---- Attention under the unified causal mask (Sec. 3.1, Eq. 4 - Eq. 5; App. A.4) --------------
+ *
+ * Grouped-query softmax attention of one sequence whose rows stand in AIFS order:
+ *   O[i, h] = sum_j P[i, j] V[j, g(h)],  P[i, :] = softmax over the allowed j of  Q[i, h] . K[j, g(h)] / sqrt(D),
+ * with g(h) = h / (n_q_heads / n_kv_heads).  Row i (original token perm[i]) may attend row j iff
+ * perm[j] <= perm[i] and row j is not padded; a padded row also attends itself (its output is defined and
+ * meant to be discarded).  With perm the AIFS permutation this is Eq. 5 for any interleaving of the
+ * modalities, and the result equals causal attention (Eq. 4) in the original order, row for row.
+ *
+ * Q [L, n_q_heads * D], K, V [L, n_kv_heads * D], O [L, n_q_heads * D]: device bf16, row-major, leading
+ * dimensions in elements, rows 16-byte aligned; Q and K already carry the rotary embedding.  perm: device
+ * int32 [L] (mq_aifs_reorder's output).  pad_u: device uint8 [L] in AIFS order (1 = padded row) or NULL.
+ * head_dim must be 128 (MQ_ERR_UNSUPPORTED otherwise).  float32 accumulation; the probabilities enter the
+ * second product rounded to bf16.  ws: device scratch of mq_aifs_attention_workspace_bytes() bytes, 16-byte
+ * aligned (it receives V transposed and the per-tile index bounds); status: device int32[2], zeroed by the
+ * caller, receives MQ_ERR_TIMEOUT and the wait site if a bounded wait inside the kernel expires.
+ * Enqueues two kernels on `stream`; nothing is allocated, retained or synchronised.
+ */
+size_t mq_aifs_attention_workspace_bytes(int32_t L, int32_t n_kv_heads, int32_t head_dim);
+int mq_aifs_attention(const void* Q, int64_t ldq, const void* K, int64_t ldk, const void* V, int64_t ldv,
+                      const int32_t* perm, const uint8_t* pad_u, int32_t L, int32_t n_q_heads, int32_t n_kv_heads,
+                      int32_t head_dim, void* O, int64_t ldo, void* ws, size_t ws_bytes, int32_t* status, void* stream);
 
 /* ---- Measurement and self-test aids (the paper has no counterpart) ------------------------- */
 

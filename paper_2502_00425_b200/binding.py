@@ -82,6 +82,8 @@ def load(build_if_missing: bool = False):
         "mq_glue_rope": (C.c_int, [vp, i32, i32, i32, i64, vp, f32, vp, i64, vp]),
         "mq_glue_swiglu": (C.c_int, [vp, i64, vp, i64, i32, i32, vp, i64, vp]),
         "mq_glue_residual_add": (C.c_int, [vp, i64, vp, i64, i32, i32, vp, i64, vp]),
+        "mq_aifs_attention_workspace_bytes": (sz, [i32, i32, i32]),
+        "mq_aifs_attention": (C.c_int, [vp, i64, vp, i64, vp, i64, vp, vp, i32, i32, i32, i32, vp, i64, vp, sz, vp, vp]),
         "mq_repack_w4": (C.c_int, [vp, i32, i32, vp, vp]),
         "mq_unpack_w4": (C.c_int, [vp, vp, i32, i32, vp, i64, vp]),
         "mq_aifs_reorder": (C.c_int, [vp, vp, i32, i32, i64, i64, vp, vp, vp, vp, vp, i32, vp]),
@@ -119,7 +121,7 @@ EXPORTED = ["mq_version", "mq_status_string", "mq_workspace_bytes", "mq_w4_layou
             "mq_w4a8_msq_linear_rms", "mq_dynamic_quant_i8", "mq_dynamic_workspace_bytes", "mq_w4a8_dynamic_linear",
             "mq_ubench_mma_i8", "mq_selftest_bounded_wait", "mq_ubench_expand", "mq_calibrate_static_scales_bits",
             "mq_w8_layout_bytes", "mq_pack_w8", "mq_fwht_quant_bits", "mq_kron_quant_i8", "mq_glue_rmsnorm", "mq_glue_rope",
-            "mq_glue_swiglu", "mq_glue_residual_add"]
+            "mq_glue_swiglu", "mq_glue_residual_add", "mq_aifs_attention_workspace_bytes", "mq_aifs_attention"]
 
 
 def status_string(status: int) -> str:
@@ -442,6 +444,24 @@ def mq_glue_residual_add(a, b, y):
     T, D = a.shape
     _check(load().mq_glue_residual_add(_ptr(a), _ld(a), _ptr(b), _ld(b), T, D, _ptr(y), _ld(y), _stream()),
            "mq_glue_residual_add")
+
+
+def mq_aifs_attention_workspace_bytes(L, n_kv_heads, head_dim=128) -> int:
+    return int(load().mq_aifs_attention_workspace_bytes(L, n_kv_heads, head_dim))
+
+
+def mq_aifs_attention(q, k, v, perm, pad_u, n_q_heads, n_kv_heads, o, ws, status):
+    """Attention under the unified mask (Eq. 5) of one sequence in AIFS order; see include/mq.h.
+    ws: uint8 tensor of mq_aifs_attention_workspace_bytes(); status: zeroed int32[2]."""
+    for t in (q, k, v, o):
+        assert t.dtype == torch.bfloat16
+    assert perm.dtype == torch.int32 and status.dtype == torch.int32 and status.numel() >= 2
+    assert pad_u is None or pad_u.dtype == torch.uint8
+    L = q.shape[0]
+    head_dim = q.shape[1] // n_q_heads
+    _check(load().mq_aifs_attention(_ptr(q), _ld(q), _ptr(k), _ld(k), _ptr(v), _ld(v), _ptr(perm), _ptr(pad_u), L,
+                                    n_q_heads, n_kv_heads, head_dim, _ptr(o), _ld(o), _ptr(ws), ws.numel(), _ptr(status),
+                                    _stream()), "mq_aifs_attention")
 
 
 def mq_last_device_status(ws):

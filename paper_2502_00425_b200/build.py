@@ -10,7 +10,7 @@ PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG_DIR)
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libmq.so")
-SOURCES = ["mq_api.cu", "mq_fwht_quant.cu", "mq_pack.cu", "mq_aifs.cu", "mq_gemm.cu", "mq_noalloc.cu", "mq_rms.cu", "mq_gemv.cu", "mq_dynquant.cu", "mq_probe.cu", "mq_kron.cu", "mq_glue.cu"]
+SOURCES = ["mq_api.cu", "mq_fwht_quant.cu", "mq_pack.cu", "mq_aifs.cu", "mq_gemm.cu", "mq_noalloc.cu", "mq_rms.cu", "mq_gemv.cu", "mq_dynquant.cu", "mq_probe.cu", "mq_kron.cu", "mq_glue.cu", "mq_attn.cu"]
 
 
 def _nvcc() -> str:

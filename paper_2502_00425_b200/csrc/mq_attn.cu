@@ -1,0 +1,523 @@
+// Attention under the unified causal mask of AIFS (Sec. 3.1, Eq. 4 - Eq. 5), written for sm_100a.
+//
+// After AIFS the rows of a sequence stand in the order [visual (and pad) block][text block]; row i is the
+// original token perm[i].  Row i may attend row j iff the original token of j does not come after that of
+// i, perm[j] <= perm[i], and j is not a padded token (App. A.4); a padded row keeps its own diagonal so that
+// its (discarded) softmax stays defined.  With that rule the output equals causal attention in the original
+// order, which is what makes the reordering free (Eq. 5; "numerically the same").
+//
+//   S = Q K^T / sqrt(D);  P = softmax over the allowed columns;  O = P V     per head, grouped-query heads
+//
+// One CTA per (128-row query tile, query head).  Both products run on the tensor cores (tcgen05.mma
+// kind::f16 on bf16 operands from shared memory, float32 accumulators in tensor memory):
+//   * Q, K tiles and V^T tiles arrive by TMA (128-byte swizzle).  V is transposed once per call by a small
+//     prep kernel so that the second product's B operand is K-major like every other operand here;
+//   * S = Q K^T (128 x 128) goes to one of two tensor-memory buffers; eight softmax warps (two per 32-lane
+//     quarter; each thread owns one query row and half of the columns) read it twice -- once for the row
+//     maximum, once to form P = exp2(...) -- apply the mask, write P as bf16 into shared memory in the
+//     swizzled K-major layout, and keep the running maximum and sum (online softmax);
+//   * O_tile = P V (128 x 128) goes to a third buffer; the softmax threads add it into float registers,
+//     scaled by the factor the running maximum moved by;
+//   * key tiles no row of the query tile may see are skipped, and tiles every row may see in full skip the
+//     mask: the prep kernel stores, per 128-row tile, the smallest and largest original index.
+// Every wait on an mbarrier is bounded (see mq_sm100.cuh); an expired wait raises the CTA's abort flag, all
+// roles leave their loops at the next tile, and the status word carries MQ_ERR_TIMEOUT and the site.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include <climits>
+
+#include "mq_common.cuh"
+#include "mq_device_table.h"
+#include "mq_sm100.cuh"
+
+namespace mq {
+namespace {
+
+constexpr int kD = 128;           // head dimension
+constexpr int kTile = 128;        // query rows per CTA, keys per step
+constexpr int kHalfBytes = 64 * kTile * 2;   // one 128-row x 64-element swizzled block
+constexpr int kTileBytes = 2 * kHalfBytes;   // a 128 x 128 bf16 operand tile
+constexpr int kThreads = 12 * 32;            // producer, MMA issuer, allocator, spare, 8 softmax warps
+constexpr int kSoftmaxThreads = 8 * 32;
+
+struct AttnBarriers {
+  uint64_t q_full;
+  uint64_t k_full[2], k_empty[2], v_full[2], v_empty[2];
+  uint64_t s_full[2], s_empty[2];
+  uint64_t p_full, pv_done, o_empty;
+  uint64_t drain;
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+struct AttnParams {
+  int L, n_tiles, n_q_heads, group;  // group = query heads per key/value head
+  const int32_t* perm;
+  const uint8_t* pad_u;
+  const int32_t* kmin;    // per key tile: smallest original index among its attendable (in range, not padded) rows
+  const int32_t* kmaxc;   // largest one if the tile is clean (all rows in range, none padded), else INT_MAX
+  const int32_t* qmin;    // per query tile: smallest / largest original index over its rows in range
+  const int32_t* qmax;
+  __nv_bfloat16* O;
+  int64_t ldo;
+  float scale_log2;       // log2(e) / sqrt(D)
+  int32_t* status;
+};
+
+// 0: no row of the query tile may attend any row of the key tile; 1: some may; 2: all may attend all.
+__device__ __forceinline__ int tile_class(const AttnParams& p, int qt, int kt) {
+  if (kt != qt && p.kmin[kt] > p.qmax[qt]) return 0;
+  return p.kmaxc[kt] <= p.qmin[qt] ? 2 : 1;
+}
+
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&v);
+}
+
+// ---------------------------------------------------------------------------------------- prep
+// V [L, n_kv_heads * D] -> Vt [n_kv_heads * D, Lp] (keys contiguous, zero beyond L), and the per-tile bounds
+// of the original indices.  Grid (key tiles, kv heads); the blocks of head 0 also write the bounds.
+__global__ void __launch_bounds__(256)
+attn_prep_kernel(const uint16_t* __restrict__ V, int64_t ldv, int L, int Lp, const int32_t* __restrict__ perm,
+                 const uint8_t* __restrict__ pad_u, uint16_t* __restrict__ Vt, int32_t* __restrict__ kmin,
+                 int32_t* __restrict__ kmaxc, int32_t* __restrict__ qmin, int32_t* __restrict__ qmax) {
+  __shared__ uint16_t tile[kTile][kD + 8];
+  __shared__ int red[4][4];
+  const int kt = blockIdx.x, g = blockIdx.y, j0 = kt * kTile;
+  for (int c = threadIdx.x; c < kTile * (kD / 8); c += 256) {
+    const int row = c / (kD / 8), piece = c % (kD / 8);
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (j0 + row < L) v = *reinterpret_cast<const uint4*>(V + (size_t)(j0 + row) * ldv + (size_t)g * kD + piece * 8);
+    *reinterpret_cast<uint4*>(&tile[row][piece * 8]) = v;
+  }
+  __syncthreads();
+  for (int c = threadIdx.x; c < kD * (kTile / 8); c += 256) {
+    const int d = c / (kTile / 8), piece = c % (kTile / 8);
+    uint32_t w[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e)
+      w[e] = (uint32_t)tile[piece * 8 + 2 * e][d] | ((uint32_t)tile[piece * 8 + 2 * e + 1][d] << 16);
+    *reinterpret_cast<uint4*>(Vt + ((size_t)g * kD + d) * Lp + j0 + piece * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+  }
+  if (g != 0) return;
+  int a_min = INT_MAX, a_max = -1, r_min = INT_MAX, r_max = -1, dirty = 0;
+  if (threadIdx.x < kTile) {
+    const int j = j0 + threadIdx.x;
+    if (j < L) {
+      const int pj = perm[j];
+      r_min = r_max = pj;
+      if (pad_u && pad_u[j]) dirty = 1;
+      else a_min = a_max = pj;
+    } else {
+      dirty = 1;
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    a_min = min(a_min, __shfl_xor_sync(0xffffffffu, a_min, o));
+    a_max = max(a_max, __shfl_xor_sync(0xffffffffu, a_max, o));
+    r_min = min(r_min, __shfl_xor_sync(0xffffffffu, r_min, o));
+    r_max = max(r_max, __shfl_xor_sync(0xffffffffu, r_max, o));
+    dirty |= __shfl_xor_sync(0xffffffffu, dirty, o);
+  }
+  const int warp = threadIdx.x >> 5;
+  if (warp < 4 && (threadIdx.x & 31) == 0) {
+    red[warp][0] = a_min; red[warp][1] = dirty ? INT_MAX : a_max; red[warp][2] = r_min; red[warp][3] = r_max;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    kmin[kt] = min(min(red[0][0], red[1][0]), min(red[2][0], red[3][0]));
+    kmaxc[kt] = max(max(red[0][1], red[1][1]), max(red[2][1], red[3][1]));
+    qmin[kt] = min(min(red[0][2], red[1][2]), min(red[2][2], red[3][2]));
+    qmax[kt] = max(max(red[0][3], red[1][3]), max(red[2][3], red[3][3]));
+  }
+}
+
+// ---------------------------------------------------------------------------------------- softmax pieces
+// Row maximum of this thread's 64 columns of S (raw, unscaled scores).
+template <bool MASKED>
+__device__ __forceinline__ float row_max_pass(uint32_t s_addr, const int32_t* kp, int perm_i, int self_col) {
+  float mx = -1.0e30f;
+#pragma unroll
+  for (int cb = 0; cb < 64; cb += 32) {
+    uint32_t v[32];
+    tmem_ld_x32(s_addr + (uint32_t)cb, v);
+    tmem_wait_ld();
+#pragma unroll
+    for (int e = 0; e < 32; ++e) {
+      const float s = __uint_as_float(v[e]);
+      if (!MASKED || kp[cb + e] <= perm_i || cb + e == self_col) mx = fmaxf(mx, s);
+    }
+  }
+  return mx;
+}
+
+// P = exp2(scale * (S - m)) for this thread's 64 columns, written as bf16 into its row of the swizzled P block;
+// returns the row sum of what was written.
+template <bool MASKED>
+__device__ __forceinline__ float prob_pass(uint32_t s_addr, const int32_t* kp, int perm_i, int self_col, float scale_log2,
+                                           float m, uint8_t* p_row, int row7) {
+  const float bias = -m * scale_log2;
+  float sum = 0.0f;
+#pragma unroll
+  for (int cb = 0; cb < 64; cb += 32) {
+    uint32_t v[32];
+    tmem_ld_x32(s_addr + (uint32_t)cb, v);
+    tmem_wait_ld();
+#pragma unroll
+    for (int c8 = 0; c8 < 4; ++c8) {
+      uint32_t pk[4];
+#pragma unroll
+      for (int e2 = 0; e2 < 4; ++e2) {
+        const int e = c8 * 8 + e2 * 2;
+        float p0 = fast_exp2(fmaf(__uint_as_float(v[e]), scale_log2, bias));
+        float p1 = fast_exp2(fmaf(__uint_as_float(v[e + 1]), scale_log2, bias));
+        if (MASKED) {
+          if (!(kp[cb + e] <= perm_i || cb + e == self_col)) p0 = 0.0f;
+          if (!(kp[cb + e + 1] <= perm_i || cb + e + 1 == self_col)) p1 = 0.0f;
+        }
+        sum += p0 + p1;
+        pk[e2] = pack_bf16x2(p0, p1);
+      }
+      const int chunk = (cb >> 3) + c8;  // 16-byte piece of the 128-byte row
+      *reinterpret_cast<uint4*>(p_row + ((chunk ^ row7) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+    }
+  }
+  return sum;
+}
+
+// ---------------------------------------------------------------------------------------- the kernel
+__global__ void __launch_bounds__(kThreads, 1)
+aifs_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
+                      const __grid_constant__ CUtensorMap tmap_vt, const AttnParams p) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* q_smem = smem;                       // 32 KB
+  uint8_t* k_smem = q_smem + kTileBytes;        // 2 x 32 KB
+  uint8_t* v_smem = k_smem + 2 * kTileBytes;    // 2 x 32 KB
+  uint8_t* p_smem = v_smem + 2 * kTileBytes;    // 32 KB
+  AttnBarriers* sh = reinterpret_cast<AttnBarriers*>(p_smem + kTileBytes);
+  float* xch = reinterpret_cast<float*>(sh + 1);              // [2 parities][2 halves][128] row maxima; reused for the sums
+  int32_t* kp_all = reinterpret_cast<int32_t*>(xch + 2 * 2 * kTile);  // [2 parities][128] keys' original indices
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // heavy query tiles (late rows see the most keys) first; the heads of one key/value group side by side
+  const int head = blockIdx.x % p.n_q_heads;
+  const int qt = p.n_tiles - 1 - blockIdx.x / p.n_q_heads;
+  const int g = head / p.group;
+  const int q0 = qt * kTile;
+
+  if (threadIdx.x == 0) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmap_q)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmap_k)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmap_vt)) : "memory");
+    mbar_init(&sh->q_full, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&sh->k_full[i], 1); mbar_init(&sh->k_empty[i], 1);
+      mbar_init(&sh->v_full[i], 1); mbar_init(&sh->v_empty[i], 1);
+      mbar_init(&sh->s_full[i], 1); mbar_init(&sh->s_empty[i], 8);
+    }
+    mbar_init(&sh->p_full, 8); mbar_init(&sh->pv_done, 1); mbar_init(&sh->o_empty, 8);
+    mbar_init(&sh->drain, 1);
+    sh->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 2) {
+    tmem_alloc(&sh->tmem_base, 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&sh->tmem_base);
+  // tensor-memory columns: S buffers at 0 and 128, the P V product at 256
+
+  if (warp == 0) {
+    // ---------------- TMA producer: Q once, then K and V^T tiles of every key tile that is not skipped
+    if (lane == 0) {
+      mbar_arrive_expect_tx(&sh->q_full, kTileBytes);
+      tma_load_2d(q_smem, &tmap_q, head * kD, q0, &sh->q_full);
+      tma_load_2d(q_smem + kHalfBytes, &tmap_q, head * kD + 64, q0, &sh->q_full);
+      int t = 0;
+      bool ok = true;
+      for (int kt = 0; kt < p.n_tiles && ok; ++kt) {
+        if (tile_class(p, qt, kt) == 0) continue;
+        const int s = t & 1;
+        const uint32_t ph = (uint32_t)(t >> 1) & 1u;
+        if (t >= 2 && !(ok = mbar_wait(&sh->k_empty[s], ph ^ 1u, &sh->abort_flag, p.status, 21))) break;
+        mbar_arrive_expect_tx(&sh->k_full[s], kTileBytes);
+        tma_load_2d(k_smem + s * kTileBytes, &tmap_k, g * kD, kt * kTile, &sh->k_full[s]);
+        tma_load_2d(k_smem + s * kTileBytes + kHalfBytes, &tmap_k, g * kD + 64, kt * kTile, &sh->k_full[s]);
+        if (t >= 2 && !(ok = mbar_wait(&sh->v_empty[s], ph ^ 1u, &sh->abort_flag, p.status, 22))) {
+          mbar_wait_drain(&sh->k_full[s], ph, 20000ull);
+          break;
+        }
+        mbar_arrive_expect_tx(&sh->v_full[s], kTileBytes);
+        tma_load_2d(v_smem + s * kTileBytes, &tmap_vt, kt * kTile, g * kD, &sh->v_full[s]);
+        tma_load_2d(v_smem + s * kTileBytes + kHalfBytes, &tmap_vt, kt * kTile + 64, g * kD, &sh->v_full[s]);
+        ++t;
+      }
+      if (!ok) {
+        // copies still landing in this CTA's shared memory get time to finish before it exits
+        mbar_wait_drain(&sh->q_full, 0, 20000ull);
+        for (int back = 1; back <= 2 && back <= t; ++back) {
+          const int u = t - back;
+          mbar_wait_drain(&sh->k_full[u & 1], (uint32_t)(u >> 1) & 1u, 20000ull);
+          mbar_wait_drain(&sh->v_full[u & 1], (uint32_t)(u >> 1) & 1u, 20000ull);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer: S_t = Q K_t^T is issued one tile ahead of O_{t-1} = P_{t-1} V_{t-1}, so
+    // that the tensor cores work on the next scores while the softmax warps are busy with the current ones
+    if (elect_one()) {
+      const uint32_t idesc = make_idesc_bf16(kTile);
+      const uint64_t qdesc = make_b_desc(smem_u32(q_smem));
+      const uint64_t pdesc = make_b_desc(smem_u32(p_smem));
+      bool ok = mbar_wait(&sh->q_full, 0, &sh->abort_flag, p.status, 23);
+      int t = 0;
+      auto issue_pv = [&](int u) -> bool {
+        if (!mbar_wait(&sh->v_full[u & 1], (uint32_t)(u >> 1) & 1u, &sh->abort_flag, p.status, 24)) return false;
+        if (!mbar_wait(&sh->p_full, (uint32_t)u & 1u, &sh->abort_flag, p.status, 25)) return false;
+        if (u >= 1 && !mbar_wait(&sh->o_empty, (uint32_t)(u - 1) & 1u, &sh->abort_flag, p.status, 26)) return false;
+        tc_fence_after();
+        const uint64_t vdesc = make_b_desc(smem_u32(v_smem + (u & 1) * kTileBytes));
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const uint64_t off = (uint64_t)((k >> 2) * (kHalfBytes >> 4) + (k & 3) * 2);
+          mma_bf16_ss(tmem_base + 256u, pdesc + off, vdesc + off, idesc, k ? 1u : 0u);
+        }
+        tc_commit(&sh->pv_done);
+        tc_commit(&sh->v_empty[u & 1]);
+        return true;
+      };
+      for (int kt = 0; kt < p.n_tiles && ok; ++kt) {
+        if (tile_class(p, qt, kt) == 0) continue;
+        const int s = t & 1;
+        const uint32_t ph = (uint32_t)(t >> 1) & 1u;
+        if (!(ok = mbar_wait(&sh->k_full[s], ph, &sh->abort_flag, p.status, 27))) break;
+        if (t >= 2 && !(ok = mbar_wait(&sh->s_empty[s], ph ^ 1u, &sh->abort_flag, p.status, 28))) break;
+        tc_fence_after();
+        const uint64_t kdesc = make_b_desc(smem_u32(k_smem + s * kTileBytes));
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const uint64_t off = (uint64_t)((k >> 2) * (kHalfBytes >> 4) + (k & 3) * 2);
+          mma_bf16_ss(tmem_base + (uint32_t)(s * kTile), qdesc + off, kdesc + off, idesc, k ? 1u : 0u);
+        }
+        tc_commit(&sh->s_full[s]);
+        tc_commit(&sh->k_empty[s]);
+        if (t >= 1 && !(ok = issue_pv(t - 1))) break;
+        ++t;
+      }
+      if (ok && t >= 1) ok = issue_pv(t - 1);
+      if (!ok) {  // let every MMA already issued finish before tensor memory is freed
+        tc_commit(&sh->drain);
+        mbar_wait_drain(&sh->drain, 0, 2000000ull);
+      }
+    }
+    __syncwarp();
+  } else if (warp >= 4) {
+    // ---------------- softmax warps: thread (row, half) owns query row q0 + row, key columns 64 half .. + 63
+    // of every S tile and head channels 64 half .. + 63 of O
+    const int quarter = warp & 3, half = (warp - 4) >> 2;
+    const int row = quarter * 32 + lane;
+    const int i = q0 + row;
+    const int tid = threadIdx.x - 4 * 32;
+    const int perm_i = i < p.L ? p.perm[i] : -1;
+    const bool pad_i = i < p.L && p.pad_u && p.pad_u[i];
+    const uint32_t lane_base = tmem_base + ((uint32_t)(quarter * 32) << 16);
+    uint8_t* p_row = p_smem + half * kHalfBytes + (row >> 3) * 1024 + (row & 7) * 128;
+    float acc[64];
+#pragma unroll
+    for (int e = 0; e < 64; ++e) acc[e] = 0.0f;
+    float m_run = -1.0e30f, l_run = 0.0f, alpha_pending = 1.0f;
+    int t = 0;
+    bool ok = true;
+    for (int kt = 0; kt < p.n_tiles; ++kt) {
+      const int cls = tile_class(p, qt, kt);
+      if (cls == 0) continue;
+      const int s = t & 1;
+      int32_t* kp = kp_all + s * kTile;
+      if (cls == 1 && tid < kTile) {
+        const int j = kt * kTile + tid;
+        kp[tid] = (j < p.L && !(p.pad_u && p.pad_u[j])) ? p.perm[j] : INT_MAX;
+      }
+      // one verdict for all softmax threads: nobody leaves the loop while others still wait at a barrier
+      if (named_bar_or(1, kSoftmaxThreads, !ok)) { ok = false; break; }
+      ok = warp_all(mbar_wait(&sh->s_full[s], (uint32_t)(t >> 1) & 1u, &sh->abort_flag, p.status, 29));  // (ok was true)
+      tc_fence_after();
+      const uint32_t s_addr = lane_base + (uint32_t)(s * kTile + half * 64);
+      // a padded row attends itself: the column of the diagonal inside this thread's 64, if it is there
+      const int self_col = (pad_i && kt == qt && (row >> 6) == half) ? (row & 63) : -1;
+      const int32_t* kph = kp + half * 64;
+      float mx = cls == 1 ? row_max_pass<true>(s_addr, kph, perm_i, self_col) : row_max_pass<false>(s_addr, kph, perm_i, self_col);
+      float* xm = xch + (s * 2) * kTile;
+      xm[half * kTile + row] = mx;
+      named_bar_sync(2, kSoftmaxThreads);
+      mx = fmaxf(mx, xm[(half ^ 1) * kTile + row]);
+      const float m_new = fmaxf(m_run, mx);
+      const float alpha = fast_exp2((m_run - m_new) * p.scale_log2);
+      m_run = m_new;
+      if (t >= 1) {
+        // fold the previous tile's P V into the running output (and free P and the product buffer)
+        ok = warp_all(mbar_wait(&sh->pv_done, (uint32_t)(t - 1) & 1u, &sh->abort_flag, p.status, 30)) && ok;
+        tc_fence_after();
+#pragma unroll
+        for (int cb = 0; cb < 64; cb += 32) {
+          uint32_t v[32];
+          tmem_ld_x32(lane_base + 256u + (uint32_t)(half * 64 + cb), v);
+          tmem_wait_ld();
+#pragma unroll
+          for (int e = 0; e < 32; ++e) acc[cb + e] = fmaf(acc[cb + e], alpha_pending, __uint_as_float(v[e]));
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sh->o_empty);
+      }
+      alpha_pending = alpha;
+      const float sum = cls == 1 ? prob_pass<true>(s_addr, kph, perm_i, self_col, p.scale_log2, m_run, p_row, row & 7)
+                                 : prob_pass<false>(s_addr, kph, perm_i, self_col, p.scale_log2, m_run, p_row, row & 7);
+      l_run = fmaf(l_run, alpha, sum);
+      tc_fence_before();
+      fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) {
+        mbar_arrive(&sh->s_empty[s]);
+        mbar_arrive(&sh->p_full);
+      }
+      ++t;
+    }
+    if (ok && t >= 1) {
+      ok = warp_all(mbar_wait(&sh->pv_done, (uint32_t)(t - 1) & 1u, &sh->abort_flag, p.status, 31));
+      tc_fence_after();
+      if (ok) {
+#pragma unroll
+        for (int cb = 0; cb < 64; cb += 32) {
+          uint32_t v[32];
+          tmem_ld_x32(lane_base + 256u + (uint32_t)(half * 64 + cb), v);
+          tmem_wait_ld();
+#pragma unroll
+          for (int e = 0; e < 32; ++e) acc[cb + e] = fmaf(acc[cb + e], alpha_pending, __uint_as_float(v[e]));
+        }
+      }
+    }
+    // the two halves of a row add their sums; then O = acc / l, rounded to bf16
+    const bool all_ok = !named_bar_or(1, kSoftmaxThreads, !ok);
+    xch[half * kTile + row] = l_run;
+    named_bar_sync(2, kSoftmaxThreads);
+    const float l_tot = l_run + xch[(half ^ 1) * kTile + row];
+    if (all_ok && i < p.L) {
+      const float inv = 1.0f / l_tot;
+      __nv_bfloat16* dst = p.O + (size_t)i * p.ldo + (size_t)head * kD + half * 64;
+#pragma unroll
+      for (int c8 = 0; c8 < 8; ++c8) {
+        uint32_t w[4];
+#pragma unroll
+        for (int e2 = 0; e2 < 4; ++e2) w[e2] = pack_bf16x2(acc[c8 * 8 + 2 * e2] * inv, acc[c8 * 8 + 2 * e2 + 1] * inv);
+        *reinterpret_cast<uint4*>(dst + c8 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 2) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+constexpr size_t kAttnSmem = 1024 + 6 * (size_t)kTileBytes + sizeof(AttnBarriers) + 2 * 2 * kTile * sizeof(float) +
+                             2 * kTile * sizeof(int32_t);
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn attn_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  return fn;
+}
+
+// bf16 matrix [rows, cols] with a row pitch in elements, read in boxes of 128 rows x 64 elements (128 bytes)
+bool encode_bf16_map(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int64_t pitch) {
+  EncodeTiledFn encode = attn_encode_fn();
+  if (!encode) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)pitch * 2};
+  const cuuint32_t box[2] = {64, (cuuint32_t)kTile};
+  const cuuint32_t estr[2] = {1, 1};
+  return encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+inline size_t round_up_256(size_t v) { return (v + 255) / 256 * 256; }
+inline bool al16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace
+}  // namespace mq
+
+using namespace mq;
+
+extern "C" size_t mq_aifs_attention_workspace_bytes(int32_t L, int32_t n_kv_heads, int32_t head_dim) {
+  if (L <= 0 || n_kv_heads <= 0 || head_dim != kD) return 0;
+  const size_t n_tiles = ((size_t)L + kTile - 1) / kTile;
+  return round_up_256((size_t)n_kv_heads * kD * n_tiles * kTile * 2) + round_up_256(4 * n_tiles * sizeof(int32_t));
+}
+
+extern "C" int mq_aifs_attention(const void* Q, int64_t ldq, const void* K, int64_t ldk, const void* V, int64_t ldv,
+                                 const int32_t* perm, const uint8_t* pad_u, int32_t L, int32_t n_q_heads,
+                                 int32_t n_kv_heads, int32_t head_dim, void* O, int64_t ldo, void* ws, size_t ws_bytes,
+                                 int32_t* status, void* stream) {
+  if (L < 0 || n_q_heads <= 0 || n_kv_heads <= 0 || n_q_heads % n_kv_heads) return MQ_ERR_INVALID_ARG;
+  if (head_dim != kD) return MQ_ERR_UNSUPPORTED;
+  if (ldq < (int64_t)n_q_heads * kD || ldo < (int64_t)n_q_heads * kD || ldk < (int64_t)n_kv_heads * kD ||
+      ldv < (int64_t)n_kv_heads * kD)
+    return MQ_ERR_INVALID_ARG;
+  if (L == 0) return MQ_OK;
+  if (!Q || !K || !V || !O || !perm || !ws || !status) return MQ_ERR_INVALID_ARG;
+  if (!al16(Q) || !al16(K) || !al16(V) || !al16(O) || !al16(ws) || (ldq * 2) % 16 || (ldk * 2) % 16 || (ldv * 2) % 16 ||
+      (ldo * 2) % 16)
+    return MQ_ERR_ALIGNMENT;
+  if (ws_bytes < mq_aifs_attention_workspace_bytes(L, n_kv_heads, head_dim)) return MQ_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int n_tiles = (L + kTile - 1) / kTile;
+  const int Lp = n_tiles * kTile;
+  uint16_t* Vt = static_cast<uint16_t*>(ws);
+  int32_t* bounds = reinterpret_cast<int32_t*>(static_cast<uint8_t*>(ws) + round_up_256((size_t)n_kv_heads * kD * Lp * 2));
+  attn_prep_kernel<<<dim3(n_tiles, n_kv_heads), 256, 0, st>>>(static_cast<const uint16_t*>(V), ldv, L, Lp, perm, pad_u, Vt,
+                                                              bounds, bounds + n_tiles, bounds + 2 * n_tiles,
+                                                              bounds + 3 * n_tiles);
+  if (cuda_status(cudaGetLastError()) != MQ_OK) return MQ_ERR_CUDA;
+
+  CUtensorMap mq_, mk, mv;
+  if (!encode_bf16_map(&mq_, Q, L, (int64_t)n_q_heads * kD, ldq) || !encode_bf16_map(&mk, K, L, (int64_t)n_kv_heads * kD, ldk) ||
+      !encode_bf16_map(&mv, Vt, (int64_t)n_kv_heads * kD, Lp, Lp))
+    return MQ_ERR_CUDA;
+  static PerDeviceTable<char> attr_set;
+  if (!ensure_dynamic_smem(attr_set, aifs_attention_kernel, (int)kAttnSmem)) return MQ_ERR_CUDA;
+  AttnParams p{};
+  p.L = L; p.n_tiles = n_tiles; p.n_q_heads = n_q_heads; p.group = n_q_heads / n_kv_heads;
+  p.perm = perm; p.pad_u = pad_u;
+  p.kmin = bounds; p.kmaxc = bounds + n_tiles; p.qmin = bounds + 2 * n_tiles; p.qmax = bounds + 3 * n_tiles;
+  p.O = static_cast<__nv_bfloat16*>(O); p.ldo = ldo;
+  p.scale_log2 = 1.4426950408889634f / sqrtf((float)kD);
+  p.status = status;
+  aifs_attention_kernel<<<dim3((unsigned)n_tiles * (unsigned)n_q_heads), kThreads, kAttnSmem, st>>>(mq_, mk, mv, p);
+  return cuda_status(cudaGetLastError());
+}
