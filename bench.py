@@ -442,14 +442,13 @@ def dynamic_linear_timing(torch, B, dev, T, K, N, rot, n_sets=4, reps=10):
 
 # ------------------------------------------------------------------------------------------ layer mode
 def layer_mode_timing(torch, dev, name, shape, seqs, reps=5):
-    """Configs 3 and 4 as a whole decoder block (layer mode): AIFS, mask / position remap and the
-    seven W4A8 MSQ linears through the C ABI, with the glue between them (RMSNorm, rotary
-    embedding, masked grouped-query attention, SwiGLU, residuals) in plain, untuned torch.  Random
-    valid weight bytes, fixed scales: timing only (parity of the block is covered by the tests).
-    Reports tokens per second for the whole block and how much of the time the glue takes."""
+    """Configs 3 and 4 as a whole decoder block (layer mode): AIFS, mask / position remap, the seven W4A8
+    MSQ linears, the glue kernels (RMSNorm, rotary embedding, SwiGLU, residuals) and attention under the
+    unified mask (mq_aifs_attention), all through the C ABI.  Random valid weight bytes, fixed scales: timing
+    only (parity of the block is covered by the tests).  Reports tokens per second for the whole block, and
+    for context the same block with attention handed to torch's fused causal kernel on un-permuted rows."""
     from paper_2502_00425_b200 import layer as LY
     blk = LY.random_block(shape, 21, dev)
-    blk.causal_glue = True  # attention in the original order with a plain causal mask (same result, Eq. 5)
     blk.fuse_groups = True  # q/k/v and gate/up as one stacked weight each: one launch per group (same results)
     for lw in blk.w.values():
         lw.s_vis, lw.s_txt = 0.5, 0.05
@@ -457,30 +456,78 @@ def layer_mode_timing(torch, dev, name, shape, seqs, reps=5):
     embs = [(torch.randn((len(s_), shape.hidden), generator=g) * 2).to(torch.bfloat16).to(dev) for s_ in seqs]
     vis = [torch.from_numpy(s_).to(dev) for s_ in seqs]
     tokens = sum(len(s_) for s_ in seqs)
-    blk.forward_batch(embs, vis)
-    torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    launch = "CUDA graph"
-    try:  # the block has ~60 small glue launches: replay it from a graph so that the GPU, not the host, is timed
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph):
-            blk.forward_batch(embs, vis)
-        graph.replay()
+
+    def timed():
+        blk.forward_batch(embs, vis)
         torch.cuda.synchronize()
-        run = graph.replay
-    except Exception:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        launch = "CUDA graph"
+        try:  # the block has dozens of small launches: replay it from a graph so that the GPU, not the host, is timed
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                blk.forward_batch(embs, vis)
+            graph.replay()
+            torch.cuda.synchronize()
+            run = graph.replay
+        except Exception:
+            torch.cuda.synchronize()
+            launch = "eager"
+            run = lambda: blk.forward_batch(embs, vis)
+        e0.record()
+        for _ in range(reps):
+            run()
+        e1.record()
         torch.cuda.synchronize()
-        launch = "eager"
-        run = lambda: blk.forward_batch(embs, vis)
-    e0.record()
-    for _ in range(reps):
-        run()
-    e1.record()
-    torch.cuda.synchronize()
-    sec = e0.elapsed_time(e1) * 1e-3 / reps
+        return e0.elapsed_time(e1) * 1e-3 / reps, launch
+
+    blk.cuda_attention = shape.head_dim == 128
+    sec, launch = timed()
+    own = blk.cuda_attention
+    blk.cuda_attention, blk.causal_glue = False, True  # (plain causal mask in the original order: same result, Eq. 5)
+    sec_torch, _ = timed()
     return {"workload": name, "tokens": tokens, "us_per_block": sec * 1e6, "tokens_per_s": tokens / sec,
-            "glue": "torch (untuned): RMSNorm, RoPE, causal GQA attention on the un-permuted rows, SwiGLU, residuals", "launch": launch,
+            "attention": "mq_aifs_attention (unified mask, AIFS order)" if own else "torch (head_dim != 128)",
+            "glue": "library kernels: RMSNorm, RoPE, SwiGLU, residuals", "launch": launch,
+            "with_torch_causal_attention": {"us_per_block": sec_torch * 1e6, "tokens_per_s": tokens / sec_torch},
             "status_ok": blk.device_status_ok()}
+
+
+def attention_timing(torch, B, dev, reps=10):
+    """mq_aifs_attention alone on the sequences of configs 3 and 4 (one sequence per call) and on a long text-only
+    sequence: microseconds and TFLOP/s over the multiply-adds the mask allows (4 * D * allowed pairs * heads)."""
+    from paper_2502_00425_b200 import synth as SY
+    out = {}
+    cases = [("config3 sequence: [img 1024][txt 96] x 3, 28 / 4 heads", SY.interleaved_modality([(1, 1024), (0, 96)] * 3), 28, 4),
+             ("config4 sequence: [txt 32][4 x 576 visual][txt 96], 32 / 8 heads", SY.interleaved_modality([(0, 32), (1, 2304), (0, 96)]), 32, 8),
+             ("text only, 8192 tokens, 32 / 8 heads", SY.interleaved_modality([(0, 8192)]), 32, 8)]
+    g = torch.Generator(device="cpu").manual_seed(31)
+    for name, is_visual, hq, hkv in cases:
+        L, D = int(is_visual.shape[0]), 128
+        q = torch.randn((L, hq * D), generator=g).to(torch.bfloat16).to(dev)
+        k = torch.randn((L, hkv * D), generator=g).to(torch.bfloat16).to(dev)
+        v = torch.randn((L, hkv * D), generator=g).to(torch.bfloat16).to(dev)
+        o = torch.empty_like(q)
+        ws = torch.empty(B.mq_aifs_attention_workspace_bytes(L, hkv), dtype=torch.uint8, device=dev)
+        status = torch.zeros(2, dtype=torch.int32, device=dev)
+        # the permutation comes from the library's own AIFS reorder (of a dummy embedding)
+        perm = torch.empty(L, dtype=torch.int32, device=dev)
+        dummy = torch.zeros((L, 64), dtype=torch.bfloat16, device=dev)
+        B.mq_aifs_reorder(dummy, torch.empty_like(dummy), torch.from_numpy(is_visual).to(dev), None, perm,
+                          torch.empty(L, dtype=torch.int32, device=dev), torch.zeros(1, dtype=torch.int32, device=dev), direction=0)
+        run = lambda: B.mq_aifs_attention(q, k, v, perm, None, hq, hkv, o, ws, status)
+        for _ in range(3):
+            run()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            run()
+        e1.record()
+        torch.cuda.synchronize()
+        us = e0.elapsed_time(e1) * 1e3 / reps
+        flops = 4.0 * D * hq * (L * (L + 1) / 2)
+        out[name] = {"L": L, "us": us, "tflops_allowed_pairs": flops / us / 1e6, "status_ok": status.tolist() == [0, 0]}
+    return out
 
 
 # ------------------------------------------------------------------------------------------ layer linear suites
@@ -870,7 +917,7 @@ def run_ours(args, info):
     e2e_ops, _ = D.aggregate_throughput(ops_per_step() * e2e_steps, e0.elapsed_time(e1) * 1e-3, dev)
 
     # ---- decode-shaped sweep (rank 0, N = 1 only): the HBM-bound regime of the same path
-    decode, suites, rms_timing, dyn_timing, layers, var_timing = None, None, None, None, None, None
+    decode, suites, rms_timing, dyn_timing, layers, var_timing, attn_timing = None, None, None, None, None, None, None
     n_sms = torch.cuda.get_device_properties(dev).multi_processor_count
     ubench = None
     if info.is_main:
@@ -896,6 +943,8 @@ def run_ours(args, info):
                                     synth.QWEN2_7B, [synth.config3_sequence()]),
                   layer_mode_timing(torch, dev, "config4: 8B-shaped block, 4 sequences of 2432 tokens",
                                     synth.LLAMA_8B, [synth.config4_sequence()] * 4)]
+        torch.cuda.empty_cache()
+        attn_timing = attention_timing(torch, B, dev)
 
     # ---- CPU baseline: the oracle on this host (rank 0, N = 1 only)
     cpu = None
@@ -989,6 +1038,7 @@ def run_ours(args, info):
             "static_vs_dynamic_a8": dyn_timing,
             "variants": var_timing,
             "layer_mode": layers,
+            "attention": attn_timing,
             "device_status": list(status),
             "cpu_baseline": cpu,
         }

@@ -13,11 +13,13 @@
 //   * Q, K tiles and V^T tiles arrive by TMA (128-byte swizzle).  V is transposed once per call by a small
 //     prep kernel so that the second product's B operand is K-major like every other operand here;
 //   * S = Q K^T (128 x 128) goes to one of two tensor-memory buffers; eight softmax warps (two per 32-lane
-//     quarter; each thread owns one query row and half of the columns) read it twice -- once for the row
-//     maximum, once to form P = exp2(...) -- apply the mask, write P as bf16 into shared memory in the
-//     swizzled K-major layout, and keep the running maximum and sum (online softmax);
-//   * O_tile = P V (128 x 128) goes to a third buffer; the softmax threads add it into float registers,
-//     scaled by the factor the running maximum moved by;
+//     quarter; each thread owns one query row and half of the columns) read it once into registers, apply
+//     the mask, form P = exp2(...) and write it as bf16 back into tensor memory, where the second product
+//     takes it as its A operand: the probabilities never touch shared memory;
+//   * O += P V accumulates in tensor memory across the key tiles.  The exponents are taken relative to a
+//     reference maximum that may lag the true running maximum by up to 8 powers of two; only when a row
+//     outgrows it are the accumulated output and sum rescaled (online softmax with a lazy rescale), so the
+//     softmax warps normally never touch O until the end;
 //   * key tiles no row of the query tile may see are skipped, and tiles every row may see in full skip the
 //     mask: the prep kernel stores, per 128-row tile, the smallest and largest original index.
 // Every wait on an mbarrier is bounded (see mq_sm100.cuh); an expired wait raises the CTA's abort flag, all
@@ -41,11 +43,13 @@ constexpr int kTileBytes = 2 * kHalfBytes;   // a 128 x 128 bf16 operand tile
 constexpr int kThreads = 12 * 32;            // producer, MMA issuer, allocator, spare, 8 softmax warps
 constexpr int kSoftmaxThreads = 8 * 32;
 
+constexpr int kStages = 2;                   // K tiles and V^T tiles in flight (each ring)
+
 struct AttnBarriers {
   uint64_t q_full;
-  uint64_t k_full[2], k_empty[2], v_full[2], v_empty[2];
-  uint64_t s_full[2], s_empty[2];
-  uint64_t p_full, pv_done, o_empty;
+  uint64_t k_full[kStages], k_empty[kStages], v_full[kStages], v_empty[kStages];
+  uint64_t s_full[2], s_empty[2];   // a score buffer is written (MMA commit) / has been read (eight softmax warps)
+  uint64_t p_full[2], pv_done[2];   // a P buffer is written (eight warps) / its product into O is complete (commit)
   uint64_t drain;
   uint32_t tmem_base;
   int abort_flag;
@@ -140,70 +144,23 @@ attn_prep_kernel(const uint16_t* __restrict__ V, int64_t ldv, int L, int Lp, con
   }
 }
 
-// ---------------------------------------------------------------------------------------- softmax pieces
-// Row maximum of this thread's 64 columns of S (raw, unscaled scores).
-template <bool MASKED>
-__device__ __forceinline__ float row_max_pass(uint32_t s_addr, const int32_t* kp, int perm_i, int self_col) {
-  float mx = -1.0e30f;
-#pragma unroll
-  for (int cb = 0; cb < 64; cb += 32) {
-    uint32_t v[32];
-    tmem_ld_x32(s_addr + (uint32_t)cb, v);
-    tmem_wait_ld();
-#pragma unroll
-    for (int e = 0; e < 32; ++e) {
-      const float s = __uint_as_float(v[e]);
-      if (!MASKED || kp[cb + e] <= perm_i || cb + e == self_col) mx = fmaxf(mx, s);
-    }
-  }
-  return mx;
-}
-
-// P = exp2(scale * (S - m)) for this thread's 64 columns, written as bf16 into its row of the swizzled P block;
-// returns the row sum of what was written.
-template <bool MASKED>
-__device__ __forceinline__ float prob_pass(uint32_t s_addr, const int32_t* kp, int perm_i, int self_col, float scale_log2,
-                                           float m, uint8_t* p_row, int row7) {
-  const float bias = -m * scale_log2;
-  float sum = 0.0f;
-#pragma unroll
-  for (int cb = 0; cb < 64; cb += 32) {
-    uint32_t v[32];
-    tmem_ld_x32(s_addr + (uint32_t)cb, v);
-    tmem_wait_ld();
-#pragma unroll
-    for (int c8 = 0; c8 < 4; ++c8) {
-      uint32_t pk[4];
-#pragma unroll
-      for (int e2 = 0; e2 < 4; ++e2) {
-        const int e = c8 * 8 + e2 * 2;
-        float p0 = fast_exp2(fmaf(__uint_as_float(v[e]), scale_log2, bias));
-        float p1 = fast_exp2(fmaf(__uint_as_float(v[e + 1]), scale_log2, bias));
-        if (MASKED) {
-          if (!(kp[cb + e] <= perm_i || cb + e == self_col)) p0 = 0.0f;
-          if (!(kp[cb + e + 1] <= perm_i || cb + e + 1 == self_col)) p1 = 0.0f;
-        }
-        sum += p0 + p1;
-        pk[e2] = pack_bf16x2(p0, p1);
-      }
-      const int chunk = (cb >> 3) + c8;  // 16-byte piece of the 128-byte row
-      *reinterpret_cast<uint4*>(p_row + ((chunk ^ row7) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-    }
-  }
-  return sum;
-}
-
 // ---------------------------------------------------------------------------------------- the kernel
+// Tensor-memory columns: S buffers at 0 and 128 (float32), the output accumulator O at 256 (float32), the
+// two P buffers at 384 and 448 (bf16 pairs: 64 columns hold 128 probabilities per row).
+constexpr uint32_t kColO = 256, kColP = 384;
+// The exponent's reference maximum may lag the true running maximum by this many powers of two before the
+// accumulated output is rescaled (probabilities then reach at most 2^8, harmless in float32 / bf16).
+constexpr float kLagLog2 = 8.0f;
+
 __global__ void __launch_bounds__(kThreads, 1)
 aifs_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                       const __grid_constant__ CUtensorMap tmap_vt, const AttnParams p) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* q_smem = smem;                       // 32 KB
-  uint8_t* k_smem = q_smem + kTileBytes;        // 2 x 32 KB
-  uint8_t* v_smem = k_smem + 2 * kTileBytes;    // 2 x 32 KB
-  uint8_t* p_smem = v_smem + 2 * kTileBytes;    // 32 KB
-  AttnBarriers* sh = reinterpret_cast<AttnBarriers*>(p_smem + kTileBytes);
+  uint8_t* k_smem = q_smem + kTileBytes;        // kStages x 32 KB
+  uint8_t* v_smem = k_smem + kStages * kTileBytes;
+  AttnBarriers* sh = reinterpret_cast<AttnBarriers*>(v_smem + kStages * kTileBytes);
   float* xch = reinterpret_cast<float*>(sh + 1);              // [2 parities][2 halves][128] row maxima; reused for the sums
   int32_t* kp_all = reinterpret_cast<int32_t*>(xch + 2 * 2 * kTile);  // [2 parities][128] keys' original indices
 
@@ -219,12 +176,14 @@ aifs_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmap_k)) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmap_vt)) : "memory");
     mbar_init(&sh->q_full, 1);
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < kStages; ++i) {
       mbar_init(&sh->k_full[i], 1); mbar_init(&sh->k_empty[i], 1);
       mbar_init(&sh->v_full[i], 1); mbar_init(&sh->v_empty[i], 1);
-      mbar_init(&sh->s_full[i], 1); mbar_init(&sh->s_empty[i], 8);
     }
-    mbar_init(&sh->p_full, 8); mbar_init(&sh->pv_done, 1); mbar_init(&sh->o_empty, 8);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&sh->s_full[i], 1); mbar_init(&sh->s_empty[i], 8);
+      mbar_init(&sh->p_full[i], 8); mbar_init(&sh->pv_done[i], 1);
+    }
     mbar_init(&sh->drain, 1);
     sh->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -237,7 +196,6 @@ aifs_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&sh->tmem_base);
-  // tensor-memory columns: S buffers at 0 and 128, the P V product at 256
 
   if (warp == 0) {
     // ---------------- TMA producer: Q once, then K and V^T tiles of every key tile that is not skipped
@@ -245,17 +203,16 @@ aifs_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
       mbar_arrive_expect_tx(&sh->q_full, kTileBytes);
       tma_load_2d(q_smem, &tmap_q, head * kD, q0, &sh->q_full);
       tma_load_2d(q_smem + kHalfBytes, &tmap_q, head * kD + 64, q0, &sh->q_full);
-      int t = 0;
+      int t = 0, s = 0;
+      uint32_t ph = 0;
       bool ok = true;
       for (int kt = 0; kt < p.n_tiles && ok; ++kt) {
         if (tile_class(p, qt, kt) == 0) continue;
-        const int s = t & 1;
-        const uint32_t ph = (uint32_t)(t >> 1) & 1u;
-        if (t >= 2 && !(ok = mbar_wait(&sh->k_empty[s], ph ^ 1u, &sh->abort_flag, p.status, 21))) break;
+        if (t >= kStages && !(ok = mbar_wait(&sh->k_empty[s], ph ^ 1u, &sh->abort_flag, p.status, 21))) break;
         mbar_arrive_expect_tx(&sh->k_full[s], kTileBytes);
         tma_load_2d(k_smem + s * kTileBytes, &tmap_k, g * kD, kt * kTile, &sh->k_full[s]);
         tma_load_2d(k_smem + s * kTileBytes + kHalfBytes, &tmap_k, g * kD + 64, kt * kTile, &sh->k_full[s]);
-        if (t >= 2 && !(ok = mbar_wait(&sh->v_empty[s], ph ^ 1u, &sh->abort_flag, p.status, 22))) {
+        if (t >= kStages && !(ok = mbar_wait(&sh->v_empty[s], ph ^ 1u, &sh->abort_flag, p.status, 22))) {
           mbar_wait_drain(&sh->k_full[s], ph, 20000ull);
           break;
         }
@@ -263,56 +220,59 @@ aifs_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
         tma_load_2d(v_smem + s * kTileBytes, &tmap_vt, kt * kTile, g * kD, &sh->v_full[s]);
         tma_load_2d(v_smem + s * kTileBytes + kHalfBytes, &tmap_vt, kt * kTile + 64, g * kD, &sh->v_full[s]);
         ++t;
+        if (++s == kStages) { s = 0; ph ^= 1u; }
       }
       if (!ok) {
         // copies still landing in this CTA's shared memory get time to finish before it exits
         mbar_wait_drain(&sh->q_full, 0, 20000ull);
-        for (int back = 1; back <= 2 && back <= t; ++back) {
+        for (int back = 1; back <= kStages && back <= t; ++back) {
           const int u = t - back;
-          mbar_wait_drain(&sh->k_full[u & 1], (uint32_t)(u >> 1) & 1u, 20000ull);
-          mbar_wait_drain(&sh->v_full[u & 1], (uint32_t)(u >> 1) & 1u, 20000ull);
+          mbar_wait_drain(&sh->k_full[u % kStages], (uint32_t)(u / kStages) & 1u, 20000ull);
+          mbar_wait_drain(&sh->v_full[u % kStages], (uint32_t)(u / kStages) & 1u, 20000ull);
         }
       }
     }
   } else if (warp == 1) {
-    // ---------------- MMA issuer: S_t = Q K_t^T is issued one tile ahead of O_{t-1} = P_{t-1} V_{t-1}, so
-    // that the tensor cores work on the next scores while the softmax warps are busy with the current ones
+    // ---------------- MMA issuer: S_t = Q K_t^T is issued one tile ahead of O += P_{t-1} V_{t-1}, so that
+    // the tensor cores work on the next scores while the softmax warps are busy with the current ones
     if (elect_one()) {
       const uint32_t idesc = make_idesc_bf16(kTile);
       const uint64_t qdesc = make_b_desc(smem_u32(q_smem));
-      const uint64_t pdesc = make_b_desc(smem_u32(p_smem));
       bool ok = mbar_wait(&sh->q_full, 0, &sh->abort_flag, p.status, 23);
-      int t = 0;
+      int t = 0, ks = 0, vs = 0;       // tile count; ring positions of the next K and the next V tile
+      uint32_t kph = 0, vph = 0;
       auto issue_pv = [&](int u) -> bool {
-        if (!mbar_wait(&sh->v_full[u & 1], (uint32_t)(u >> 1) & 1u, &sh->abort_flag, p.status, 24)) return false;
-        if (!mbar_wait(&sh->p_full, (uint32_t)u & 1u, &sh->abort_flag, p.status, 25)) return false;
-        if (u >= 1 && !mbar_wait(&sh->o_empty, (uint32_t)(u - 1) & 1u, &sh->abort_flag, p.status, 26)) return false;
+        const int b = u & 1;
+        if (!mbar_wait(&sh->v_full[vs], vph, &sh->abort_flag, p.status, 24)) return false;
+        if (!mbar_wait(&sh->p_full[b], (uint32_t)(u >> 1) & 1u, &sh->abort_flag, p.status, 25)) return false;
         tc_fence_after();
-        const uint64_t vdesc = make_b_desc(smem_u32(v_smem + (u & 1) * kTileBytes));
+        const uint64_t vdesc = make_b_desc(smem_u32(v_smem + vs * kTileBytes));
+        const uint32_t p_tmem = tmem_base + kColP + (uint32_t)(b * 64);
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
           const uint64_t off = (uint64_t)((k >> 2) * (kHalfBytes >> 4) + (k & 3) * 2);
-          mma_bf16_ss(tmem_base + 256u, pdesc + off, vdesc + off, idesc, k ? 1u : 0u);
+          mma_bf16_ts(tmem_base + kColO, p_tmem + (uint32_t)(k * 8), vdesc + off, idesc, (u > 0 || k > 0) ? 1u : 0u);
         }
-        tc_commit(&sh->pv_done);
-        tc_commit(&sh->v_empty[u & 1]);
+        tc_commit(&sh->pv_done[b]);
+        tc_commit(&sh->v_empty[vs]);
+        if (++vs == kStages) { vs = 0; vph ^= 1u; }
         return true;
       };
       for (int kt = 0; kt < p.n_tiles && ok; ++kt) {
         if (tile_class(p, qt, kt) == 0) continue;
-        const int s = t & 1;
-        const uint32_t ph = (uint32_t)(t >> 1) & 1u;
-        if (!(ok = mbar_wait(&sh->k_full[s], ph, &sh->abort_flag, p.status, 27))) break;
-        if (t >= 2 && !(ok = mbar_wait(&sh->s_empty[s], ph ^ 1u, &sh->abort_flag, p.status, 28))) break;
+        const int sb = t & 1;
+        if (!(ok = mbar_wait(&sh->k_full[ks], kph, &sh->abort_flag, p.status, 27))) break;
+        if (t >= 2 && !(ok = mbar_wait(&sh->s_empty[sb], ((uint32_t)(t >> 1) & 1u) ^ 1u, &sh->abort_flag, p.status, 28))) break;
         tc_fence_after();
-        const uint64_t kdesc = make_b_desc(smem_u32(k_smem + s * kTileBytes));
+        const uint64_t kdesc = make_b_desc(smem_u32(k_smem + ks * kTileBytes));
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
           const uint64_t off = (uint64_t)((k >> 2) * (kHalfBytes >> 4) + (k & 3) * 2);
-          mma_bf16_ss(tmem_base + (uint32_t)(s * kTile), qdesc + off, kdesc + off, idesc, k ? 1u : 0u);
+          mma_bf16_ss(tmem_base + (uint32_t)(sb * kTile), qdesc + off, kdesc + off, idesc, k ? 1u : 0u);
         }
-        tc_commit(&sh->s_full[s]);
-        tc_commit(&sh->k_empty[s]);
+        tc_commit(&sh->s_full[sb]);
+        tc_commit(&sh->k_empty[ks]);
+        if (++ks == kStages) { ks = 0; kph ^= 1u; }
         if (t >= 1 && !(ok = issue_pv(t - 1))) break;
         ++t;
       }
@@ -333,79 +293,109 @@ aifs_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
     const int perm_i = i < p.L ? p.perm[i] : -1;
     const bool pad_i = i < p.L && p.pad_u && p.pad_u[i];
     const uint32_t lane_base = tmem_base + ((uint32_t)(quarter * 32) << 16);
-    uint8_t* p_row = p_smem + half * kHalfBytes + (row >> 3) * 1024 + (row & 7) * 128;
-    float acc[64];
-#pragma unroll
-    for (int e = 0; e < 64; ++e) acc[e] = 0.0f;
-    float m_run = -1.0e30f, l_run = 0.0f, alpha_pending = 1.0f;
+    const uint32_t o_addr = lane_base + kColO + (uint32_t)(half * 64);
+    const float lag_raw = kLagLog2 / p.scale_log2;   // the lag in units of the raw scores
+    float m_used = -1.0e30f, l_run = 0.0f;           // reference maximum of the exponents; sum relative to it
     int t = 0;
     bool ok = true;
     for (int kt = 0; kt < p.n_tiles; ++kt) {
       const int cls = tile_class(p, qt, kt);
       if (cls == 0) continue;
-      const int s = t & 1;
-      int32_t* kp = kp_all + s * kTile;
+      const int sb = t & 1;
+      int32_t* kp = kp_all + sb * kTile;
       if (cls == 1 && tid < kTile) {
         const int j = kt * kTile + tid;
         kp[tid] = (j < p.L && !(p.pad_u && p.pad_u[j])) ? p.perm[j] : INT_MAX;
       }
       // one verdict for all softmax threads: nobody leaves the loop while others still wait at a barrier
       if (named_bar_or(1, kSoftmaxThreads, !ok)) { ok = false; break; }
-      ok = warp_all(mbar_wait(&sh->s_full[s], (uint32_t)(t >> 1) & 1u, &sh->abort_flag, p.status, 29));  // (ok was true)
+      ok = warp_all(mbar_wait(&sh->s_full[sb], (uint32_t)(t >> 1) & 1u, &sh->abort_flag, p.status, 29));  // (ok was true)
       tc_fence_after();
-      const uint32_t s_addr = lane_base + (uint32_t)(s * kTile + half * 64);
-      // a padded row attends itself: the column of the diagonal inside this thread's 64, if it is there
-      const int self_col = (pad_i && kt == qt && (row >> 6) == half) ? (row & 63) : -1;
-      const int32_t* kph = kp + half * 64;
-      float mx = cls == 1 ? row_max_pass<true>(s_addr, kph, perm_i, self_col) : row_max_pass<false>(s_addr, kph, perm_i, self_col);
-      float* xm = xch + (s * 2) * kTile;
+      // this thread's 64 scores, read once; the buffer goes back to the MMA issuer right away
+      uint32_t sv[64];
+      {
+        uint32_t (&lo)[32] = *reinterpret_cast<uint32_t (*)[32]>(&sv[0]);
+        uint32_t (&hi)[32] = *reinterpret_cast<uint32_t (*)[32]>(&sv[32]);
+        const uint32_t s_addr = lane_base + (uint32_t)(sb * kTile + half * 64);
+        tmem_ld_x32(s_addr, lo);
+        tmem_ld_x32(s_addr + 32u, hi);
+        tmem_wait_ld();
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sh->s_empty[sb]);
+      // mask (a padded row attends itself: the column of the diagonal inside this thread's 64, if it is there)
+      if (cls == 1) {
+        const int self_col = (pad_i && kt == qt && (row >> 6) == half) ? (row & 63) : -1;
+        const int32_t* kph2 = kp + half * 64;
+#pragma unroll
+        for (int e = 0; e < 64; ++e)
+          if (!(kph2[e] <= perm_i || e == self_col)) sv[e] = 0xff800000u;  // -inf
+      }
+      float mx = -1.0e30f;
+#pragma unroll
+      for (int e = 0; e < 64; ++e) mx = fmaxf(mx, __uint_as_float(sv[e]));
+      float* xm = xch + (sb * 2) * kTile;
       xm[half * kTile + row] = mx;
       named_bar_sync(2, kSoftmaxThreads);
-      mx = fmaxf(mx, xm[(half ^ 1) * kTile + row]);
-      const float m_new = fmaxf(m_run, mx);
-      const float alpha = fast_exp2((m_run - m_new) * p.scale_log2);
-      m_run = m_new;
-      if (t >= 1) {
-        // fold the previous tile's P V into the running output (and free P and the product buffer)
-        ok = warp_all(mbar_wait(&sh->pv_done, (uint32_t)(t - 1) & 1u, &sh->abort_flag, p.status, 30)) && ok;
-        tc_fence_after();
+      const float m_new = fmaxf(m_used, fmaxf(mx, xm[(half ^ 1) * kTile + row]));
+      // move the reference maximum only when some row of this quarter has outgrown it (both halves of a row see
+      // the same numbers and decide alike); then the accumulated output and sum are rescaled
+      const bool move = __any_sync(0xffffffffu, m_new > m_used + lag_raw);
+      if (move) {
+        if (t >= 1) {
+          ok = warp_all(mbar_wait(&sh->pv_done[(t - 1) & 1], (uint32_t)((t - 1) >> 1) & 1u, &sh->abort_flag, p.status, 30)) && ok;
+          tc_fence_after();
+          const float f = fast_exp2((m_used - m_new) * p.scale_log2);
 #pragma unroll
-        for (int cb = 0; cb < 64; cb += 32) {
-          uint32_t v[32];
-          tmem_ld_x32(lane_base + 256u + (uint32_t)(half * 64 + cb), v);
-          tmem_wait_ld();
+          for (int cb = 0; cb < 64; cb += 32) {
+            uint32_t v[32];
+            tmem_ld_x32(o_addr + (uint32_t)cb, v);
+            tmem_wait_ld();
 #pragma unroll
-          for (int e = 0; e < 32; ++e) acc[cb + e] = fmaf(acc[cb + e], alpha_pending, __uint_as_float(v[e]));
+            for (int e = 0; e < 32; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) * f);
+            tmem_st_x32(o_addr + (uint32_t)cb, v);
+          }
+          tmem_wait_st();
+          l_run *= f;
         }
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&sh->o_empty);
+        m_used = m_new;
       }
-      alpha_pending = alpha;
-      const float sum = cls == 1 ? prob_pass<true>(s_addr, kph, perm_i, self_col, p.scale_log2, m_run, p_row, row & 7)
-                                 : prob_pass<false>(s_addr, kph, perm_i, self_col, p.scale_log2, m_run, p_row, row & 7);
-      l_run = fmaf(l_run, alpha, sum);
+      // the P buffer of this parity is free once the product of two tiles ago has read it
+      if (t >= 2)
+        ok = warp_all(mbar_wait(&sh->pv_done[sb], (uint32_t)((t - 2) >> 1) & 1u, &sh->abort_flag, p.status, 31)) && ok;
+      tc_fence_after();
+      const float bias = -m_used * p.scale_log2;
+      float sum = 0.0f;
+      uint32_t pk[32];
+#pragma unroll
+      for (int e = 0; e < 64; e += 2) {
+        // (a masked score is -inf: exp2 gives 0; a row with nothing to attend yet has m_used = -1e30 and only such scores)
+        const float p0 = fast_exp2(fmaf(__uint_as_float(sv[e]), p.scale_log2, bias));
+        const float p1 = fast_exp2(fmaf(__uint_as_float(sv[e + 1]), p.scale_log2, bias));
+        sum += p0 + p1;
+        pk[e >> 1] = pack_bf16x2(p0, p1);
+      }
+      l_run += sum;
+      tmem_st_x32(lane_base + kColP + (uint32_t)(sb * 64 + half * 32), pk);
+      tmem_wait_st();
       tc_fence_before();
-      fence_proxy_async_smem();
       __syncwarp();
-      if (lane == 0) {
-        mbar_arrive(&sh->s_empty[s]);
-        mbar_arrive(&sh->p_full);
-      }
+      if (lane == 0) mbar_arrive(&sh->p_full[sb]);
       ++t;
     }
+    float acc[64];
+#pragma unroll
+    for (int e = 0; e < 64; ++e) acc[e] = 0.0f;
     if (ok && t >= 1) {
-      ok = warp_all(mbar_wait(&sh->pv_done, (uint32_t)(t - 1) & 1u, &sh->abort_flag, p.status, 31));
+      ok = warp_all(mbar_wait(&sh->pv_done[(t - 1) & 1], (uint32_t)((t - 1) >> 1) & 1u, &sh->abort_flag, p.status, 32));
       tc_fence_after();
       if (ok) {
-#pragma unroll
-        for (int cb = 0; cb < 64; cb += 32) {
-          uint32_t v[32];
-          tmem_ld_x32(lane_base + 256u + (uint32_t)(half * 64 + cb), v);
-          tmem_wait_ld();
-#pragma unroll
-          for (int e = 0; e < 32; ++e) acc[cb + e] = fmaf(acc[cb + e], alpha_pending, __uint_as_float(v[e]));
-        }
+        uint32_t (&lo)[32] = *reinterpret_cast<uint32_t (*)[32]>(&acc[0]);
+        uint32_t (&hi)[32] = *reinterpret_cast<uint32_t (*)[32]>(&acc[32]);
+        tmem_ld_x32(o_addr, lo);
+        tmem_ld_x32(o_addr + 32u, hi);
+        tmem_wait_ld();
       }
     }
     // the two halves of a row add their sums; then O = acc / l, rounded to bf16
@@ -434,7 +424,7 @@ aifs_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
   }
 }
 
-constexpr size_t kAttnSmem = 1024 + 6 * (size_t)kTileBytes + sizeof(AttnBarriers) + 2 * 2 * kTile * sizeof(float) +
+constexpr size_t kAttnSmem = 1024 + (1 + 2 * kStages) * (size_t)kTileBytes + sizeof(AttnBarriers) + 2 * 2 * kTile * sizeof(float) +
                              2 * kTile * sizeof(int32_t);
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,

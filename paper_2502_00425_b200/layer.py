@@ -2,10 +2,11 @@
 
 The linears, the AIFS reorder and the mask / position remap run through the C ABI (the
 product).  Everything between them -- RMSNorm, rotary embedding, masked grouped-query
-attention, SwiGLU, the residual adds -- is plain torch on the same device: glue that lets a
+attention, SwiGLU, the residual adds -- runs as the library's glue kernels (mq_glue_*,
+mq_aifs_attention) or, with those switched off, as plain torch on the same device: glue that lets a
 sequence flow through a whole block (Sec. 3.1: AIFS once at the input, the unified mask and the
 remapped positions in attention, MSQ in front of every linear, the online Hadamard in front of
-the down-projection, Fig. 4(a)).  The glue is not tuned and not part of the measured kernels.
+the down-projection, Fig. 4(a)).
 
 A block takes one sequence, or a batch of sequences, in the original token order and returns
 the outputs in that order.  Every sequence is reordered on its own; the linears then see the
@@ -108,6 +109,7 @@ class W4A8DecoderBlock:
         self.shape, self.w, self.g_attn, self.g_mlp, self.device = shape, weights, g_attn, g_mlp, device
         self._ws: Dict[Tuple[str, int], torch.Tensor] = {}
         self._fused: Dict[str, Optional[LinearWeights]] = {}
+        self._attn_ws: Dict[int, Tuple[torch.Tensor, torch.Tensor]] = {}   # per sequence length: (scratch, status word)
         # True: q/k/v and gate/up each run as one linear over the stacked weight (same results)
         self.fuse_groups = False
         # True: RMSNorm, rotary embedding, SwiGLU and the residual adds run as the library's single-pass
@@ -116,6 +118,9 @@ class W4A8DecoderBlock:
         # True: attention in the original order with a plain causal mask instead of the dense unified
         # mask (same result, much faster glue); the dense mask is still produced and kept in the trace
         self.causal_glue = False
+        # True: attention under the unified mask runs as the library's tensor-core kernel (mq_aifs_attention),
+        # in AIFS order, straight from the permutation -- no dense mask, no reordering; head_dim must be 128
+        self.cuda_attention = shape.head_dim == 128
 
     # ---- pieces ------------------------------------------------------------------------
     def aifs(self, embs, is_visuals, tr: BlockTrace) -> torch.Tensor:
@@ -256,7 +261,17 @@ class W4A8DecoderBlock:
         qr = self._rope(q, tr, sh.n_q_heads)
         kr = self._rope(k, tr, sh.n_kv_heads)
         t["q_rope"], t["k_rope"] = qr, kr
-        if self.causal_glue:
+        if self.cuda_attention:
+            a = torch.empty((qr.shape[0], qr.shape[1]), dtype=torch.bfloat16, device=qr.device)
+            for b in range(n_seq):
+                L_b = bd[b + 1] - bd[b]
+                if L_b not in self._attn_ws:
+                    self._attn_ws[L_b] = (torch.empty(B.mq_aifs_attention_workspace_bytes(L_b, sh.n_kv_heads), dtype=torch.uint8,
+                                                 device=qr.device), torch.zeros(2, dtype=torch.int32, device=qr.device))
+                ws, status = self._attn_ws[L_b]
+                B.mq_aifs_attention(qr[bd[b]:bd[b + 1]], kr[bd[b]:bd[b + 1]], v[bd[b]:bd[b + 1]], tr.perms[b], None,
+                                    sh.n_q_heads, sh.n_kv_heads, a[bd[b]:bd[b + 1]], ws, status)
+        elif self.causal_glue:
             a = torch.cat([gqa_attention_unpermuted(qr[bd[b]:bd[b + 1]], kr[bd[b]:bd[b + 1]], v[bd[b]:bd[b + 1]],
                                                     tr.perms[b], sh.n_q_heads, sh.n_kv_heads) for b in range(n_seq)])
         else:
@@ -310,7 +325,8 @@ class W4A8DecoderBlock:
         return y
 
     def device_status_ok(self) -> bool:
-        return all(B.mq_last_device_status(ws)[0] == B.MQ_OK for ws in self._ws.values())
+        return (all(B.mq_last_device_status(ws)[0] == B.MQ_OK for ws in self._ws.values())
+                and all(int(status[0]) == B.MQ_OK for _, status in self._attn_ws.values()))
 
 
 def random_block(shape: LayerShape, seed: int, device="cuda") -> W4A8DecoderBlock:
