@@ -444,7 +444,7 @@ int mq_glue_residual_add(const void* A, int64_t lda, const void* Bm, int64_t ldb
  * Q [L, n_q_heads * D], K, V [L, n_kv_heads * D], O [L, n_q_heads * D]: device bf16, row-major, leading
  * dimensions in elements, rows 16-byte aligned; Q and K already carry the rotary embedding.  perm: device
  * int32 [L] (mq_aifs_reorder's output).  pad_u: device uint8 [L] in AIFS order (1 = padded row) or NULL.
- * head_dim must be 128 (MQ_ERR_UNSUPPORTED otherwise).  float32 accumulation; the probabilities enter the
+ * head_dim must be 128 and L at most 131072 (MQ_ERR_UNSUPPORTED otherwise).  float32 accumulation; the probabilities enter the
  * second product rounded to bf16.  ws: device scratch of mq_aifs_attention_workspace_bytes() bytes, 16-byte
  * aligned (it receives V transposed and the per-tile index bounds); status: device int32[2], zeroed by the
  * caller, receives MQ_ERR_TIMEOUT and the wait site if a bounded wait inside the kernel expires.

@@ -12,14 +12,17 @@
 // kind::f16 on bf16 operands from shared memory, float32 accumulators in tensor memory):
 //   * Q, K tiles and V^T tiles arrive by TMA (128-byte swizzle).  V is transposed once per call by a small
 //     prep kernel so that the second product's B operand is K-major like every other operand here;
-//   * S = Q K^T (128 x 128) goes to one of two tensor-memory buffers; eight softmax warps (two per 32-lane
-//     quarter; each thread owns one query row and half of the columns) read it once into registers, apply
-//     the mask, form P = exp2(...) and write it as bf16 back into tensor memory, where the second product
-//     takes it as its A operand: the probabilities never touch shared memory;
-//   * O += P V accumulates in tensor memory across the key tiles.  The exponents are taken relative to a
-//     reference maximum that may lag the true running maximum by up to 8 powers of two; only when a row
-//     outgrows it are the accumulated output and sum rescaled (online softmax with a lazy rescale), so the
-//     softmax warps normally never touch O until the end;
+//   * the key tiles a query tile has to process go alternately to two groups of four softmax warps.  Each
+//     group has its own score buffer and its own output accumulator in tensor memory and runs a complete
+//     online softmax over its tiles; the two partial results are merged at the end (as for a split over
+//     the keys).  While one group works on its scores the tensor cores compute the other group's;
+//   * a softmax thread owns one query row: it reads its 128 scores from tensor memory (once for the row
+//     maximum, once for the exponentials), applies the mask and writes P = exp2(...) as bf16 over the
+//     scores it has read, where the second product takes it as its A operand: the probabilities never
+//     touch shared memory;
+//   * O_g += P V accumulates in tensor memory.  The exponents are taken relative to a reference maximum
+//     that may lag the true running maximum by up to 8 powers of two; only when a row outgrows it are the
+//     accumulated output and sum rescaled, so the softmax warps normally never touch O until the end;
 //   * key tiles no row of the query tile may see are skipped, and tiles every row may see in full skip the
 //     mask: the prep kernel stores, per 128-row tile, the smallest and largest original index.
 // Every wait on an mbarrier is bounded (see mq_sm100.cuh); an expired wait raises the CTA's abort flag, all
@@ -42,17 +45,20 @@ constexpr int kHalfBytes = 64 * kTile * 2;   // one 128-row x 64-element swizzle
 constexpr int kTileBytes = 2 * kHalfBytes;   // a 128 x 128 bf16 operand tile
 constexpr int kThreads = 12 * 32;            // producer, MMA issuer, allocator, spare, 8 softmax warps
 constexpr int kSoftmaxThreads = 8 * 32;
+constexpr int kMaxTiles = 1024;              // 128-row tiles per sequence (the CTA's tile list lives in shared memory)
 
 constexpr int kStages = 2;                   // K tiles and V^T tiles in flight (each ring)
 
 struct AttnBarriers {
   uint64_t q_full;
   uint64_t k_full[kStages], k_empty[kStages], v_full[kStages], v_empty[kStages];
-  uint64_t s_full[2], s_empty[2];   // a score buffer is written (MMA commit) / has been read (eight softmax warps)
-  uint64_t p_full[2], pv_done[2];   // a P buffer is written (eight warps) / its product into O is complete (commit)
+  // per softmax group: its score buffer is written (MMA commit); P has replaced the scores (the group's four
+  // warps); the product of that P into the group's accumulator is complete (MMA commit)
+  uint64_t s_full[2], p_full[2], pv_done[2];
   uint64_t drain;
   uint32_t tmem_base;
   int abort_flag;
+  int n_list;     // entries of the CTA's tile list
 };
 
 struct AttnParams {
@@ -69,15 +75,17 @@ struct AttnParams {
   int32_t* status;
 };
 
-// 0: no row of the query tile may attend any row of the key tile; 1: some may; 2: all may attend all.
-__device__ __forceinline__ int tile_class(const AttnParams& p, int qt, int kt) {
-  if (kt != qt && p.kmin[kt] > p.qmax[qt]) return 0;
-  return p.kmaxc[kt] <= p.qmin[qt] ? 2 : 1;
-}
+// Classes of a key tile for a query tile: 0: no row of the query tile may attend any row of the key tile (it is
+// skipped); 1: some may (masked); 2: all may attend all (no mask needed).
 
 __device__ __forceinline__ float fast_exp2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float fast_rcp(float x) {
+  float y;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
@@ -144,10 +152,106 @@ attn_prep_kernel(const uint16_t* __restrict__ V, int64_t ldv, int L, int Lp, con
   }
 }
 
+// ---------------------------------------------------------------------------------------- softmax pieces
+// A thread's 128 scores are read from tensor memory in four chunks of 32 columns; the load of the next chunk is
+// in flight while the current one is worked on (two register buffers), because a tensor-memory load takes a few
+// hundred cycles and only two softmax warps share a scheduler.
+//
+// Maximum of one chunk into four independent partial maxima (a single chain of 128 dependent max operations
+// would cost more than the exponentials).
+template <bool MASKED>
+__device__ __forceinline__ void chunk_max(const uint32_t (&v)[32], uint32_t allowed, float (&mx)[4]) {
+#pragma unroll
+  for (int e = 0; e < 32; ++e) {
+    const float x = __uint_as_float(v[e]);
+    if (!MASKED || ((allowed >> e) & 1u)) mx[e & 3] = fmaxf(mx[e & 3], x);
+  }
+}
+
+// P = exp2(scale * s + bias) of one chunk as 16 bf16 pairs; adds the chunk's probabilities into two packed sums.
+template <bool MASKED>
+__device__ __forceinline__ void chunk_prob(const uint32_t (&v)[32], uint32_t allowed, float2 scale2, float2 bias2,
+                                           float2 (&sum2)[2], uint32_t (&pk)[16]) {
+#pragma unroll
+  for (int e = 0; e < 32; e += 2) {
+    const float2 x = __ffma2_rn(make_float2(__uint_as_float(v[e]), __uint_as_float(v[e + 1])), scale2, bias2);
+    float2 pr = make_float2(fast_exp2(x.x), fast_exp2(x.y));
+    if (MASKED) {
+      if (!((allowed >> e) & 1u)) pr.x = 0.0f;
+      if (!((allowed >> (e + 1)) & 1u)) pr.y = 0.0f;
+    }
+    sum2[(e >> 1) & 1] = __fadd2_rn(sum2[(e >> 1) & 1], pr);
+    pk[e >> 1] = pack_bf16x2(pr.x, pr.y);
+  }
+}
+
+// Row maximum of the 128 scores at s_addr.
+template <bool MASKED>
+__device__ __forceinline__ float row_max(uint32_t s_addr, const uint32_t (&allowed)[4]) {
+  float mx[4] = {-1.0e30f, -1.0e30f, -1.0e30f, -1.0e30f};
+  uint32_t a[32], b[32];
+  tmem_ld_x32(s_addr, a);
+  tmem_wait_ld();
+  tmem_ld_x32(s_addr + 32u, b);
+  chunk_max<MASKED>(a, allowed[0], mx);
+  tmem_wait_ld();
+  tmem_ld_x32(s_addr + 64u, a);
+  chunk_max<MASKED>(b, allowed[1], mx);
+  tmem_wait_ld();
+  tmem_ld_x32(s_addr + 96u, b);
+  chunk_max<MASKED>(a, allowed[2], mx);
+  tmem_wait_ld();
+  chunk_max<MASKED>(b, allowed[3], mx);
+  return fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+}
+
+// The 128 probabilities of the row, written as bf16 pairs over the first 64 columns of the score buffer; every
+// store lands on columns whose scores this thread has already consumed.  Returns the row sum.
+template <bool MASKED>
+__device__ __forceinline__ float row_prob(uint32_t s_addr, const uint32_t (&allowed)[4], float scale_log2, float m_used) {
+  const float2 scale2 = make_float2(scale_log2, scale_log2);
+  const float bias = -m_used * scale_log2;
+  const float2 bias2 = make_float2(bias, bias);
+  float2 sum2[2] = {make_float2(0.0f, 0.0f), make_float2(0.0f, 0.0f)};
+  uint32_t a[32], b[32], pk[16];
+  tmem_ld_x32(s_addr, a);
+  tmem_wait_ld();
+  tmem_ld_x32(s_addr + 32u, b);
+  chunk_prob<MASKED>(a, allowed[0], scale2, bias2, sum2, pk);
+  tmem_st_x16(s_addr, pk);
+  tmem_wait_ld();
+  tmem_ld_x32(s_addr + 64u, a);
+  chunk_prob<MASKED>(b, allowed[1], scale2, bias2, sum2, pk);
+  tmem_st_x16(s_addr + 16u, pk);
+  tmem_wait_ld();
+  tmem_ld_x32(s_addr + 96u, b);
+  chunk_prob<MASKED>(a, allowed[2], scale2, bias2, sum2, pk);
+  tmem_st_x16(s_addr + 32u, pk);
+  tmem_wait_ld();
+  chunk_prob<MASKED>(b, allowed[3], scale2, bias2, sum2, pk);
+  tmem_st_x16(s_addr + 48u, pk);
+  tmem_wait_st();
+  return (sum2[0].x + sum2[0].y) + (sum2[1].x + sum2[1].y);
+}
+
+// Bit j of the result: may this thread's row attend key column j of the tile (kp: the keys' original indices,
+// INT_MAX for padded or out-of-range keys; self_col: the diagonal column of a padded row, or -1).
+__device__ __forceinline__ void allowed_bits(const int32_t* kp, int perm_i, int self_col, uint32_t (&allowed)[4]) {
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    uint32_t w = 0;
+#pragma unroll 8
+    for (int b = 0; b < 32; ++b) w |= (uint32_t)(kp[c * 32 + b] <= perm_i) << b;
+    allowed[c] = w;
+  }
+  if (self_col >= 0) allowed[self_col >> 5] |= 1u << (self_col & 31);
+}
+
 // ---------------------------------------------------------------------------------------- the kernel
-// Tensor-memory columns: S buffers at 0 and 128 (float32), the output accumulator O at 256 (float32), the
-// two P buffers at 384 and 448 (bf16 pairs: 64 columns hold 128 probabilities per row).
-constexpr uint32_t kColO = 256, kColP = 384;
+// Tensor-memory columns: group g (0: the even, 1: the odd processed key tiles) has its score buffer at 128 g --
+// whose first 64 columns are overwritten in place by P (bf16 pairs) once the scores have been read -- and
+// its output accumulator at 256 + 128 g.
+constexpr uint32_t kColO = 256;
 // The exponent's reference maximum may lag the true running maximum by this many powers of two before the
 // accumulated output is rescaled (probabilities then reach at most 2^8, harmless in float32 / bf16).
 constexpr float kLagLog2 = 8.0f;
@@ -161,8 +265,9 @@ aifs_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
   uint8_t* k_smem = q_smem + kTileBytes;        // kStages x 32 KB
   uint8_t* v_smem = k_smem + kStages * kTileBytes;
   AttnBarriers* sh = reinterpret_cast<AttnBarriers*>(v_smem + kStages * kTileBytes);
-  float* xch = reinterpret_cast<float*>(sh + 1);              // [2 parities][2 halves][128] row maxima; reused for the sums
-  int32_t* kp_all = reinterpret_cast<int32_t*>(xch + 2 * 2 * kTile);  // [2 parities][128] keys' original indices
+  float* xch = reinterpret_cast<float*>(sh + 1);                     // [2 groups][128 rows][m, l] for the final merge
+  int32_t* kp_all = reinterpret_cast<int32_t*>(xch + 2 * kTile * 2);  // [8 warps][128] keys' original indices
+  int32_t* tile_list = kp_all + 8 * kTile;   // [kMaxTiles] the key tiles this query tile processes: index | class << 16
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // heavy query tiles (late rows see the most keys) first; the heads of one key/value group side by side
@@ -181,8 +286,7 @@ aifs_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
       mbar_init(&sh->v_full[i], 1); mbar_init(&sh->v_empty[i], 1);
     }
     for (int i = 0; i < 2; ++i) {
-      mbar_init(&sh->s_full[i], 1); mbar_init(&sh->s_empty[i], 8);
-      mbar_init(&sh->p_full[i], 8); mbar_init(&sh->pv_done[i], 1);
+      mbar_init(&sh->s_full[i], 1); mbar_init(&sh->p_full[i], 4); mbar_init(&sh->pv_done[i], 1);
     }
     mbar_init(&sh->drain, 1);
     sh->abort_flag = 0;
@@ -192,10 +296,27 @@ aifs_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
     tmem_alloc(&sh->tmem_base, 512);
     tmem_relinquish();
   }
+  if (warp == 1) {
+    // The key tiles to process, in order, once per CTA: every role walks this list instead of classifying
+    // all tiles itself (four dependent global loads per tile, also for the skipped ones, were most of a short
+    // CTA's life).  32 tiles are classified per step, one per lane.
+    const int q_lo = p.qmin[qt], q_hi = p.qmax[qt];
+    int count = 0;
+    for (int base = 0; base < p.n_tiles; base += 32) {
+      const int kt = base + lane;
+      int cls = 0;
+      if (kt < p.n_tiles) cls = (kt != qt && p.kmin[kt] > q_hi) ? 0 : (p.kmaxc[kt] <= q_lo ? 2 : 1);
+      const unsigned take = __ballot_sync(0xffffffffu, cls != 0);
+      if (cls != 0) tile_list[count + __popc(take & ((1u << lane) - 1u))] = kt | (cls << 16);
+      count += __popc(take);
+    }
+    if (lane == 0) sh->n_list = count;
+  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&sh->tmem_base);
+  const int n_list = *reinterpret_cast<volatile int*>(&sh->n_list);
 
   if (warp == 0) {
     // ---------------- TMA producer: Q once, then K and V^T tiles of every key tile that is not skipped
@@ -206,8 +327,8 @@ aifs_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
       int t = 0, s = 0;
       uint32_t ph = 0;
       bool ok = true;
-      for (int kt = 0; kt < p.n_tiles && ok; ++kt) {
-        if (tile_class(p, qt, kt) == 0) continue;
+      for (int idx = 0; idx < n_list && ok; ++idx) {
+        const int kt = tile_list[idx] & 0xffff;
         if (t >= kStages && !(ok = mbar_wait(&sh->k_empty[s], ph ^ 1u, &sh->abort_flag, p.status, 21))) break;
         mbar_arrive_expect_tx(&sh->k_full[s], kTileBytes);
         tma_load_2d(k_smem + s * kTileBytes, &tmap_k, g * kD, kt * kTile, &sh->k_full[s]);
@@ -233,8 +354,10 @@ aifs_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
       }
     }
   } else if (warp == 1) {
-    // ---------------- MMA issuer: S_t = Q K_t^T is issued one tile ahead of O += P_{t-1} V_{t-1}, so that
-    // the tensor cores work on the next scores while the softmax warps are busy with the current ones
+    // ---------------- MMA issuer.  Processed tile u belongs to group u & 1.  S_u = Q K_u^T is issued one tile
+    // ahead of O_g += P_{u-1} V_{u-1}, so the tensor cores work on the other group's scores while one group's
+    // softmax runs.  S_u overwrites the buffer P_{u-2} is read from by the product issued just before it: the
+    // MMAs of one thread execute in the order they were issued, so no wait is needed between the two.
     if (elect_one()) {
       const uint32_t idesc = make_idesc_bf16(kTile);
       const uint64_t qdesc = make_b_desc(smem_u32(q_smem));
@@ -242,35 +365,34 @@ aifs_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
       int t = 0, ks = 0, vs = 0;       // tile count; ring positions of the next K and the next V tile
       uint32_t kph = 0, vph = 0;
       auto issue_pv = [&](int u) -> bool {
-        const int b = u & 1;
+        const int grp = u & 1, n = u >> 1;
         if (!mbar_wait(&sh->v_full[vs], vph, &sh->abort_flag, p.status, 24)) return false;
-        if (!mbar_wait(&sh->p_full[b], (uint32_t)(u >> 1) & 1u, &sh->abort_flag, p.status, 25)) return false;
+        if (!mbar_wait(&sh->p_full[grp], (uint32_t)n & 1u, &sh->abort_flag, p.status, 25)) return false;
         tc_fence_after();
         const uint64_t vdesc = make_b_desc(smem_u32(v_smem + vs * kTileBytes));
-        const uint32_t p_tmem = tmem_base + kColP + (uint32_t)(b * 64);
+        const uint32_t p_tmem = tmem_base + (uint32_t)(grp * kTile);
+        const uint32_t o_tmem = tmem_base + kColO + (uint32_t)(grp * kTile);
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
           const uint64_t off = (uint64_t)((k >> 2) * (kHalfBytes >> 4) + (k & 3) * 2);
-          mma_bf16_ts(tmem_base + kColO, p_tmem + (uint32_t)(k * 8), vdesc + off, idesc, (u > 0 || k > 0) ? 1u : 0u);
+          mma_bf16_ts(o_tmem, p_tmem + (uint32_t)(k * 8), vdesc + off, idesc, (n > 0 || k > 0) ? 1u : 0u);
         }
-        tc_commit(&sh->pv_done[b]);
+        tc_commit(&sh->pv_done[grp]);
         tc_commit(&sh->v_empty[vs]);
         if (++vs == kStages) { vs = 0; vph ^= 1u; }
         return true;
       };
-      for (int kt = 0; kt < p.n_tiles && ok; ++kt) {
-        if (tile_class(p, qt, kt) == 0) continue;
-        const int sb = t & 1;
+      for (int idx = 0; idx < n_list && ok; ++idx) {
+        const int grp = t & 1;
         if (!(ok = mbar_wait(&sh->k_full[ks], kph, &sh->abort_flag, p.status, 27))) break;
-        if (t >= 2 && !(ok = mbar_wait(&sh->s_empty[sb], ((uint32_t)(t >> 1) & 1u) ^ 1u, &sh->abort_flag, p.status, 28))) break;
         tc_fence_after();
         const uint64_t kdesc = make_b_desc(smem_u32(k_smem + ks * kTileBytes));
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
           const uint64_t off = (uint64_t)((k >> 2) * (kHalfBytes >> 4) + (k & 3) * 2);
-          mma_bf16_ss(tmem_base + (uint32_t)(sb * kTile), qdesc + off, kdesc + off, idesc, k ? 1u : 0u);
+          mma_bf16_ss(tmem_base + (uint32_t)(grp * kTile), qdesc + off, kdesc + off, idesc, k ? 1u : 0u);
         }
-        tc_commit(&sh->s_full[sb]);
+        tc_commit(&sh->s_full[grp]);
         tc_commit(&sh->k_empty[ks]);
         if (++ks == kStages) { ks = 0; kph ^= 1u; }
         if (t >= 1 && !(ok = issue_pv(t - 1))) break;
@@ -284,134 +406,115 @@ aifs_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
     }
     __syncwarp();
   } else if (warp >= 4) {
-    // ---------------- softmax warps: thread (row, half) owns query row q0 + row, key columns 64 half .. + 63
-    // of every S tile and head channels 64 half .. + 63 of O
-    const int quarter = warp & 3, half = (warp - 4) >> 2;
+    // ---------------- softmax warps.  Group grp = warps 4 + 4 grp .. 7 + 4 grp takes every second processed key
+    // tile; its thread `row` owns query row q0 + row with all 128 columns of the group's score buffer and keeps
+    // that row's reference maximum and sum over the group's tiles.  A warp depends on no other softmax warp
+    // until the two groups' partial results are merged at the end.
+    const int quarter = warp & 3, grp = (warp - 4) >> 2;
     const int row = quarter * 32 + lane;
     const int i = q0 + row;
-    const int tid = threadIdx.x - 4 * 32;
     const int perm_i = i < p.L ? p.perm[i] : -1;
     const bool pad_i = i < p.L && p.pad_u && p.pad_u[i];
     const uint32_t lane_base = tmem_base + ((uint32_t)(quarter * 32) << 16);
-    const uint32_t o_addr = lane_base + kColO + (uint32_t)(half * 64);
-    const float lag_raw = kLagLog2 / p.scale_log2;   // the lag in units of the raw scores
+    const uint32_t s_addr = lane_base + (uint32_t)(grp * kTile);
+    const uint32_t o_addr = lane_base + kColO + (uint32_t)(grp * kTile);
+    int32_t* kp = kp_all + (warp - 4) * kTile;       // this warp's copy of the key tile's original indices
+    const float lag_raw = kLagLog2 * fast_rcp(p.scale_log2);   // the lag in units of the raw scores
     float m_used = -1.0e30f, l_run = 0.0f;           // reference maximum of the exponents; sum relative to it
-    int t = 0;
+    int n = 0;                                       // this group's tiles so far
     bool ok = true;
-    for (int kt = 0; kt < p.n_tiles; ++kt) {
-      const int cls = tile_class(p, qt, kt);
-      if (cls == 0) continue;
-      const int sb = t & 1;
-      int32_t* kp = kp_all + sb * kTile;
-      if (cls == 1 && tid < kTile) {
-        const int j = kt * kTile + tid;
-        kp[tid] = (j < p.L && !(p.pad_u && p.pad_u[j])) ? p.perm[j] : INT_MAX;
+    for (int idx = grp; idx < n_list && ok; idx += 2) {
+      const int kt = tile_list[idx] & 0xffff;
+      const bool masked = (tile_list[idx] >> 16) == 1;
+      // a padded row attends itself: the column of the diagonal, if this is the diagonal tile
+      const int self_col = (pad_i && kt == qt) ? row : -1;
+      if (masked) {
+        __syncwarp();
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          const int j = kt * kTile + c * 32 + lane;
+          kp[c * 32 + lane] = (j < p.L && !(p.pad_u && p.pad_u[j])) ? p.perm[j] : INT_MAX;
+        }
+        __syncwarp();
       }
-      // one verdict for all softmax threads: nobody leaves the loop while others still wait at a barrier
-      if (named_bar_or(1, kSoftmaxThreads, !ok)) { ok = false; break; }
-      ok = warp_all(mbar_wait(&sh->s_full[sb], (uint32_t)(t >> 1) & 1u, &sh->abort_flag, p.status, 29));  // (ok was true)
+      if (!(ok = warp_all(mbar_wait(&sh->s_full[grp], (uint32_t)n & 1u, &sh->abort_flag, p.status, 29)))) break;
       tc_fence_after();
-      // this thread's 64 scores, read once; the buffer goes back to the MMA issuer right away
-      uint32_t sv[64];
-      {
-        uint32_t (&lo)[32] = *reinterpret_cast<uint32_t (*)[32]>(&sv[0]);
-        uint32_t (&hi)[32] = *reinterpret_cast<uint32_t (*)[32]>(&sv[32]);
-        const uint32_t s_addr = lane_base + (uint32_t)(sb * kTile + half * 64);
-        tmem_ld_x32(s_addr, lo);
-        tmem_ld_x32(s_addr + 32u, hi);
-        tmem_wait_ld();
-      }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&sh->s_empty[sb]);
-      // mask (a padded row attends itself: the column of the diagonal inside this thread's 64, if it is there)
-      if (cls == 1) {
-        const int self_col = (pad_i && kt == qt && (row >> 6) == half) ? (row & 63) : -1;
-        const int32_t* kph2 = kp + half * 64;
-#pragma unroll
-        for (int e = 0; e < 64; ++e)
-          if (!(kph2[e] <= perm_i || e == self_col)) sv[e] = 0xff800000u;  // -inf
-      }
-      float mx = -1.0e30f;
-#pragma unroll
-      for (int e = 0; e < 64; ++e) mx = fmaxf(mx, __uint_as_float(sv[e]));
-      float* xm = xch + (sb * 2) * kTile;
-      xm[half * kTile + row] = mx;
-      named_bar_sync(2, kSoftmaxThreads);
-      const float m_new = fmaxf(m_used, fmaxf(mx, xm[(half ^ 1) * kTile + row]));
-      // move the reference maximum only when some row of this quarter has outgrown it (both halves of a row see
-      // the same numbers and decide alike); then the accumulated output and sum are rescaled
-      const bool move = __any_sync(0xffffffffu, m_new > m_used + lag_raw);
-      if (move) {
-        if (t >= 1) {
-          ok = warp_all(mbar_wait(&sh->pv_done[(t - 1) & 1], (uint32_t)((t - 1) >> 1) & 1u, &sh->abort_flag, p.status, 30)) && ok;
+      // the scores, masked, and the row maximum
+      uint32_t allowed[4] = {~0u, ~0u, ~0u, ~0u};
+      if (masked) allowed_bits(kp, perm_i, self_col, allowed);
+      const float mx = masked ? row_max<true>(s_addr, allowed) : row_max<false>(s_addr, allowed);
+      const float m_new = fmaxf(m_used, mx);
+      // move the reference maximum only when some row of this warp has outgrown it; then the accumulated output
+      // and sum of the warp's rows are rescaled
+      if (__any_sync(0xffffffffu, m_new > m_used + lag_raw)) {
+        if (n >= 1) {
+          if (!(ok = warp_all(mbar_wait(&sh->pv_done[grp], (uint32_t)(n - 1) & 1u, &sh->abort_flag, p.status, 30)))) break;
           tc_fence_after();
           const float f = fast_exp2((m_used - m_new) * p.scale_log2);
 #pragma unroll
-          for (int cb = 0; cb < 64; cb += 32) {
-            uint32_t v[32];
-            tmem_ld_x32(o_addr + (uint32_t)cb, v);
+          for (int cb = 0; cb < kD; cb += 16) {
+            uint32_t v[16];
+            tmem_ld_x16(o_addr + (uint32_t)cb, v);
             tmem_wait_ld();
 #pragma unroll
-            for (int e = 0; e < 32; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) * f);
-            tmem_st_x32(o_addr + (uint32_t)cb, v);
+            for (int e = 0; e < 16; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) * f);
+            tmem_st_x16(o_addr + (uint32_t)cb, v);
           }
           tmem_wait_st();
           l_run *= f;
         }
         m_used = m_new;
       }
-      // the P buffer of this parity is free once the product of two tiles ago has read it
-      if (t >= 2)
-        ok = warp_all(mbar_wait(&sh->pv_done[sb], (uint32_t)((t - 2) >> 1) & 1u, &sh->abort_flag, p.status, 31)) && ok;
-      tc_fence_after();
-      const float bias = -m_used * p.scale_log2;
-      float sum = 0.0f;
-      uint32_t pk[32];
-#pragma unroll
-      for (int e = 0; e < 64; e += 2) {
-        // (a masked score is -inf: exp2 gives 0; a row with nothing to attend yet has m_used = -1e30 and only such scores)
-        const float p0 = fast_exp2(fmaf(__uint_as_float(sv[e]), p.scale_log2, bias));
-        const float p1 = fast_exp2(fmaf(__uint_as_float(sv[e + 1]), p.scale_log2, bias));
-        sum += p0 + p1;
-        pk[e >> 1] = pack_bf16x2(p0, p1);
-      }
-      l_run += sum;
-      tmem_st_x32(lane_base + kColP + (uint32_t)(sb * 64 + half * 32), pk);
-      tmem_wait_st();
+      // P = exp2(scale * (S - m_used)) replaces the scores
+      l_run += masked ? row_prob<true>(s_addr, allowed, p.scale_log2, m_used) : row_prob<false>(s_addr, allowed, p.scale_log2, m_used);
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&sh->p_full[sb]);
-      ++t;
+      if (lane == 0) mbar_arrive(&sh->p_full[grp]);
+      ++n;
     }
-    float acc[64];
-#pragma unroll
-    for (int e = 0; e < 64; ++e) acc[e] = 0.0f;
-    if (ok && t >= 1) {
-      ok = warp_all(mbar_wait(&sh->pv_done[(t - 1) & 1], (uint32_t)((t - 1) >> 1) & 1u, &sh->abort_flag, p.status, 32));
-      tc_fence_after();
-      if (ok) {
-        uint32_t (&lo)[32] = *reinterpret_cast<uint32_t (*)[32]>(&acc[0]);
-        uint32_t (&hi)[32] = *reinterpret_cast<uint32_t (*)[32]>(&acc[32]);
-        tmem_ld_x32(o_addr, lo);
-        tmem_ld_x32(o_addr + 32u, hi);
-        tmem_wait_ld();
-      }
-    }
-    // the two halves of a row add their sums; then O = acc / l, rounded to bf16
+    // this group's last product must have landed before its accumulator is read
+    if (ok && n >= 1) ok = warp_all(mbar_wait(&sh->pv_done[grp], (uint32_t)(n - 1) & 1u, &sh->abort_flag, p.status, 32));
+    tc_fence_after();
+    // merge the two groups: each is a softmax over its own key tiles with its own reference maximum
+    xch[(grp * kTile + row) * 2] = m_used;
+    xch[(grp * kTile + row) * 2 + 1] = l_run;
+    tc_fence_before();
     const bool all_ok = !named_bar_or(1, kSoftmaxThreads, !ok);
-    xch[half * kTile + row] = l_run;
-    named_bar_sync(2, kSoftmaxThreads);
-    const float l_tot = l_run + xch[(half ^ 1) * kTile + row];
-    if (all_ok && i < p.L) {
-      const float inv = 1.0f / l_tot;
-      __nv_bfloat16* dst = p.O + (size_t)i * p.ldo + (size_t)head * kD + half * 64;
+    tc_fence_after();
+    if (all_ok) {
+      // group 0 always has a tile (the diagonal tile is never skipped); group 1 only if two or more were processed
+      const bool two = n_list >= 2;
+      const float m0 = xch[row * 2], l0 = xch[row * 2 + 1];
+      const float m1 = two ? xch[(kTile + row) * 2] : -1.0e30f, l1 = two ? xch[(kTile + row) * 2 + 1] : 0.0f;
+      const float m = fmaxf(m0, m1);
+      const float f0 = fast_exp2((m0 - m) * p.scale_log2), f1 = two ? fast_exp2((m1 - m) * p.scale_log2) : 0.0f;
+      const float inv = fast_rcp(l0 * f0 + l1 * f1);  // (an IEEE division would compile to a subroutine call)
+      // this thread writes head channels 64 grp .. 64 grp + 63 of its row
+      const float w0 = f0 * inv, w1 = f1 * inv;
+      __nv_bfloat16* dst = p.O + (size_t)i * p.ldo + (size_t)head * kD + grp * 64;
 #pragma unroll
-      for (int c8 = 0; c8 < 8; ++c8) {
-        uint32_t w[4];
+      for (int cb = 0; cb < 64; cb += 32) {
+        uint32_t a0[32], a1[32];
+        tmem_ld_x32(lane_base + kColO + (uint32_t)(grp * 64 + cb), a0);
+        if (two) tmem_ld_x32(lane_base + kColO + (uint32_t)(kTile + grp * 64 + cb), a1);
+        tmem_wait_ld();
+        if (i < p.L) {
 #pragma unroll
-        for (int e2 = 0; e2 < 4; ++e2) w[e2] = pack_bf16x2(acc[c8 * 8 + 2 * e2] * inv, acc[c8 * 8 + 2 * e2 + 1] * inv);
-        *reinterpret_cast<uint4*>(dst + c8 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+          for (int c8 = 0; c8 < 4; ++c8) {
+            uint32_t w[4];
+#pragma unroll
+            for (int e2 = 0; e2 < 4; ++e2) {
+              const int e = c8 * 8 + 2 * e2;
+              float x0 = __uint_as_float(a0[e]) * w0, x1 = __uint_as_float(a0[e + 1]) * w0;
+              if (two) {
+                x0 = fmaf(__uint_as_float(a1[e]), w1, x0);
+                x1 = fmaf(__uint_as_float(a1[e + 1]), w1, x1);
+              }
+              w[e2] = pack_bf16x2(x0, x1);
+            }
+            *reinterpret_cast<uint4*>(dst + cb + c8 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+          }
+        }
       }
     }
   }
@@ -424,8 +527,8 @@ aifs_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
   }
 }
 
-constexpr size_t kAttnSmem = 1024 + (1 + 2 * kStages) * (size_t)kTileBytes + sizeof(AttnBarriers) + 2 * 2 * kTile * sizeof(float) +
-                             2 * kTile * sizeof(int32_t);
+constexpr size_t kAttnSmem = 1024 + (1 + 2 * kStages) * (size_t)kTileBytes + sizeof(AttnBarriers) + 2 * kTile * 2 * sizeof(float) +
+                             8 * kTile * sizeof(int32_t) + kMaxTiles * sizeof(int32_t);
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -475,7 +578,7 @@ extern "C" int mq_aifs_attention(const void* Q, int64_t ldq, const void* K, int6
                                  int32_t n_kv_heads, int32_t head_dim, void* O, int64_t ldo, void* ws, size_t ws_bytes,
                                  int32_t* status, void* stream) {
   if (L < 0 || n_q_heads <= 0 || n_kv_heads <= 0 || n_q_heads % n_kv_heads) return MQ_ERR_INVALID_ARG;
-  if (head_dim != kD) return MQ_ERR_UNSUPPORTED;
+  if (head_dim != kD || L > kMaxTiles * kTile) return MQ_ERR_UNSUPPORTED;
   if (ldq < (int64_t)n_q_heads * kD || ldo < (int64_t)n_q_heads * kD || ldk < (int64_t)n_kv_heads * kD ||
       ldv < (int64_t)n_kv_heads * kD)
     return MQ_ERR_INVALID_ARG;

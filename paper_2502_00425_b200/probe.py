@@ -1,10 +1,13 @@
 """Prints the library's tensor-pipe measurements on the current GPU:
 
     python -m paper_2502_00425_b200.probe [--ctas N]
+    python -m paper_2502_00425_b200.probe --attention [--reps R]
 
 1. cycles per tcgen05.mma kind::i8 (128 x N x 32) for several token-tile widths N, accumulator counts and both
    sources of the A operand (mq_ubench_mma_i8), and the int8 operations per clock and SM they amount to;
 2. cycles of the weight expander's inner step (mq_ubench_expand).
+--attention instead times mq_aifs_attention on the 3360-token, three-image sequence with 28 / 4 heads of 128
+(the run that the attention kernel's profile is captured from).
 Timing only: it needs a CUDA device and the built library, computes nothing with the results."""
 from __future__ import annotations
 
@@ -45,11 +48,47 @@ def expand_table(n_iter: int = 2000):
     return rows
 
 
+def attention_run(reps: int):
+    from . import synth
+    is_visual = synth.config3_sequence()
+    L, D, hq, hkv = int(is_visual.shape[0]), 128, 28, 4
+    g = torch.Generator(device="cpu").manual_seed(5)
+    q = torch.randn((L, hq * D), generator=g).to(torch.bfloat16).cuda()
+    k = torch.randn((L, hkv * D), generator=g).to(torch.bfloat16).cuda()
+    v = torch.randn((L, hkv * D), generator=g).to(torch.bfloat16).cuda()
+    o = torch.empty_like(q)
+    perm = torch.empty(L, dtype=torch.int32, device="cuda")
+    dummy = torch.zeros((L, 64), dtype=torch.bfloat16, device="cuda")
+    B.mq_aifs_reorder(dummy, torch.empty_like(dummy), torch.from_numpy(is_visual).cuda(), None, perm,
+                      torch.empty(L, dtype=torch.int32, device="cuda"), torch.zeros(1, dtype=torch.int32, device="cuda"),
+                      direction=0)
+    ws = torch.empty(B.mq_aifs_attention_workspace_bytes(L, hkv), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(2, dtype=torch.int32, device="cuda")
+    run = lambda: B.mq_aifs_attention(q, k, v, perm, None, hq, hkv, o, ws, status)
+    run()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        run()
+    e1.record()
+    torch.cuda.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / reps
+    flops = 4.0 * D * hq * (L * (L + 1) / 2)
+    print("mq_aifs_attention, L = %d, %d / %d heads x %d: %.1f us per call, %.0f TFLOP/s over the allowed pairs, status %s"
+          % (L, hq, hkv, D, us, flops / us / 1e6, status.cpu().tolist()))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--ctas", type=int, default=0, help="CTAs of the MMA microbenchmark (default: one per SM)")
+    ap.add_argument("--attention", action="store_true", help="time the attention kernel instead")
+    ap.add_argument("--reps", type=int, default=5)
     args = ap.parse_args()
     B.load(build_if_missing=True)
+    if args.attention:
+        attention_run(args.reps)
+        return
     ctas = args.ctas or torch.cuda.get_device_properties(0).multi_processor_count
     print("tcgen05.mma kind::i8, 128 x N x 32, %d CTAs" % ctas)
     for r in mma_table(ctas):
