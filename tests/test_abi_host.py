@@ -206,3 +206,28 @@ def test_binding_refuses_cpu_tensors():
     import torch
     with pytest.raises(ValueError):
         B._ptr(torch.zeros(4))
+
+
+def test_attention_entry_point_validates(lib):
+    A = 0x10000
+    at = lib.mq_aifs_attention
+    ws_bytes = B.mq_aifs_attention_workspace_bytes(3360, 4)
+    # V transposed (4 heads x 128 channels x 27 tiles of 128 keys, bf16) + four index bounds per tile
+    assert ws_bytes == 4 * 128 * 27 * 128 * 2 + 512
+    assert B.mq_aifs_attention_workspace_bytes(3360, 4, 64) == 0
+    assert B.mq_aifs_attention_workspace_bytes(0, 4) == 0
+
+    def call(L=256, hq=4, hkv=2, d=128, q=A, ldq=512, ldk=256, ldv=256, ldo=512, perm=A, ws=A, wsb=1 << 30, status=A):
+        return at(q, ldq, A, ldk, A, ldv, perm, None, L, hq, hkv, d, A, ldo, ws, wsb, status, None)
+
+    assert call(L=-1) == B.MQ_ERR_INVALID_ARG
+    assert call(hq=3) == B.MQ_ERR_INVALID_ARG                      # query heads not a multiple of key/value heads
+    assert call(d=64) == B.MQ_ERR_UNSUPPORTED
+    assert call(L=131072 + 1) == B.MQ_ERR_UNSUPPORTED
+    assert call(ldq=256) == B.MQ_ERR_INVALID_ARG                   # pitch shorter than the heads
+    assert call(L=0) == B.MQ_OK                                    # nothing to do
+    assert call(perm=None) == B.MQ_ERR_INVALID_ARG
+    assert call(status=None) == B.MQ_ERR_INVALID_ARG
+    assert call(q=A + 2) == B.MQ_ERR_ALIGNMENT
+    assert call(ldq=516) == B.MQ_ERR_ALIGNMENT
+    assert call(wsb=1024) == B.MQ_ERR_WORKSPACE
