@@ -52,6 +52,8 @@ def _check(o, ref, rows=None, tol=2e-2):
     ([("t", 10), ("v", 200), ("t", 70)], 23, 2, 1),                 # left pads sort with the visual block
     ([("t", 300)], 0, 1, 1),                                        # all text: plain causal attention
     ([("v", 260)], 0, 1, 1),                                        # all visual
+    ([("t", 1)], 0, 2, 1),                                          # a single token
+    ([("v", 100), ("t", 29)], 0, 1, 1),                             # 129 rows: one row in the second tile
 ])
 def test_attention_matches_oracle(spans, pad_left, hq, hkv):
     rng = np.random.default_rng(11)
@@ -91,6 +93,26 @@ def test_attention_config3_shape_sampled_rows():
     o, qb, kb, vb = _run(q[perm], k[perm], v[perm], perm, None, hq, hkv)
     rows = np.unique(np.concatenate([np.arange(0, L, 97), [0, 1, 127, 128, 3071, 3072, 3073, L - 1]]))
     for h in (0, 6, 7, 13, 27):
+        g = h // (hq // hkv)
+        for i in rows:
+            allowed = (perm <= perm[i])[None, :]
+            ref = O.attention(qb[i:i + 1, h * D:(h + 1) * D], kb[:, g * D:(g + 1) * D], vb[:, g * D:(g + 1) * D], allowed)
+            _check(o[i:i + 1, h * D:(h + 1) * D], ref)
+
+
+def test_attention_config4_shape_sampled_rows():
+    """8B-shaped heads (32 query / 8 key-value heads x 128) on one config-4 sequence, [32 text][2304 visual][96 text]:
+    leading text rows sit behind the visual block after AIFS and see only themselves and earlier text."""
+    rng = np.random.default_rng(13)
+    is_visual, _ = _layout([("t", 32), ("v", 2304), ("t", 96)], rng)
+    L, D, hq, hkv = is_visual.shape[0], 128, 32, 8
+    perm = O.aifs_perm(is_visual, None)
+    q = rng.standard_normal((L, hq * D)).astype(np.float32)
+    k = rng.standard_normal((L, hkv * D)).astype(np.float32)
+    v = rng.standard_normal((L, hkv * D)).astype(np.float32)
+    o, qb, kb, vb = _run(q[perm], k[perm], v[perm], perm, None, hq, hkv)
+    rows = np.unique(np.concatenate([np.arange(0, L, 131), [0, 127, 128, 2303, 2304, 2305, 2335, 2336, L - 1]]))
+    for h in (0, 3, 4, 31):
         g = h // (hq // hkv)
         for i in rows:
             allowed = (perm <= perm[i])[None, :]
