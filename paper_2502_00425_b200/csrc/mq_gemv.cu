@@ -7,11 +7,13 @@
 // dedicated W4A8 GEMV kernel (Sec. 4.3, decode table); this is that case.
 //
 // Why not the tensor-core kernel.  With a handful of tokens the product is one pass over the
-// int4 weights, i.e. bounded by HBM.  A tcgen05 MMA with the 128 weight channels as its rows
-// keeps the tensor pipe busy for ~112 cycles per K = 32 step however few token columns it
-// has, which caps a CTA at 8 KB of packed weights per ~450 cycles -- below the HBM rate per
-// SM.  For very few tokens the integer dot-product instruction (dp4a) needs a fraction of the
-// issue slots at the HBM rate, so the CUDA cores are enough and nothing has to be staged.
+// int4 weights, i.e. bounded by HBM, and a launch lasts only a few microseconds.  The tensor-core
+// kernel's CTA takes a whole SM (512 threads, 226 KB of shared memory), so the next launch cannot
+// be resident and prefetching while it runs, and its fixed parts (tensor-memory allocation,
+// pipeline fill, epilogue, the boundary to the next launch) weigh as much as the stream itself;
+// measured, it stays below 3 TB/s on these shapes.  For very few tokens the integer dot-product
+// instruction (dp4a) needs a fraction of the issue slots at the HBM rate, so the CUDA cores are
+// enough, nothing has to be staged, and small CTAs of consecutive launches overlap.
 //
 // Mapping.  A CTA owns 32 consecutive output channels (one quarter of a 128-channel layout
 // tile) and ALL of K; warp w takes the K blocks w, w + W, w + 2W, ...  A lane owns one channel:
