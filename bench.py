@@ -322,7 +322,7 @@ def decode_sweep(torch, B, dev, peaks, n_sets=6, reps=20):
             gbs = w_bytes / sec / 1e9
             res["T%d" % T] = {"us_per_mlp": sec * 1e6, "weight_gbs": gbs, "frac_of_measured_hbm": gbs / peaks["hbm_gbs"],
                               "frac_of_nominal_8tbs": gbs / 8000.0, "per_linear": per_linear,
-                              "kernel": ("w4a8_gemv_kernel (rotation + quantizer + dp4a product in one launch)" if T <= 4 else
+                              "kernel": ("w4a8_gemv_kernel (rotation + quantizer + dp4a product in one launch)" if T <= 3 else
                                          "fwht_quant_kernel + w4a8_gemm_kernel (+ splitk_finalize_kernel when K is split)"),
                               "tokens_per_s": T / sec, "status_ok": all(v == 0 for v in status)}
         out[name] = res

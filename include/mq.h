@@ -257,7 +257,7 @@ int mq_fwht_quant_bits(const void* X, int32_t T, int32_t K, int64_t ldx, const m
  *                       The group sums are folded into float registers after every K block, which costs
  *                       about half of the per-channel kernel's throughput (see DESIGN notes in the source).
  * MQ_FLAG_W8 and group_size = 128 exclude each other (MQ_ERR_UNSUPPORTED).
- * Which kernel runs is an internal choice that does not change the result: one to four
+ * Which kernel runs is an internal choice that does not change the result: one to three
  * rows (single-sequence decode, the case the paper times with a W4A8 GEMV kernel,
  * Sec. 4.3) run rotation, quantizer and a CUDA-core GEMV in ONE kernel; more rows run the
  * quantizer kernel and the tensor-core GEMM (with split-K partial sums in ws for small T).

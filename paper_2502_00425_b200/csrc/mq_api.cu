@@ -270,7 +270,7 @@ int mq_w4a8_msq_linear(const mq_linear_desc* d, const void* X, int64_t ldx, cons
   const int w_bits = (d->flags & MQ_FLAG_W8) ? 8 : 4;
   const bool variant = act_bits != 8 || w_bits != 4 || d->group_size != 0;  // neighbours of the hot path
   if (!variant && !x_i8 && gemv_applies(d->T, d->K, d->N)) {
-    // one to four tokens: a single kernel rotates, quantizes and multiplies (mq_gemv.cu)
+    // one to three tokens: a single kernel rotates, quantizes and multiplies (mq_gemv.cu)
     GemmArgs g{};
     g.T = d->T; g.K = d->K; g.N = d->N;
     g.Xb = X; g.ldx = ldx; g.rot_block = d->rot_block; g.seg = st; g.s_vis = s_vis; g.s_txt = s_txt;
@@ -379,7 +379,7 @@ int mq_w4a8_msq_linear_rms(const mq_linear_desc* d, const void* X, int64_t ldx, 
   uint8_t* wsb = static_cast<uint8_t*>(ws);
   const int sk = rms_side_k(d->K, d->rot_block);
   if (gemv_applies(d->T, d->K, d->N, sk)) {
-    // one to four tokens: rotation, quantizer, both products and the epilogue in one GEMV kernel
+    // one to three tokens: rotation, quantizer, both products and the epilogue in one GEMV kernel
     GemmArgs g{};
     g.T = d->T; g.K = d->K; g.N = d->N;
     g.Xb = X; g.ldx = ldx; g.rot_block = d->rot_block; g.seg = st; g.s_vis = s_vis; g.s_txt = s_txt;

@@ -185,7 +185,7 @@ struct GemmArgs {
   int w_bits;
 };
 int launch_gemm(const GemmArgs& a, cudaStream_t st);
-// one to four tokens: CUDA-core GEMV (mq_gemv.cu); launch_gemm routes there when it applies
+// one to three tokens: CUDA-core GEMV (mq_gemv.cu); launch_gemm routes there when it applies
 bool gemv_applies(int T, int K, int N, int side_k = 0);
 int launch_gemv(const GemmArgs& a, cudaStream_t st);
 size_t gemm_splitk_bytes(int T, int K, int N, bool rms = false, int group_size = 0, int w_bits = 4);

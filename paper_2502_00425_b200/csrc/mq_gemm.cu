@@ -895,8 +895,9 @@ Plan make_plan(int T, int K, int N, int mode = kPlain) {
     ksplit = (kb_total + per - 1) / per;  // no empty split
     // Splitting pays only while the partial sums are small: each split writes a [T,N] int32 slice
     // that the finalize kernel reads back (about 4 TB/s for the pair), and that kernel costs
-    // about 3 us on top.  Against it stands the main loop, 4 MMAs of ~112 cycles per K block at
-    // ~1.9 GHz.  (Decode shapes split; a prefill-sized T with few output channels does not.)
+    // about 3 us on top.  Against it stands the main loop, whose K blocks follow one another every ~450
+    // cycles (the pipeline's measured period for small token tiles) at ~1.9 GHz.  (Decode shapes split; a
+    // prefill-sized T with few output channels does not.)
     const double loop_us = kb_total * 4.0 * 112.0 / 1900.0;
     const double slices_us = (ksplit + 0.5) * (double)T * N * 4.0 * 2.0 / 4.0e6 + 3.0;
     if (loop_us / ksplit + slices_us >= loop_us) ksplit = 1;
@@ -944,7 +945,7 @@ int launch_gemm(const GemmArgs& a, cudaStream_t st) {
   const int mode = mode_of(rms, a.group_size, a.w_bits);
   if (rms && (a.group_size || a.w_bits == 8)) return MQ_ERR_UNSUPPORTED;
   if (a.group_size && (a.group_size != kBlockK || a.K % kBlockK || a.row_scales || a.w_bits == 8)) return MQ_ERR_UNSUPPORTED;
-  if (mode == kPlain && gemv_applies(a.T, a.K, a.N)) return launch_gemv(a, st);  // one to four tokens: see mq_gemv.cu
+  if (mode == kPlain && gemv_applies(a.T, a.K, a.N)) return launch_gemv(a, st);  // one to three tokens: see mq_gemv.cu
   const Plan pl = make_plan(a.T, a.K, a.N, mode);
   EncodeTiledFn encode = get_encode_fn();
   if (!encode) return MQ_ERR_CUDA;

@@ -1,4 +1,4 @@
-// K2v: the W4A8 linear for one to four tokens (single-sequence decode) as a GEMV on the
+// K2v: the W4A8 linear for one to three tokens (single-sequence decode) as a GEMV on the
 // CUDA cores, with rotation and quantizer in the same kernel.
 //
 // Method: the same arithmetic as the quantizer + GEMM pair (Fig. 4(a), App. A.3, Eq. 2, Eq. 3):
@@ -19,7 +19,7 @@
 // tile) and ALL of K; warp w takes the K blocks w, w + W, w + 2W, ...  A lane owns one channel:
 // its 32 codes of a K = 32 piece are one 16-byte load, and the 32 lanes of a warp read 512
 // contiguous bytes of the layout tile.  The weights of the next K block are in flight while
-// the current one is multiplied.  The int8 activation codes of the (up to four) tokens sit
+// the current one is multiplied.  The int8 activation codes of the (up to three) tokens sit
 // in shared memory; every lane reads the same address (broadcast).  With bf16 input every
 // CTA rotates and quantizes the few rows for itself (the quantizer kernel's own warp routine),
 // which removes one kernel boundary -- about 2 us, as much as the weights of a 4096 x 13696
@@ -41,7 +41,7 @@
 namespace mq {
 namespace {
 
-constexpr int kGemvMaxT = 4;
+constexpr int kGemvMaxT = 3;   // at four tokens the tensor-core kernel is faster (measured: 31.8 vs 34.1 us per MLP pass)
 constexpr int kGemvMaxWarps = 32;
 constexpr int kGemvWarpsPerSm = 24;
 constexpr int kGemvSmemLimit = 200 * 1024;
@@ -283,7 +283,7 @@ w4a8_gemv_kernel(const GemvParams p) {
 }
 
 size_t gemv_smem(int T, int K, int warps, int side_k = 0) {
-  const int tt = T <= 1 ? 1 : (T <= 2 ? 2 : 4);
+  const int tt = T <= 1 ? 1 : (T <= 2 ? 2 : 3);
   const size_t kpad = (size_t)((K + MQ_W_TILE_K - 1) / MQ_W_TILE_K) * MQ_W_TILE_K;
   const size_t side_pad = (size_t)((side_k + MQ_W_TILE_K - 1) / MQ_W_TILE_K) * MQ_W_TILE_K;
   return (size_t)tt * kpad + (size_t)warps * tt * 32 * sizeof(int32_t) + (size_t)tt * side_pad;
@@ -326,7 +326,7 @@ int launch_gemv(const GemmArgs& a, cudaStream_t st) {
   if (warps > p.kb_total) warps = p.kb_total;
   if (warps < 1) warps = 1;
   const size_t smem = gemv_smem(a.T, a.K, warps, a.side_layout ? a.side_k : 0);
-  auto kernel = a.T <= 1 ? w4a8_gemv_kernel<1> : (a.T <= 2 ? w4a8_gemv_kernel<2> : w4a8_gemv_kernel<4>);
+  auto kernel = a.T <= 1 ? w4a8_gemv_kernel<1> : (a.T <= 2 ? w4a8_gemv_kernel<2> : w4a8_gemv_kernel<3>);
   static PerDeviceTable<char> attr_set[3];
   const int ki = a.T <= 1 ? 0 : (a.T <= 2 ? 1 : 2);
   if (!ensure_dynamic_smem(attr_set[ki], kernel, kGemvSmemLimit)) return MQ_ERR_CUDA;

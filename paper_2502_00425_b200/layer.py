@@ -222,7 +222,7 @@ class W4A8DecoderBlock:
             B.mq_calibrate_static_scales(x, tr.seg, 0, state, sv, st)
             for n in names:
                 self.w[n].s_vis, self.w[n].s_txt = float(sv.item()), float(st.item())
-        if T <= 4:  # the few-token kernel quantizes inside: nothing to share
+        if T <= 3:  # the few-token kernel quantizes inside: nothing to share
             return [self.linear(n, x, tr, False) for n in names]
         codes = torch.empty((T, first.K), dtype=torch.int8, device=x.device)
         B.mq_fwht_quant_i8(x, tr.seg, first.s_vis, first.s_txt, 0, codes, None)

@@ -273,14 +273,15 @@ def test_linear_edge_shapes(T_vis, T_txt, K, N, rot):
 @pytest.mark.parametrize("T_vis,T_txt,K,N,rot", [
     (0, 1, 4096, 272, 128),    # one token, ragged last channel quarter (N % 32 = 16), 32 K blocks
     (1, 1, 160, 144, 32),      # two tokens of different modality, K not a multiple of the K block
-    (1, 2, 1152, 528, 128),    # three tokens in the four-token variant, nine K blocks
-    (2, 2, 13696, 64, 128),    # four tokens, 107 K blocks over 32 warps, 14 warp passes per row
+    (1, 2, 1152, 528, 128),    # three tokens, nine K blocks
+    (2, 2, 13696, 64, 128),    # four tokens: the first count that takes the tensor-core path (split K, 107 K blocks)
+    (1, 2, 13696, 64, 128),    # three tokens, 107 K blocks over 32 warps, 14 warp passes per row
     (0, 1, 32, 16, 0),         # one K piece, half a channel quarter
     (1, 1, 2048, 96, 1024),    # the largest rotation block (a whole warp pass)
     (0, 2, 512, 48, 64),       # rotation 64
 ])
 def test_linear_gemv_shapes(T_vis, T_txt, K, N, rot):
-    # T <= 4 runs the CUDA-core GEMV (mq_gemv.cu): with bf16 input it rotates and quantizes in the
+    # T <= 3 runs the CUDA-core GEMV (mq_gemv.cu): with bf16 input it rotates and quantizes in the
     # same kernel, with int8 input it only multiplies; _check_linear exercises both
     c = synth.small_linear(500 + K + N + T_vis, T_vis, T_txt, K, N, rot, calib_vis=24, calib_txt=8)
     bias = (np.random.default_rng(2).standard_normal(N)).astype(np.float32)
