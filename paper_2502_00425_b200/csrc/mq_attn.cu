@@ -12,14 +12,14 @@
 // kind::f16 on bf16 operands from shared memory, float32 accumulators in tensor memory):
 //   * Q, K tiles and V^T tiles arrive by TMA (128-byte swizzle).  V is transposed once per call by a small
 //     prep kernel so that the second product's B operand is K-major like every other operand here;
-//   * the key tiles a query tile has to process go alternately to two groups of four softmax warps.  Each
-//     group has its own score buffer and its own output accumulator in tensor memory and runs a complete
-//     online softmax over its tiles; the two partial results are merged at the end (as for a split over
-//     the keys).  While one group works on its scores the tensor cores compute the other group's;
-//   * a softmax thread owns one query row: it reads its 128 scores from tensor memory (once for the row
-//     maximum, once for the exponentials), applies the mask and writes P = exp2(...) as bf16 over the
-//     scores it has read, where the second product takes it as its A operand: the probabilities never
-//     touch shared memory;
+//   * two groups of four softmax warps share every key tile: group 0 takes its keys 0 .. 63, group 1 its keys
+//     64 .. 127.  Each group has two score buffers (128 x 64) and its own output accumulator in tensor memory
+//     and runs a complete online softmax over its keys; the two partial results are merged at the end (as
+//     for a split over the keys).  With two buffers a group's scores for the next tile are computed while
+//     its softmax works on the current one;
+//   * a softmax thread owns one query row: it reads its 64 scores from tensor memory once, applies the
+//     mask, takes the maximum and writes P = exp2(...) as bf16 over the scores it has read, where the second
+//     product takes it as its A operand: the probabilities never touch shared memory;
 //   * O_g += P V accumulates in tensor memory.  The exponents are taken relative to a reference maximum
 //     that may lag the true running maximum by up to 8 powers of two; only when a row outgrows it are the
 //     accumulated output and sum rescaled, so the softmax warps normally never touch O until the end;
@@ -52,9 +52,9 @@ constexpr int kStages = 2;                   // K tiles and V^T tiles in flight 
 struct AttnBarriers {
   uint64_t q_full;
   uint64_t k_full[kStages], k_empty[kStages], v_full[kStages], v_empty[kStages];
-  // per softmax group: its score buffer is written (MMA commit); P has replaced the scores (the group's four
-  // warps); the product of that P into the group's accumulator is complete (MMA commit)
-  uint64_t s_full[2], p_full[2], pv_done[2];
+  // per softmax group and score buffer ([2 g + b]): the scores are written (MMA commit); P has replaced them (the
+  // group's four warps); the product of that P into the group's accumulator is complete (MMA commit)
+  uint64_t s_full[4], p_full[4], pv_done[4];
   uint64_t drain;
   uint32_t tmem_base;
   int abort_flag;
@@ -153,104 +153,64 @@ attn_prep_kernel(const uint16_t* __restrict__ V, int64_t ldv, int L, int Lp, con
 }
 
 // ---------------------------------------------------------------------------------------- softmax pieces
-// A thread's 128 scores are read from tensor memory in four chunks of 32 columns; the load of the next chunk is
-// in flight while the current one is worked on (two register buffers), because a tensor-memory load takes a few
-// hundred cycles and only two softmax warps share a scheduler.
+// A softmax thread works on one query row and the 64 key columns of its group's half of a key tile.  Both
+// 32-column loads of the scores are in flight together and the scores stay in registers for the maximum and
+// the exponentials (one read of tensor memory per tile).
 //
-// Maximum of one chunk into four independent partial maxima (a single chain of 128 dependent max operations
-// would cost more than the exponentials).
+// Loads the 64 scores at s_addr, masks them (-inf where the row may not attend the key), returns the maximum.
 template <bool MASKED>
-__device__ __forceinline__ void chunk_max(const uint32_t (&v)[32], uint32_t allowed, float (&mx)[4]) {
-#pragma unroll
-  for (int e = 0; e < 32; ++e) {
-    const float x = __uint_as_float(v[e]);
-    if (!MASKED || ((allowed >> e) & 1u)) mx[e & 3] = fmaxf(mx[e & 3], x);
-  }
-}
-
-// P = exp2(scale * s + bias) of one chunk as 16 bf16 pairs; adds the chunk's probabilities into two packed sums.
-template <bool MASKED>
-__device__ __forceinline__ void chunk_prob(const uint32_t (&v)[32], uint32_t allowed, float2 scale2, float2 bias2,
-                                           float2 (&sum2)[2], uint32_t (&pk)[16]) {
-#pragma unroll
-  for (int e = 0; e < 32; e += 2) {
-    const float2 x = __ffma2_rn(make_float2(__uint_as_float(v[e]), __uint_as_float(v[e + 1])), scale2, bias2);
-    float2 pr = make_float2(fast_exp2(x.x), fast_exp2(x.y));
-    if (MASKED) {
-      if (!((allowed >> e) & 1u)) pr.x = 0.0f;
-      if (!((allowed >> (e + 1)) & 1u)) pr.y = 0.0f;
-    }
-    sum2[(e >> 1) & 1] = __fadd2_rn(sum2[(e >> 1) & 1], pr);
-    pk[e >> 1] = pack_bf16x2(pr.x, pr.y);
-  }
-}
-
-// Row maximum of the 128 scores at s_addr.
-template <bool MASKED>
-__device__ __forceinline__ float row_max(uint32_t s_addr, const uint32_t (&allowed)[4]) {
+__device__ __forceinline__ float scores_load_max(uint32_t s_addr, uint32_t allowed_lo, uint32_t allowed_hi, uint32_t (&sv)[64]) {
+  tmem_ld_x32(s_addr, *reinterpret_cast<uint32_t (*)[32]>(&sv[0]));
+  tmem_ld_x32(s_addr + 32u, *reinterpret_cast<uint32_t (*)[32]>(&sv[32]));
+  tmem_wait_ld();
+  // four independent partial maxima (one chain of dependent max operations would cost more than the exponentials)
   float mx[4] = {-1.0e30f, -1.0e30f, -1.0e30f, -1.0e30f};
-  uint32_t a[32], b[32];
-  tmem_ld_x32(s_addr, a);
-  tmem_wait_ld();
-  tmem_ld_x32(s_addr + 32u, b);
-  chunk_max<MASKED>(a, allowed[0], mx);
-  tmem_wait_ld();
-  tmem_ld_x32(s_addr + 64u, a);
-  chunk_max<MASKED>(b, allowed[1], mx);
-  tmem_wait_ld();
-  tmem_ld_x32(s_addr + 96u, b);
-  chunk_max<MASKED>(a, allowed[2], mx);
-  tmem_wait_ld();
-  chunk_max<MASKED>(b, allowed[3], mx);
+#pragma unroll
+  for (int e = 0; e < 64; ++e) {
+    if (MASKED && !(((e < 32 ? allowed_lo : allowed_hi) >> (e & 31)) & 1u)) sv[e] = 0xff800000u;  // -inf: its exponential is 0
+    mx[e & 3] = fmaxf(mx[e & 3], __uint_as_float(sv[e]));
+  }
   return fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
 }
 
-// The 128 probabilities of the row, written as bf16 pairs over the first 64 columns of the score buffer; every
-// store lands on columns whose scores this thread has already consumed.  Returns the row sum.
-template <bool MASKED>
-__device__ __forceinline__ float row_prob(uint32_t s_addr, const uint32_t (&allowed)[4], float scale_log2, float m_used) {
+// P = exp2(scale * (s - m_used)) of the 64 scores as 32 bf16 pairs over the first 32 columns of the score buffer
+// (all of whose scores are in registers by now).  Returns the sum of the probabilities.
+__device__ __forceinline__ float probs_store(uint32_t s_addr, const uint32_t (&sv)[64], float scale_log2, float m_used) {
   const float2 scale2 = make_float2(scale_log2, scale_log2);
   const float bias = -m_used * scale_log2;
   const float2 bias2 = make_float2(bias, bias);
   float2 sum2[2] = {make_float2(0.0f, 0.0f), make_float2(0.0f, 0.0f)};
-  uint32_t a[32], b[32], pk[16];
-  tmem_ld_x32(s_addr, a);
-  tmem_wait_ld();
-  tmem_ld_x32(s_addr + 32u, b);
-  chunk_prob<MASKED>(a, allowed[0], scale2, bias2, sum2, pk);
-  tmem_st_x16(s_addr, pk);
-  tmem_wait_ld();
-  tmem_ld_x32(s_addr + 64u, a);
-  chunk_prob<MASKED>(b, allowed[1], scale2, bias2, sum2, pk);
-  tmem_st_x16(s_addr + 16u, pk);
-  tmem_wait_ld();
-  tmem_ld_x32(s_addr + 96u, b);
-  chunk_prob<MASKED>(a, allowed[2], scale2, bias2, sum2, pk);
-  tmem_st_x16(s_addr + 32u, pk);
-  tmem_wait_ld();
-  chunk_prob<MASKED>(b, allowed[3], scale2, bias2, sum2, pk);
-  tmem_st_x16(s_addr + 48u, pk);
+  uint32_t pk[32];
+#pragma unroll
+  for (int e = 0; e < 64; e += 2) {
+    const float2 x = __ffma2_rn(make_float2(__uint_as_float(sv[e]), __uint_as_float(sv[e + 1])), scale2, bias2);
+    const float2 pr = make_float2(fast_exp2(x.x), fast_exp2(x.y));
+    sum2[(e >> 1) & 1] = __fadd2_rn(sum2[(e >> 1) & 1], pr);
+    pk[e >> 1] = pack_bf16x2(pr.x, pr.y);
+  }
+  tmem_st_x32(s_addr, pk);
   tmem_wait_st();
   return (sum2[0].x + sum2[0].y) + (sum2[1].x + sum2[1].y);
 }
 
-// Bit j of the result: may this thread's row attend key column j of the tile (kp: the keys' original indices,
-// INT_MAX for padded or out-of-range keys; self_col: the diagonal column of a padded row, or -1).
-__device__ __forceinline__ void allowed_bits(const int32_t* kp, int perm_i, int self_col, uint32_t (&allowed)[4]) {
-#pragma unroll
-  for (int c = 0; c < 4; ++c) {
-    uint32_t w = 0;
+// Bit j of (lo, hi): may this thread's row attend key column j of its group's half tile (kp: the 64 keys'
+// original indices, INT_MAX for padded or out-of-range keys; self_col: the diagonal column of a padded row, or -1).
+__device__ __forceinline__ void allowed_bits(const int32_t* kp, int perm_i, int self_col, uint32_t& lo, uint32_t& hi) {
+  lo = 0; hi = 0;
 #pragma unroll 8
-    for (int b = 0; b < 32; ++b) w |= (uint32_t)(kp[c * 32 + b] <= perm_i) << b;
-    allowed[c] = w;
+  for (int b = 0; b < 32; ++b) lo |= (uint32_t)(kp[b] <= perm_i) << b;
+#pragma unroll 8
+  for (int b = 0; b < 32; ++b) hi |= (uint32_t)(kp[32 + b] <= perm_i) << b;
+  if (self_col >= 0) {
+    if (self_col < 32) lo |= 1u << self_col;
+    else hi |= 1u << (self_col - 32);
   }
-  if (self_col >= 0) allowed[self_col >> 5] |= 1u << (self_col & 31);
 }
 
 // ---------------------------------------------------------------------------------------- the kernel
-// Tensor-memory columns: group g (0: the even, 1: the odd processed key tiles) has its score buffer at 128 g --
-// whose first 64 columns are overwritten in place by P (bf16 pairs) once the scores have been read -- and
-// its output accumulator at 256 + 128 g.
+// Tensor-memory columns: group g (0: keys 0 .. 63 of every key tile, 1: keys 64 .. 127) has two score buffers of
+// 64 columns at 128 g and 128 g + 64 -- the first 32 columns of a buffer are overwritten in place by P (bf16
+// pairs) once its scores have been read -- and its output accumulator at 256 + 128 g.
 constexpr uint32_t kColO = 256;
 // The exponent's reference maximum may lag the true running maximum by this many powers of two before the
 // accumulated output is rescaled (probabilities then reach at most 2^8, harmless in float32 / bf16).
@@ -285,7 +245,7 @@ aifs_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
       mbar_init(&sh->k_full[i], 1); mbar_init(&sh->k_empty[i], 1);
       mbar_init(&sh->v_full[i], 1); mbar_init(&sh->v_empty[i], 1);
     }
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < 4; ++i) {   // [group][buffer]
       mbar_init(&sh->s_full[i], 1); mbar_init(&sh->p_full[i], 4); mbar_init(&sh->pv_done[i], 1);
     }
     mbar_init(&sh->drain, 1);
@@ -354,51 +314,59 @@ aifs_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
       }
     }
   } else if (warp == 1) {
-    // ---------------- MMA issuer.  Processed tile u belongs to group u & 1.  S_u = Q K_u^T is issued one tile
-    // ahead of O_g += P_{u-1} V_{u-1}, so the tensor cores work on the other group's scores while one group's
-    // softmax runs.  S_u overwrites the buffer P_{u-2} is read from by the product issued just before it: the
-    // MMAs of one thread execute in the order they were issued, so no wait is needed between the two.
+    // ---------------- MMA issuer.  Per key tile t: the scores of both groups (S_g = Q K_g^T, 128 x 64, into the
+    // group's buffer t & 1), then the products of tile t - 1 (O_g += P_g V_g).  A group's scores for tile t + 1
+    // are therefore computed while its softmax works on tile t.  S_g(t) overwrites the buffer P_g(t - 2) is read
+    // from by a product issued before it: the MMAs of one thread execute in the order they were issued, so no
+    // wait is needed between the two.
     if (elect_one()) {
-      const uint32_t idesc = make_idesc_bf16(kTile);
+      const uint32_t idesc_s = make_idesc_bf16(64);      // 128 rows x 64 keys
+      const uint32_t idesc_o = make_idesc_bf16(kTile);   // 128 rows x 128 head channels
       const uint64_t qdesc = make_b_desc(smem_u32(q_smem));
       bool ok = mbar_wait(&sh->q_full, 0, &sh->abort_flag, p.status, 23);
-      int t = 0, ks = 0, vs = 0;       // tile count; ring positions of the next K and the next V tile
+      int ks = 0, vs = 0;       // ring positions of the next K and the next V tile
       uint32_t kph = 0, vph = 0;
       auto issue_pv = [&](int u) -> bool {
-        const int grp = u & 1, n = u >> 1;
+        const int b = u & 1;
+        const uint32_t par = (uint32_t)(u >> 1) & 1u;
         if (!mbar_wait(&sh->v_full[vs], vph, &sh->abort_flag, p.status, 24)) return false;
-        if (!mbar_wait(&sh->p_full[grp], (uint32_t)n & 1u, &sh->abort_flag, p.status, 25)) return false;
-        tc_fence_after();
         const uint64_t vdesc = make_b_desc(smem_u32(v_smem + vs * kTileBytes));
-        const uint32_t p_tmem = tmem_base + (uint32_t)(grp * kTile);
-        const uint32_t o_tmem = tmem_base + kColO + (uint32_t)(grp * kTile);
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-          const uint64_t off = (uint64_t)((k >> 2) * (kHalfBytes >> 4) + (k & 3) * 2);
-          mma_bf16_ts(o_tmem, p_tmem + (uint32_t)(k * 8), vdesc + off, idesc, (n > 0 || k > 0) ? 1u : 0u);
+        for (int grp = 0; grp < 2; ++grp) {
+          if (!mbar_wait(&sh->p_full[2 * grp + b], par, &sh->abort_flag, p.status, 25)) return false;
+          tc_fence_after();
+          const uint32_t p_tmem = tmem_base + (uint32_t)(grp * kTile + b * 64);
+          const uint32_t o_tmem = tmem_base + kColO + (uint32_t)(grp * kTile);
+#pragma unroll
+          for (int k = 0; k < 4; ++k)   // the group's 64 keys: key block grp of the V^T tile
+            mma_bf16_ts(o_tmem, p_tmem + (uint32_t)(k * 8), vdesc + (uint64_t)(grp * (kHalfBytes >> 4) + k * 2), idesc_o,
+                        (u > 0 || k > 0) ? 1u : 0u);
+          tc_commit(&sh->pv_done[2 * grp + b]);
         }
-        tc_commit(&sh->pv_done[grp]);
         tc_commit(&sh->v_empty[vs]);
         if (++vs == kStages) { vs = 0; vph ^= 1u; }
         return true;
       };
-      for (int idx = 0; idx < n_list && ok; ++idx) {
-        const int grp = t & 1;
+      for (int t = 0; t < n_list && ok; ++t) {
+        const int b = t & 1;
         if (!(ok = mbar_wait(&sh->k_full[ks], kph, &sh->abort_flag, p.status, 27))) break;
         tc_fence_after();
         const uint64_t kdesc = make_b_desc(smem_u32(k_smem + ks * kTileBytes));
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-          const uint64_t off = (uint64_t)((k >> 2) * (kHalfBytes >> 4) + (k & 3) * 2);
-          mma_bf16_ss(tmem_base + (uint32_t)(grp * kTile), qdesc + off, kdesc + off, idesc, k ? 1u : 0u);
+        for (int grp = 0; grp < 2; ++grp) {
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {   // head channels 16 k ..: channel block k >> 2; key rows 64 grp .. of the K tile
+            const uint64_t off = (uint64_t)((k >> 2) * (kHalfBytes >> 4) + (k & 3) * 2);
+            mma_bf16_ss(tmem_base + (uint32_t)(grp * kTile + b * 64), qdesc + off, kdesc + off + (uint64_t)(grp * (64 * 128 >> 4)),
+                        idesc_s, k ? 1u : 0u);
+          }
+          tc_commit(&sh->s_full[2 * grp + b]);
         }
-        tc_commit(&sh->s_full[grp]);
         tc_commit(&sh->k_empty[ks]);
         if (++ks == kStages) { ks = 0; kph ^= 1u; }
         if (t >= 1 && !(ok = issue_pv(t - 1))) break;
-        ++t;
       }
-      if (ok && t >= 1) ok = issue_pv(t - 1);
+      if (ok && n_list >= 1) ok = issue_pv(n_list - 1);
       if (!ok) {  // let every MMA already issued finish before tensor memory is freed
         tc_commit(&sh->drain);
         mbar_wait_drain(&sh->drain, 0, 2000000ull);
@@ -406,49 +374,53 @@ aifs_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
     }
     __syncwarp();
   } else if (warp >= 4) {
-    // ---------------- softmax warps.  Group grp = warps 4 + 4 grp .. 7 + 4 grp takes every second processed key
-    // tile; its thread `row` owns query row q0 + row with all 128 columns of the group's score buffer and keeps
-    // that row's reference maximum and sum over the group's tiles.  A warp depends on no other softmax warp
-    // until the two groups' partial results are merged at the end.
+    // ---------------- softmax warps.  Group grp = warps 4 + 4 grp .. 7 + 4 grp takes keys 64 grp .. 64 grp + 63 of
+    // every processed key tile; its thread `row` owns query row q0 + row and keeps that row's reference maximum and
+    // sum over the group's keys.  A warp depends on no other softmax warp until the two groups' partial results are
+    // merged at the end.
     const int quarter = warp & 3, grp = (warp - 4) >> 2;
     const int row = quarter * 32 + lane;
     const int i = q0 + row;
     const int perm_i = i < p.L ? p.perm[i] : -1;
     const bool pad_i = i < p.L && p.pad_u && p.pad_u[i];
     const uint32_t lane_base = tmem_base + ((uint32_t)(quarter * 32) << 16);
-    const uint32_t s_addr = lane_base + (uint32_t)(grp * kTile);
     const uint32_t o_addr = lane_base + kColO + (uint32_t)(grp * kTile);
-    int32_t* kp = kp_all + (warp - 4) * kTile;       // this warp's copy of the key tile's original indices
+    int32_t* kp = kp_all + (warp - 4) * kTile;       // this warp's copy of its 64 keys' original indices
     const float lag_raw = kLagLog2 * fast_rcp(p.scale_log2);   // the lag in units of the raw scores
     float m_used = -1.0e30f, l_run = 0.0f;           // reference maximum of the exponents; sum relative to it
-    int n = 0;                                       // this group's tiles so far
     bool ok = true;
-    for (int idx = grp; idx < n_list && ok; idx += 2) {
-      const int kt = tile_list[idx] & 0xffff;
-      const bool masked = (tile_list[idx] >> 16) == 1;
-      // a padded row attends itself: the column of the diagonal, if this is the diagonal tile
-      const int self_col = (pad_i && kt == qt) ? row : -1;
+    for (int t = 0; t < n_list && ok; ++t) {
+      const int kt = tile_list[t] & 0xffff;
+      const bool masked = (tile_list[t] >> 16) == 1;
+      const int b = t & 1;
+      const uint32_t par = (uint32_t)(t >> 1) & 1u;
+      uint32_t allowed_lo = ~0u, allowed_hi = ~0u;
       if (masked) {
         __syncwarp();
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          const int j = kt * kTile + c * 32 + lane;
+        for (int c = 0; c < 2; ++c) {
+          const int j = kt * kTile + grp * 64 + c * 32 + lane;
           kp[c * 32 + lane] = (j < p.L && !(p.pad_u && p.pad_u[j])) ? p.perm[j] : INT_MAX;
         }
         __syncwarp();
+        // a padded row attends itself: the column of the diagonal, if it lies in this group's half of the diagonal tile
+        const int self_col = (pad_i && kt == qt && (row >> 6) == grp) ? (row & 63) : -1;
+        allowed_bits(kp, perm_i, self_col, allowed_lo, allowed_hi);
       }
-      if (!(ok = warp_all(mbar_wait(&sh->s_full[grp], (uint32_t)n & 1u, &sh->abort_flag, p.status, 29)))) break;
+      if (!(ok = warp_all(mbar_wait(&sh->s_full[2 * grp + b], par, &sh->abort_flag, p.status, 29)))) break;
       tc_fence_after();
-      // the scores, masked, and the row maximum
-      uint32_t allowed[4] = {~0u, ~0u, ~0u, ~0u};
-      if (masked) allowed_bits(kp, perm_i, self_col, allowed);
-      const float mx = masked ? row_max<true>(s_addr, allowed) : row_max<false>(s_addr, allowed);
+      const uint32_t s_addr = lane_base + (uint32_t)(grp * kTile + b * 64);
+      uint32_t sv[64];
+      const float mx = masked ? scores_load_max<true>(s_addr, allowed_lo, allowed_hi, sv)
+                              : scores_load_max<false>(s_addr, allowed_lo, allowed_hi, sv);
       const float m_new = fmaxf(m_used, mx);
       // move the reference maximum only when some row of this warp has outgrown it; then the accumulated output
       // and sum of the warp's rows are rescaled
       if (__any_sync(0xffffffffu, m_new > m_used + lag_raw)) {
-        if (n >= 1) {
-          if (!(ok = warp_all(mbar_wait(&sh->pv_done[grp], (uint32_t)(n - 1) & 1u, &sh->abort_flag, p.status, 30)))) break;
+        if (t >= 1) {
+          // the product of the previous tile (and with it every earlier one) must have landed in the accumulator
+          if (!(ok = warp_all(mbar_wait(&sh->pv_done[2 * grp + ((t - 1) & 1)], (uint32_t)((t - 1) >> 1) & 1u, &sh->abort_flag,
+                                        p.status, 30)))) break;
           tc_fence_after();
           const float f = fast_exp2((m_used - m_new) * p.scale_log2);
 #pragma unroll
@@ -466,14 +438,15 @@ aifs_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
         m_used = m_new;
       }
       // P = exp2(scale * (S - m_used)) replaces the scores
-      l_run += masked ? row_prob<true>(s_addr, allowed, p.scale_log2, m_used) : row_prob<false>(s_addr, allowed, p.scale_log2, m_used);
+      l_run += probs_store(s_addr, sv, p.scale_log2, m_used);
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&sh->p_full[grp]);
-      ++n;
+      if (lane == 0) mbar_arrive(&sh->p_full[2 * grp + b]);
     }
+    const int n = n_list;   // both groups work on every processed tile
     // this group's last product must have landed before its accumulator is read
-    if (ok && n >= 1) ok = warp_all(mbar_wait(&sh->pv_done[grp], (uint32_t)(n - 1) & 1u, &sh->abort_flag, p.status, 32));
+    if (ok && n >= 1)
+      ok = warp_all(mbar_wait(&sh->pv_done[2 * grp + ((n - 1) & 1)], (uint32_t)((n - 1) >> 1) & 1u, &sh->abort_flag, p.status, 32));
     tc_fence_after();
     // merge the two groups: each is a softmax over its own key tiles with its own reference maximum
     xch[(grp * kTile + row) * 2] = m_used;
@@ -482,8 +455,8 @@ aifs_attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
     const bool all_ok = !named_bar_or(1, kSoftmaxThreads, !ok);
     tc_fence_after();
     if (all_ok) {
-      // group 0 always has a tile (the diagonal tile is never skipped); group 1 only if two or more were processed
-      const bool two = n_list >= 2;
+      // (the diagonal tile is never skipped, so both groups have worked on at least one tile)
+      constexpr bool two = true;
       const float m0 = xch[row * 2], l0 = xch[row * 2 + 1];
       const float m1 = two ? xch[(kTile + row) * 2] : -1.0e30f, l1 = two ? xch[(kTile + row) * 2 + 1] : 0.0f;
       const float m = fmaxf(m0, m1);
