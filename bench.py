@@ -492,9 +492,10 @@ def layer_mode_timing(torch, dev, name, shape, seqs, reps=5):
             "status_ok": blk.device_status_ok()}
 
 
-def attention_timing(torch, B, dev, reps=10):
+def attention_timing(torch, B, dev, peaks, reps=10):
     """mq_aifs_attention alone on the sequences of configs 3 and 4 (one sequence per call) and on a long text-only
-    sequence: microseconds and TFLOP/s over the multiply-adds the mask allows (4 * D * allowed pairs * heads)."""
+    sequence: microseconds and TFLOP/s over the multiply-adds the mask allows (4 * D * allowed pairs * heads), and
+    that rate as a fraction of the measured dense bf16 rate (the kernel's products are bf16 tensor-core MMAs)."""
     from paper_2502_00425_b200 import synth as SY
     out = {}
     cases = [("config3 sequence: [img 1024][txt 96] x 3, 28 / 4 heads", SY.interleaved_modality([(1, 1024), (0, 96)] * 3), 28, 4),
@@ -526,7 +527,9 @@ def attention_timing(torch, B, dev, reps=10):
         torch.cuda.synchronize()
         us = e0.elapsed_time(e1) * 1e3 / reps
         flops = 4.0 * D * hq * (L * (L + 1) / 2)
-        out[name] = {"L": L, "us": us, "tflops_allowed_pairs": flops / us / 1e6, "status_ok": status.tolist() == [0, 0]}
+        out[name] = {"L": L, "us": us, "tflops_allowed_pairs": flops / us / 1e6,
+                     "frac_of_measured_bf16_burst": flops / us / 1e6 / peaks["bf16_burst"], "bound": "tensor (bf16)",
+                     "status_ok": status.tolist() == [0, 0]}
     return out
 
 
@@ -944,7 +947,7 @@ def run_ours(args, info):
                   layer_mode_timing(torch, dev, "config4: 8B-shaped block, 4 sequences of 2432 tokens",
                                     synth.LLAMA_8B, [synth.config4_sequence()] * 4)]
         torch.cuda.empty_cache()
-        attn_timing = attention_timing(torch, B, dev)
+        attn_timing = attention_timing(torch, B, dev, peaks)
 
     # ---- CPU baseline: the oracle on this host (rank 0, N = 1 only)
     cpu = None
